@@ -1,0 +1,415 @@
+/*
+ * CPU oracle for arithmetic sampling -- TEST INFRASTRUCTURE, not a product path.
+ *
+ * A plain, slow, fp64 restatement of decoding a code point against a
+ * next-token distribution, written from the paper (Vilnis et al.,
+ * "Arithmetic Sampling", arXiv 2210.15458).  Only the tests, the smoke check
+ * and the benchmark's CPU-baseline leg may call it.  It shares no code with
+ * the CUDA library.
+ *
+ * What each function follows:
+ *   orc_lattice_codes     Definition "Arithmetic sampling" (Sec. 4.2) and Eq. 2:
+ *                         a regular lattice with one shared uniform shift,
+ *                         taken modulo 1; spacing 1/N so that every gap on the
+ *                         circle (including the wrap) is exactly 1/N.
+ *   orc_step              one pass of the loop body of Algorithm 1 ("Sampling
+ *                         from a Code Point"): CDF w over the ordered
+ *                         vocabulary, the token whose interval holds the code,
+ *                         and the rescaled code c <- (c - m)/(M - m); with the
+ *                         logit modifiers the paper names as compatible
+ *                         (temperature, top-k: Sec. 2 and "Top-k sampling" in
+ *                         Sec. 5.1; nucleus: Sec. 2).
+ *   orc_decode_bigram*    Algorithm 1's REPEAT ... UNTIL X = EOS loop over a
+ *                         bigram model (row = next-token logits given the
+ *                         previous token), stopping at EOS and padding
+ *                         (Sec. 3.3, last paragraph).
+ *   orc_encode_bigram     the other direction of the codebook (Sec. 4.1): the
+ *                         interval [w, w + P(sequence)) of a sequence in
+ *                         dictionary order.
+ *
+ * Readings taken where the paper is silent (all also stated in the design
+ * notes): intervals are half-open [F_{i-1}, F_i); order of modifiers is
+ * temperature -> top-k -> softmax -> nucleus on that renormalised distribution
+ * -> renormalise; ties in top-k / nucleus order go to the lower token index;
+ * nucleus keeps the smallest probability-sorted prefix with mass >= top_p;
+ * -inf logits are masked; NaN / +inf logits, an all-masked row or a code
+ * outside [0,1] give status ORC_ERR_NUMERIC, token -1, code unchanged; pad
+ * id is -1.  Parity unpinned by the paper for: modifier order, pad id, the
+ * non-finite policy (they are pinned only by these stated readings).
+ *
+ * All sums are Neumaier-compensated so the oracle's own rounding (~1e-16) is
+ * far below every tolerance used against it.
+ */
+#define _GNU_SOURCE
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_F32 0
+#define ORC_BF16 1
+#define ORC_OK 0
+#define ORC_ERR_INVALID_ARG (-1)
+#define ORC_ERR_NUMERIC (-5)
+
+static const double ORC_ONE_BELOW = 1.0 - 0x1p-53; /* largest double below 1 */
+
+/* ---- exact widening of a stored logit to fp64 ---- */
+static double load_logit(const void *base, int dtype, long idx)
+{
+    if (dtype == ORC_BF16) {
+        uint32_t bits = (uint32_t)((const uint16_t *)base)[idx] << 16;
+        float f;
+        memcpy(&f, &bits, sizeof f);
+        return (double)f;
+    }
+    return (double)((const float *)base)[idx];
+}
+
+/* ---- Neumaier compensated sum ---- */
+typedef struct { double s, c; } nsum;
+static void nsum_add(nsum *a, double x)
+{
+    double t = a->s + x;
+    if (fabs(a->s) >= fabs(x)) a->c += (a->s - t) + x;
+    else                       a->c += (x - t) + a->s;
+    a->s = t;
+}
+static double nsum_val(const nsum *a) { return a->s + a->c; }
+
+typedef struct { double key; long idx; } ranked;
+static int cmp_key_desc_idx_asc(const void *pa, const void *pb)
+{
+    const ranked *a = (const ranked *)pa, *b = (const ranked *)pb;
+    if (a->key > b->key) return -1;
+    if (a->key < b->key) return 1;
+    if (a->idx < b->idx) return -1;
+    if (a->idx > b->idx) return 1;
+    return 0;
+}
+
+typedef struct {
+    int32_t token;
+    double code_out, p_tok, cdf_lo, d_tok, d_topp;
+    int32_t n_kept, tie_topk, status;
+} step_result;
+
+/*
+ * One step for one lane (Algorithm 1, loop body).  row points at V stored
+ * logits.  Work arrays l, e (V doubles), keep (V bytes), rk (V ranked) are
+ * supplied by the caller.
+ */
+static void step_lane(const void *row, int dtype, long V, double c, double temp,
+                      long top_k, double top_p, double *l, double *e, char *keep,
+                      ranked *rk, step_result *out)
+{
+    long j, nK = 0;
+    out->token = -1; out->code_out = c; out->p_tok = 0.0; out->cdf_lo = 0.0;
+    out->d_tok = 0.0; out->d_topp = INFINITY; out->n_kept = 0; out->tie_topk = 0;
+    out->status = ORC_ERR_NUMERIC;
+
+    if (!(c >= 0.0 && c <= 1.0)) return;          /* also rejects NaN */
+    if (c == 1.0) c = ORC_ONE_BELOW;              /* code domain is [0,1) */
+
+    /* 1-2: widen exactly; masked = -inf; NaN / +inf are errors */
+    for (j = 0; j < V; ++j) {
+        l[j] = load_logit(row, dtype, j);
+        if (isnan(l[j]) || l[j] == INFINITY) return;
+        keep[j] = (l[j] > -INFINITY);
+        nK += keep[j];
+    }
+    if (nK == 0) return;
+
+    /* 3: top-k on the logits, order (value desc, index asc) */
+    if (top_k > 0 && top_k < nK) {
+        long n = 0, r;
+        for (j = 0; j < V; ++j) if (keep[j]) { rk[n].key = l[j]; rk[n].idx = j; ++n; }
+        qsort(rk, (size_t)n, sizeof(ranked), cmp_key_desc_idx_asc);
+        for (r = top_k; r < n; ++r) keep[rk[r].idx] = 0;
+        for (r = 0; r < n; ++r) if (rk[r].key == rk[top_k - 1].key) out->tie_topk++;
+        nK = top_k;
+    }
+
+    /* 4: temperature and stable softmax numerators over the survivors */
+    double m = -INFINITY;
+    for (j = 0; j < V; ++j) if (keep[j]) { double x = l[j] / temp; if (x > m) m = x; }
+    nsum z1 = {0.0, 0.0};
+    for (j = 0; j < V; ++j) {
+        if (keep[j]) { e[j] = exp(l[j] / temp - m); nsum_add(&z1, e[j]); }
+        else e[j] = 0.0;
+    }
+    double Z1 = nsum_val(&z1);
+
+    /* 5: nucleus: smallest (prob desc, index asc) prefix with mass >= top_p */
+    if (top_p > 0.0 && top_p < 1.0) {
+        long n = 0, r, cut;
+        for (j = 0; j < V; ++j) if (keep[j]) { rk[n].key = e[j]; rk[n].idx = j; ++n; }
+        qsort(rk, (size_t)n, sizeof(ranked), cmp_key_desc_idx_asc);
+        double target = top_p * Z1, before = 0.0, after = 0.0;
+        nsum run = {0.0, 0.0};
+        cut = n;                                   /* keep everything if never reached */
+        for (r = 0; r < n; ++r) {
+            before = nsum_val(&run);
+            nsum_add(&run, rk[r].key);
+            after = nsum_val(&run);
+            if (after >= target) { cut = r + 1; break; }
+        }
+        for (r = cut; r < n; ++r) keep[rk[r].idx] = 0;
+        if (cut < n || after >= target) {
+            double a = fabs(target - before), b = fabs(after - target);
+            out->d_topp = (a < b ? a : b) / Z1;
+        }
+        nK = cut;
+    }
+
+    /* 6: renormalise over the final kept set, summed in index order */
+    nsum z = {0.0, 0.0};
+    for (j = 0; j < V; ++j) if (keep[j]) nsum_add(&z, e[j]);
+    double Z = nsum_val(&z);
+
+    /* 7: first kept j (ascending index) with c*Z < S_j (inclusive prefix) */
+    double t = c * Z, S_excl = 0.0;
+    long chosen = -1, last = -1;
+    double S_last = 0.0;
+    nsum run = {0.0, 0.0};
+    for (j = 0; j < V; ++j) {
+        if (!keep[j]) continue;
+        double before = nsum_val(&run);
+        nsum_add(&run, e[j]);
+        last = j; S_last = before;
+        if (t < nsum_val(&run)) { chosen = j; S_excl = before; break; }
+    }
+    if (chosen < 0) { chosen = last; S_excl = S_last; }  /* rounding at the top end */
+
+    /* 8: rescale the code into the chosen interval */
+    double cn = (t - S_excl) / e[chosen];
+    if (!(cn >= 0.0)) cn = 0.0;
+    if (cn > ORC_ONE_BELOW) cn = ORC_ONE_BELOW;
+
+    /* 9: diagnostics */
+    double lo = S_excl / Z, hi = (S_excl + e[chosen]) / Z;
+    double da = c - lo, db = hi - c;
+    out->token = (int32_t)chosen;
+    out->code_out = cn;
+    out->p_tok = e[chosen] / Z;
+    out->cdf_lo = lo;
+    out->d_tok = da < db ? da : db;
+    out->n_kept = (int32_t)nK;
+    out->status = ORC_OK;
+}
+
+typedef struct { double *l, *e; char *keep; ranked *rk; } workspace;
+static int ws_alloc(workspace *w, long V)
+{
+    w->l = (double *)malloc(sizeof(double) * (size_t)V);
+    w->e = (double *)malloc(sizeof(double) * (size_t)V);
+    w->keep = (char *)malloc((size_t)V);
+    w->rk = (ranked *)malloc(sizeof(ranked) * (size_t)V);
+    return w->l && w->e && w->keep && w->rk;
+}
+static void ws_free(workspace *w) { free(w->l); free(w->e); free(w->keep); free(w->rk); }
+
+static int check_params(long V, double temp, long top_k, double top_p)
+{
+    if (V < 1) return 0;
+    if (!(temp > 0.0) || isinf(temp)) return 0;
+    if (top_k < 0) return 0;
+    if (isnan(top_p)) return 0;
+    return 1;
+}
+
+/*
+ * Lattice of N codes with one shared shift u in [0,1):  c_j = (j + u)/N, j = 0..N-1.
+ */
+int orc_lattice_codes(long N, double u, double *codes)
+{
+    long j;
+    if (N < 1 || !(u >= 0.0 && u < 1.0) || !codes) return ORC_ERR_INVALID_ARG;
+    for (j = 0; j < N; ++j) {
+        double c = ((double)j + u) / (double)N;
+        if (c >= 1.0) c -= 1.0;
+        codes[j] = c;
+    }
+    return ORC_OK;
+}
+
+/*
+ * One decode step for lanes [lane_begin, lane_end) of logits[lanes, ld].
+ * Any output pointer may be NULL.  Outputs are indexed by absolute lane.
+ */
+int orc_step(const void *logits, int dtype, long lanes, long V, long ld,
+             const double *codes, double temp, long top_k, double top_p,
+             int32_t *tokens, double *codes_out, double *p_tok, double *cdf_lo,
+             int32_t *n_kept, double *d_tok, double *d_topp, int32_t *tie_topk,
+             int32_t *status, long lane_begin, long lane_end)
+{
+    workspace w;
+    long i;
+    size_t esz = dtype == ORC_BF16 ? 2 : 4;
+    if (!logits || !codes || lanes < 0 || ld < V || !check_params(V, temp, top_k, top_p))
+        return ORC_ERR_INVALID_ARG;
+    if (dtype != ORC_F32 && dtype != ORC_BF16) return ORC_ERR_INVALID_ARG;
+    if (lane_begin < 0 || lane_end > lanes) return ORC_ERR_INVALID_ARG;
+    if (!ws_alloc(&w, V)) { ws_free(&w); return ORC_ERR_INVALID_ARG; }
+    for (i = lane_begin; i < lane_end; ++i) {
+        step_result r;
+        const char *row = (const char *)logits + (size_t)i * (size_t)ld * esz;
+        step_lane(row, dtype, V, codes[i], temp, top_k, top_p, w.l, w.e, w.keep, w.rk, &r);
+        if (tokens) tokens[i] = r.token;
+        if (codes_out) codes_out[i] = r.code_out;
+        if (p_tok) p_tok[i] = r.p_tok;
+        if (cdf_lo) cdf_lo[i] = r.cdf_lo;
+        if (n_kept) n_kept[i] = r.n_kept;
+        if (d_tok) d_tok[i] = r.d_tok;
+        if (d_topp) d_topp[i] = r.d_topp;
+        if (tie_topk) tie_topk[i] = r.tie_topk;
+        if (status) status[i] = r.status;
+    }
+    ws_free(&w);
+    return ORC_OK;
+}
+
+/*
+ * Algorithm 1's loop over a bigram model for lanes [lane_begin, lane_end):
+ * lane i starts from previous token prev[i] and code codes_in[i]; at each of
+ * at most T steps the row table[prev] gives the next-token logits.  A lane
+ * stops after emitting eos (pass eos < 0 for "no EOS"); the rest of its row of
+ * seq[lanes, T] is padded with -1 and len[i] = number of tokens emitted.
+ * Optional per-step traces (each [lanes, T], may be NULL): the code the step
+ * started from, its rescaled code, p_tok and d_tok.
+ */
+int orc_decode_bigram_codes(const void *table, int dtype, long V, long ld,
+                            const int32_t *prev, const double *codes_in, long lanes,
+                            long T, long eos, double temp, long top_k, double top_p,
+                            int32_t *seq, int32_t *len, double *codes_final,
+                            int32_t *status, double *trace_code_in,
+                            double *trace_code_out, double *trace_p_tok,
+                            double *trace_d_tok, long lane_begin, long lane_end)
+{
+    workspace w;
+    long i, t;
+    size_t esz = dtype == ORC_BF16 ? 2 : 4;
+    if (!table || !prev || !codes_in || !seq || lanes < 0 || T < 0 || ld < V ||
+        !check_params(V, temp, top_k, top_p))
+        return ORC_ERR_INVALID_ARG;
+    if (dtype != ORC_F32 && dtype != ORC_BF16) return ORC_ERR_INVALID_ARG;
+    if (lane_begin < 0 || lane_end > lanes) return ORC_ERR_INVALID_ARG;
+    for (i = lane_begin; i < lane_end; ++i)
+        if (prev[i] < 0 || prev[i] >= V) return ORC_ERR_INVALID_ARG;
+    if (!ws_alloc(&w, V)) { ws_free(&w); return ORC_ERR_INVALID_ARG; }
+    for (i = lane_begin; i < lane_end; ++i) {
+        long p = prev[i], n = 0;
+        double c = codes_in[i];
+        int32_t st = ORC_OK;
+        for (t = 0; t < T; ++t) {
+            seq[i * T + t] = -1;
+            if (trace_code_in) trace_code_in[i * T + t] = NAN;
+            if (trace_code_out) trace_code_out[i * T + t] = NAN;
+            if (trace_p_tok) trace_p_tok[i * T + t] = NAN;
+            if (trace_d_tok) trace_d_tok[i * T + t] = NAN;
+        }
+        for (t = 0; t < T; ++t) {
+            step_result r;
+            const char *row = (const char *)table + (size_t)p * (size_t)ld * esz;
+            step_lane(row, dtype, V, c, temp, top_k, top_p, w.l, w.e, w.keep, w.rk, &r);
+            if (r.status != ORC_OK) { st = r.status; break; }
+            if (trace_code_in) trace_code_in[i * T + t] = c;
+            if (trace_code_out) trace_code_out[i * T + t] = r.code_out;
+            if (trace_p_tok) trace_p_tok[i * T + t] = r.p_tok;
+            if (trace_d_tok) trace_d_tok[i * T + t] = r.d_tok;
+            seq[i * T + t] = r.token;
+            n = t + 1;
+            c = r.code_out;
+            p = r.token;
+            if (r.token == eos) break;
+        }
+        if (len) len[i] = (int32_t)n;
+        if (codes_final) codes_final[i] = c;
+        if (status) status[i] = st;
+    }
+    ws_free(&w);
+    return ORC_OK;
+}
+
+/*
+ * Same loop with the code set of the Definition in Sec. 4.2: S start tokens,
+ * N lattice codes each sharing one shift u; lane = s*N + j decodes code c_j
+ * from previous token start[s].
+ */
+int orc_decode_bigram(const void *table, int dtype, long V, long ld,
+                      const int32_t *start, long S, long N, double u, long T, long eos,
+                      double temp, long top_k, double top_p,
+                      int32_t *seq, int32_t *len, double *codes_final, int32_t *status)
+{
+    long s, j, lanes = S * N;
+    int rc;
+    if (S < 0 || N < 1 || !start) return ORC_ERR_INVALID_ARG;
+    double *lat = (double *)malloc(sizeof(double) * (size_t)N);
+    double *codes = (double *)malloc(sizeof(double) * (size_t)(lanes > 0 ? lanes : 1));
+    int32_t *prev = (int32_t *)malloc(sizeof(int32_t) * (size_t)(lanes > 0 ? lanes : 1));
+    if (!lat || !codes || !prev) { free(lat); free(codes); free(prev); return ORC_ERR_INVALID_ARG; }
+    rc = orc_lattice_codes(N, u, lat);
+    if (rc == ORC_OK) {
+        for (s = 0; s < S; ++s)
+            for (j = 0; j < N; ++j) { codes[s * N + j] = lat[j]; prev[s * N + j] = start[s]; }
+        rc = orc_decode_bigram_codes(table, dtype, V, ld, prev, codes, lanes, T, eos, temp,
+                                     top_k, top_p, seq, len, codes_final, status,
+                                     NULL, NULL, NULL, NULL, 0, lanes);
+    }
+    free(lat); free(codes); free(prev);
+    return rc;
+}
+
+/*
+ * Codebook, sequence -> interval (Sec. 4.1): for each lane, the interval
+ * [lo, lo + width) in dictionary order of the token sequence seq[i, 0..len-1]
+ * continued from prev[i]: lo accumulates width * F_{i-1}, width multiplies by
+ * p_i, with the same modified conditional distributions as orc_step.  A token
+ * of probability zero gives status ORC_ERR_NUMERIC.
+ */
+int orc_encode_bigram(const void *table, int dtype, long V, long ld,
+                      const int32_t *prev, const int32_t *seq, const int32_t *len,
+                      long lanes, long T, double temp, long top_k, double top_p,
+                      double *lo_out, double *width_out, int32_t *status)
+{
+    workspace w;
+    long i, t, j;
+    size_t esz = dtype == ORC_BF16 ? 2 : 4;
+    if (!table || !prev || !seq || !len || lanes < 0 || T < 0 || ld < V ||
+        !check_params(V, temp, top_k, top_p))
+        return ORC_ERR_INVALID_ARG;
+    if (!ws_alloc(&w, V)) { ws_free(&w); return ORC_ERR_INVALID_ARG; }
+    for (i = 0; i < lanes; ++i) {
+        nsum lo = {0.0, 0.0};
+        double width = 1.0;
+        long p = prev[i];
+        int32_t st = ORC_OK;
+        for (t = 0; t < len[i] && t < T; ++t) {
+            long tok = seq[i * T + t];
+            if (p < 0 || p >= V || tok < 0 || tok >= V) { st = ORC_ERR_INVALID_ARG; break; }
+            /* the distribution of this step: run the step with a code that
+               cannot fail, then rebuild the kept set's masses from keep/e */
+            step_result r;
+            const char *row = (const char *)table + (size_t)p * (size_t)ld * esz;
+            step_lane(row, dtype, V, 0.0, temp, top_k, top_p, w.l, w.e, w.keep, w.rk, &r);
+            if (r.status != ORC_OK) { st = r.status; break; }
+            if (!w.keep[tok]) { st = ORC_ERR_NUMERIC; break; }
+            nsum z = {0.0, 0.0}, below = {0.0, 0.0};
+            for (j = 0; j < V; ++j) if (w.keep[j]) {
+                nsum_add(&z, w.e[j]);
+                if (j < tok) nsum_add(&below, w.e[j]);
+            }
+            double Z = nsum_val(&z);
+            nsum_add(&lo, width * (nsum_val(&below) / Z));
+            width *= w.e[tok] / Z;
+            p = tok;
+        }
+        if (lo_out) lo_out[i] = nsum_val(&lo);
+        if (width_out) width_out[i] = width;
+        if (status) status[i] = st;
+    }
+    ws_free(&w);
+    return ORC_OK;
+}
+
+int orc_version(void) { return 1; }

@@ -1,0 +1,426 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+Each test names the passage it checks.  References come from tests/exact_ref.py
+(sequence-level brute force in 60-digit decimals, counting definitions of the
+truncations), from closed forms, or from the small fixtures in tests/golden/.
+"""
+import math
+import os
+from decimal import Decimal
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from tests import exact_ref as ex
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+F32, BF16 = 0, 1
+
+
+def _rows(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float32))
+
+
+def _golden_kv(name):
+    out = {}
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            k, v = line.split()
+            out[k] = float(v)
+    return out
+
+
+# --------------------------------------------------------------------------- Example, Sec. 4.2
+def test_worked_example_naive_code(orc):
+    g = _golden_kv("example_bias.txt")
+    logits = _rows([[math.log(g["p_A"]), math.log(g["p_B"])]])
+    o = orc.step(logits, F32, np.array([g["code"]]))
+    assert o.status[0] == 0 and o.tokens[0] == int(g["token"])
+    assert o.codes[0] == pytest.approx(g["rescaled_num"] / g["rescaled_den"], rel=1e-7)
+    assert o.p_tok[0] == pytest.approx(g["p_A"], rel=1e-7)
+
+
+def test_worked_example_shift_removes_bias(orc):
+    # Proposition 3 on the example: averaged over the shift, P(token A) = 0.6 with N = 1.
+    g = _golden_kv("example_bias.txt")
+    logits = _rows([[math.log(g["p_A"]), math.log(g["p_B"])]])
+    K = 20000
+    us = (np.arange(K) + 0.5) / K
+    hits = 0
+    for u in us:
+        c = orc.lattice_codes(1, float(u))
+        hits += int(orc.step(logits, F32, c).tokens[0] == 0)
+    assert hits / K == pytest.approx(g["shifted_mean_A"], abs=2.0 / K)
+
+
+# --------------------------------------------------------------------------- lattice, Def. Sec. 4.2 / Eq. 2
+@pytest.mark.parametrize("N", [1, 2, 7, 32, 1000])
+def test_lattice_even_on_circle(orc, N):
+    for u in [0.0, 0.25, 0.999999, 1.0 - 2 ** -53]:
+        c = orc.lattice_codes(N, u)
+        assert c.shape == (N,) and (c >= 0).all() and (c < 1).all()
+        s = np.sort(c)
+        gaps = np.diff(np.concatenate([s, [s[0] + 1.0]]))
+        np.testing.assert_allclose(gaps, 1.0 / N, rtol=0, atol=4e-16)
+        # the shift of the whole set is u/N
+        np.testing.assert_allclose(c[0], u / N, rtol=0, atol=1e-16)
+
+
+def test_lattice_rejects_bad_arguments(orc):
+    for N, u in [(0, 0.5), (-1, 0.5), (4, 1.0), (4, -0.1), (4, float("nan"))]:
+        with pytest.raises(ValueError):
+            orc.lattice_codes(N, u)
+
+
+def test_lattice_interval_counts(orc):
+    # proofs of the duplicate bounds (Sec. 4.3): an interval of length ell holds
+    # floor(N ell) or ceil(N ell) of N evenly spaced shifted points.
+    rng = np.random.default_rng(5)
+    for _ in range(200):
+        N = int(rng.integers(1, 65))
+        u = float(rng.random())
+        a, ell = float(rng.random()), float(rng.random())
+        c = orc.lattice_codes(N, u)
+        inside = int((((c - a) % 1.0) < ell).sum())
+        assert math.floor(N * ell - 1e-9) <= inside <= math.ceil(N * ell + 1e-9)
+
+
+def test_appendix_b_constants(orc):
+    with open(os.path.join(GOLD, "appendix_b.txt")) as f:
+        rows = [l.split() for l in f if l.strip() and not l.startswith("#")]
+    for n_s, con_s, coff_s in rows:
+        N = int(n_s)
+        M = N + 1
+        K = 8 * N * M
+        e_ll = Fraction(0)
+        e_lr = Fraction(0)
+        for k in range(K):
+            u = (k + 0.5) / K        # midpoints: never on a breakpoint, average is exact
+            c = orc.lattice_codes(M, u)
+            l = int((c < 1.0 / N).sum())
+            r = int(((c >= 1.0 / N) & (c < 2.0 / N)).sum())
+            e_ll += Fraction(l * (l - 1), K)
+            e_lr += Fraction(l * r, K)
+        mu2 = Fraction(M * (M - 1), N * N)
+        assert e_ll - mu2 == Fraction(con_s)
+        assert e_lr - mu2 == Fraction(coff_s)
+
+
+# --------------------------------------------------------------------------- one step: interval semantics
+def test_step_measure_of_each_token_equals_probability(orc):
+    # Sec. 3.1: token i owns an interval of length P(x_i), intervals in vocabulary order.
+    rng = np.random.default_rng(11)
+    V = 7
+    logits = _rows(rng.normal(0, 2, (1, V)))
+    p = [float(x) for x in ex.conditional([float(v) for v in logits[0]])]
+    M = 40000
+    codes = (np.arange(M) + 0.5) / M
+    o = orc.step(np.repeat(logits, M, 0), F32, codes)
+    assert (o.status == 0).all()
+    assert (np.diff(o.tokens) >= 0).all()            # vocabulary order along the code axis
+    for j in range(V):
+        assert (o.tokens == j).mean() == pytest.approx(p[j], abs=1.5 / M)
+    # rescaled code = position inside the interval
+    cdf = np.concatenate([[0.0], np.cumsum(p)])
+    want = (codes - cdf[o.tokens]) / np.array(p)[o.tokens]
+    np.testing.assert_allclose(o.codes, want, rtol=0, atol=1e-9)
+    np.testing.assert_allclose(o.cdf_lo, cdf[o.tokens], atol=1e-12)
+    np.testing.assert_allclose(o.p_tok, np.array(p)[o.tokens], rtol=1e-12)
+
+
+def test_step_boundaries_half_open(orc):
+    # p = (1/4, 1/4, 1/4, 1/4) exactly: a code on a boundary belongs to the upper interval.
+    logits = _rows([[1.5, 1.5, 1.5, 1.5]] * 6)
+    codes = np.array([0.0, 0.25, 0.75, np.nextafter(0.25, 0), np.nextafter(0.75, 0), 1.0])
+    o = orc.step(logits, F32, codes)
+    assert o.tokens.tolist() == [0, 1, 3, 0, 2, 3]
+    assert o.codes[0] == 0.0 and o.codes[1] == pytest.approx(0.0, abs=1e-15)
+    assert (o.codes < 1.0).all() and (o.codes >= 0.0).all()
+
+
+def test_step_masked_and_nonfinite(orc):
+    ninf = -np.inf
+    o = orc.step(_rows([[ninf, 0.0, ninf, 0.0]] * 2), F32, np.array([0.25, 0.75]))
+    assert o.tokens.tolist() == [1, 3] and o.n_kept.tolist() == [2, 2]
+    bad = orc.step(_rows([[0.0, np.nan], [np.inf, 0.0], [ninf, ninf], [0.0, 0.0], [0.0, 0.0]]),
+                   F32, np.array([0.5, 0.5, 0.5, 1.5, np.nan]))
+    assert (bad.status == orc.ERR_NUMERIC).all() and (bad.tokens == -1).all()
+    assert bad.codes[0] == 0.5 and bad.codes[3] == 1.5
+
+
+def test_step_bf16_storage_is_widened_exactly(orc):
+    from paper_2210_15458_b200 import synth
+    rng = np.random.default_rng(3)
+    x = rng.normal(0, 3, (5, 33)).astype(np.float32)
+    bits = synth.f32_to_bf16_bits(x)
+    codes = rng.random(5)
+    a = orc.step(bits, BF16, codes, temp=0.7, top_k=4)
+    b = orc.step(synth.bf16_bits_to_f32(bits), F32, codes, temp=0.7, top_k=4)
+    assert (a.tokens == b.tokens).all() and (a.codes == b.codes).all()
+
+
+# --------------------------------------------------------------------------- modifiers
+@pytest.mark.parametrize("temp", [0.1, 0.7, 1.0, 2.5])
+def test_temperature(orc, temp):
+    # softmax temperature (Sec. 5.1): p_i proportional to exp(l_i / T); with l = T ln n the
+    # distribution is n / sum n exactly.
+    n = np.array([1, 2, 3, 4, 10], dtype=np.float64)
+    logits = _rows([temp * np.log(n)])
+    M = 2000
+    codes = (np.arange(M) + 0.5) / M
+    o = orc.step(np.repeat(logits, M, 0), F32, codes, temp=temp)
+    for j in range(5):
+        assert (o.tokens == j).mean() == pytest.approx(n[j] / n.sum(), abs=2.0 / M)
+
+
+def _check_against_counting_definition(orc, logits_row, temp, top_k, top_p, M=3001):
+    p = ex.conditional([float(v) for v in logits_row], temp, top_k, top_p)
+    codes = (np.arange(M) + 0.5) / M
+    o = orc.step(np.repeat(_rows([logits_row]), M, 0), F32, codes, temp=temp, top_k=top_k, top_p=top_p)
+    assert (o.status == 0).all()
+    kept = sum(1 for x in p if x > 0)
+    assert (o.n_kept == kept).all()
+    cdf = [Decimal(0)]
+    for x in p:
+        cdf.append(cdf[-1] + x)
+    for i in range(0, M, 7):
+        c = ex.D(codes[i])
+        tok = next(j for j in range(len(p)) if cdf[j] <= c < cdf[j + 1])
+        d = min(c - cdf[tok], cdf[tok + 1] - c)
+        if d > Decimal("1e-12"):
+            assert o.tokens[i] == tok
+            assert o.codes[i] == pytest.approx(float((c - cdf[tok]) / p[tok]), abs=1e-9)
+            assert o.p_tok[i] == pytest.approx(float(p[tok]), rel=1e-12)
+
+
+def test_top_k_counting_definition_with_ties(orc):
+    rng = np.random.default_rng(21)
+    for trial in range(30):
+        V = int(rng.integers(2, 12))
+        row = rng.integers(-3, 4, V).astype(np.float32)      # many ties
+        k = int(rng.integers(1, V + 2))
+        _check_against_counting_definition(orc, row, float(rng.choice([0.5, 1.0, 2.0])), k, 1.0, M=501)
+
+
+def test_top_k_special_cases(orc):
+    rng = np.random.default_rng(22)
+    row = _rows([[1.0, 3.0, 3.0, -2.0, 0.5]])
+    codes = rng.random(64)
+    rows = np.repeat(row, 64, 0)
+    k1 = orc.step(rows, F32, codes, top_k=1)
+    assert (k1.tokens == 1).all() and (k1.n_kept == 1).all()      # argmax, lowest index among maxima
+    np.testing.assert_allclose(k1.codes, codes, atol=1e-15)        # whole interval -> code unchanged
+    assert (k1.tie_topk == 2).all()
+    base = orc.step(rows, F32, codes)
+    for k in (0, 5, 6, 100):
+        kk = orc.step(rows, F32, codes, top_k=k)
+        assert (kk.tokens == base.tokens).all() and (kk.codes == base.codes).all()
+    k2 = orc.step(rows, F32, codes, top_k=2)                        # the two tied maxima, half each
+    assert set(k2.tokens.tolist()) == {1, 2}
+    np.testing.assert_allclose(k2.p_tok, 0.5, rtol=1e-15)
+
+
+def test_nucleus_counting_definition(orc):
+    rng = np.random.default_rng(23)
+    for trial in range(30):
+        V = int(rng.integers(2, 12))
+        row = (rng.integers(-4, 5, V) * 0.5).astype(np.float32)
+        top_p = float(rng.choice([0.05, 0.3, 0.5, 0.9, 0.99]))
+        _check_against_counting_definition(orc, row, float(rng.choice([0.7, 1.0])), 0, top_p, M=501)
+
+
+def test_nucleus_special_cases(orc):
+    rng = np.random.default_rng(24)
+    row = _rows([[1.0, 3.0, 3.0, -2.0, 0.5]])
+    codes = rng.random(32)
+    rows = np.repeat(row, 32, 0)
+    tiny = orc.step(rows, F32, codes, top_p=1e-9)
+    assert (tiny.tokens == 1).all() and (tiny.n_kept == 1).all()
+    base = orc.step(rows, F32, codes)
+    for tp in (1.0, 0.0, 1.5, -1.0):
+        off = orc.step(rows, F32, codes, top_p=tp)
+        assert (off.tokens == base.tokens).all() and (off.codes == base.codes).all()
+    # p = (.1, .2, .3, .4): top_p = 0.7 keeps exactly {3, 2}; 0.71 also needs token 1
+    row2 = _rows([np.log([1.0, 2.0, 3.0, 4.0])])
+    a = orc.step(np.repeat(row2, 32, 0), F32, codes, top_p=0.65)
+    b = orc.step(np.repeat(row2, 32, 0), F32, codes, top_p=0.75)
+    assert (a.n_kept == 2).all() and set(a.tokens.tolist()) <= {2, 3}
+    assert (b.n_kept == 3).all() and set(b.tokens.tolist()) <= {1, 2, 3}
+    assert a.d_topp[0] == pytest.approx(0.05, abs=1e-6)
+
+
+def test_top_k_then_nucleus_order(orc):
+    # reading: the nucleus mass is measured on the distribution renormalised over the
+    # top-k survivors.  p = (.4,.3,.2,.1); top_k = 2 -> (4/7, 3/7); top_p = .6 then needs both
+    # (on the full softmax, .4 + .3 >= .6 as well, but top_p = .5: 4/7 >= .5 keeps ONE token,
+    # whereas measured on the full softmax .4 < .5 would keep two).
+    row = _rows([np.log([4.0, 3.0, 2.0, 1.0])])
+    codes = (np.arange(50) + 0.5) / 50
+    o = orc.step(np.repeat(row, 50, 0), F32, codes, top_k=2, top_p=0.5)
+    assert (o.n_kept == 1).all() and (o.tokens == 0).all()
+    for k, tp in [(3, 0.8), (2, 0.9), (4, 0.35)]:
+        _check_against_counting_definition(orc, row[0], 1.0, k, tp, M=301)
+
+
+# --------------------------------------------------------------------------- whole decode: brute force, Sec. 4.1
+def _tiny_model(V, seed, sigma=1.5):
+    rng = np.random.default_rng(seed)
+    return _rows(rng.normal(0, sigma, (V, V)))
+
+
+def _book(table, start, T, eos, temp=1.0, top_k=0, top_p=1.0):
+    cache = {}
+
+    def row_probs(prev):
+        if prev not in cache:
+            cache[prev] = ex.conditional([float(v) for v in table[prev]], temp, top_k, top_p)
+        return cache[prev]
+    return ex.enumerate_codebook(row_probs, start, T, eos)
+
+
+@pytest.mark.parametrize("V,T,eos,kw", [
+    (3, 2, -1, {}),                       # the shape of Fig. 1
+    (5, 4, -1, {}),
+    (5, 4, 0, {}),                        # EOS makes a prefix-free set of unequal lengths
+    (4, 5, 2, {"temp": 0.6}),
+    (5, 3, -1, {"top_k": 3}),
+    (5, 3, 1, {"top_p": 0.8, "temp": 1.3}),
+])
+def test_decode_matches_dictionary_order_codebook(orc, V, T, eos, kw):
+    table = _tiny_model(V, seed=100 + V * 10 + T)
+    start = 1
+    book = _book(table, start, T, eos, **kw)
+    assert sum(w for _, _, w in book) == pytest.approx(Decimal(1), abs=Decimal("1e-50"))
+    rng = np.random.default_rng(7)
+    codes = np.concatenate([rng.random(400), (np.arange(100) + 0.5) / 100])
+    o = orc.decode_bigram_codes(table, F32, np.full(len(codes), start, np.int32), codes, T, eos, **kw)
+    checked = 0
+    for i, c in enumerate(codes):
+        seq, lo, width, dist = ex.locate(book, c)
+        if dist < Decimal("1e-11"):
+            continue
+        checked += 1
+        assert tuple(o.seq[i, :o.len[i]]) == seq
+        assert (o.seq[i, o.len[i]:] == -1).all()
+        want_final = float((ex.D(c) - lo) / width)
+        assert o.codes_final[i] == pytest.approx(want_final, abs=1e-13 / float(width) + 1e-12)
+    assert checked > 450
+
+
+def test_encode_is_the_inverse_map(orc):
+    # Sec. 4.1, item (1): sequence -> interval; it must contain the code that produced it.
+    table = _tiny_model(6, seed=77)
+    rng = np.random.default_rng(8)
+    codes = rng.random(200)
+    prev = np.full(200, 2, np.int32)
+    o = orc.decode_bigram_codes(table, F32, prev, codes, 5, 0, temp=0.8)
+    lo, width, st = orc.encode_bigram(table, F32, prev, o.seq, o.len, temp=0.8)
+    assert (st == 0).all()
+    assert (lo <= codes + 1e-14).all() and (codes < lo + width + 1e-14).all()
+    book = _book(table, 2, 5, 0, temp=0.8)
+    lut = {seq: (l, w) for seq, l, w in book}
+    for i in range(0, 200, 9):
+        l, w = lut[tuple(o.seq[i, :o.len[i]])]
+        assert lo[i] == pytest.approx(float(l), abs=1e-14)
+        assert width[i] == pytest.approx(float(w), rel=1e-13)
+
+
+def test_lattice_coverage_and_duplicate_bounds(orc):
+    # Sec. 4.3 (restated for spacing 1/N): a sequence of probability P is decoded by
+    # floor(N P) or ceil(N P) lanes for every shift; in particular P > 1/N => at least once.
+    table = _tiny_model(4, seed=55, sigma=2.0)
+    T, start, N = 3, 0, 16
+    book = _book(table, start, T, -1)
+    for u in np.random.default_rng(9).random(25):
+        o = orc.decode_bigram(table, F32, np.array([start], np.int32), N, float(u), T, -1)
+        got = {}
+        for i in range(N):
+            got[tuple(o.seq[i])] = got.get(tuple(o.seq[i]), 0) + 1
+        for seq, lo, w in book:
+            n = got.get(seq, 0)
+            assert math.floor(float(w) * N - 1e-9) <= n <= math.ceil(float(w) * N + 1e-9)
+            if w > Decimal(1) / N + Decimal("1e-9"):
+                assert n >= 1
+
+
+def test_unbiased_over_shifts_prop3(orc):
+    table = _tiny_model(4, seed=56)
+    T, start, N = 3, 1, 5
+    book = _book(table, start, T, -1)
+
+    def f(seq):
+        return 1.0 + 3.0 * seq[0] - 2.0 * seq[-1] + (seq[1] == 2)
+    want = float(ex.expectation(book, f))
+    K = 4000
+    tot = 0.0
+    for k in range(K):
+        o = orc.decode_bigram(table, F32, np.array([start], np.int32), N, (k + 0.5) / K, T, -1)
+        tot += np.mean([f(tuple(s)) for s in o.seq])
+    assert tot / K == pytest.approx(want, abs=5e-3)   # deterministic midpoint rule over the shift
+    # a biased variant for contrast: the unshifted lattice differs measurably
+    o0 = orc.decode_bigram(table, F32, np.array([start], np.int32), N, 0.0, T, -1)
+    assert abs(np.mean([f(tuple(s)) for s in o0.seq]) - want) > 5e-3
+
+
+def test_zero_variance_when_widths_are_multiples_of_1_over_N(orc):
+    # Sec. 4.4, first proposition: every sequence of a uniform 4-symbol model with T = 2 has
+    # probability exactly 1/16 (token 2 masked out of a 5-symbol vocabulary); with N = 16 each
+    # is decoded exactly once for every shift, and with N = 32 exactly twice.
+    row = [0.5, 0.5, -np.inf, 0.5, 0.5]
+    table = _rows([row] * 5)
+    for N in (16, 32):
+        for u in np.random.default_rng(10).random(40):
+            o = orc.decode_bigram(table, F32, np.array([0], np.int32), N, float(u), 2, -1)
+            counts = {}
+            for s in o.seq:
+                counts[tuple(s)] = counts.get(tuple(s), 0) + 1
+            assert len(counts) == 16 and set(counts.values()) == {N // 16}
+            assert all(2 not in k for k in counts)
+
+
+def test_monotone_codes_give_dictionary_ordered_sequences(orc):
+    table = _tiny_model(5, seed=57)
+    codes = np.sort(np.random.default_rng(12).random(300))
+    o = orc.decode_bigram_codes(table, F32, np.full(300, 3, np.int32), codes, 4, -1)
+    seqs = [tuple(s) for s in o.seq]
+    assert seqs == sorted(seqs)
+
+
+def test_iid_codes_sample_the_model_prop1(orc):
+    table = _tiny_model(3, seed=58)
+    book = _book(table, 0, 2, -1)
+    n = 60000
+    codes = np.random.default_rng(13).random(n)
+    o = orc.decode_bigram_codes(table, F32, np.zeros(n, np.int32), codes, 2, -1, threads=4)
+    chi2 = 0.0
+    for seq, lo, w in book:
+        obs = int(((o.seq[:, 0] == seq[0]) & (o.seq[:, 1] == seq[1])).sum())
+        chi2 += (obs - n * float(w)) ** 2 / (n * float(w))
+    assert chi2 < 30.0           # 8 degrees of freedom; P(chi2 > 30) ~ 2e-4
+
+
+def test_decode_split_and_resume(orc):
+    table = _tiny_model(6, seed=59)
+    codes = np.random.default_rng(14).random(50)
+    prev = np.full(50, 4, np.int32)
+    full = orc.decode_bigram_codes(table, F32, prev, codes, 8, 0)
+    a = orc.decode_bigram_codes(table, F32, prev, codes, 4, 0)
+    alive = a.len == 4
+    alive &= a.seq[:, 3] != 0
+    idx = np.nonzero(alive)[0]
+    b = orc.decode_bigram_codes(table, F32, a.seq[idx, 3], a.codes_final[idx], 4, 0)
+    for n, i in enumerate(idx):
+        assert (full.seq[i, 4:] == b.seq[n]).all()
+        assert full.codes_final[i] == b.codes_final[n]
+
+
+def test_threads_do_not_change_results(orc):
+    rng = np.random.default_rng(15)
+    logits = _rows(rng.normal(0, 2, (37, 50)))
+    codes = rng.random(37)
+    a = orc.step(logits, F32, codes, temp=0.9, top_k=7, top_p=0.9)
+    b = orc.step(logits, F32, codes, temp=0.9, top_k=7, top_p=0.9, threads=5)
+    assert (a.tokens == b.tokens).all() and (a.codes == b.codes).all()
