@@ -1,0 +1,197 @@
+/*
+ * arith_sampling.h -- C ABI of the B200 (sm_100a) arithmetic-sampling decode library.
+ *
+ * Arithmetic sampling (Vilnis et al., arXiv 2210.15458) decodes a set of code
+ * points in [0,1) against a sequence model: every code lane repeatedly takes
+ * the model's next-token distribution, finds the token whose CDF interval
+ * (vocabulary-index order) holds the code, and rescales the code into that
+ * interval (Algorithm 1, "Sampling from a Code Point").  The code set is a
+ * regular lattice with one shared uniform shift (Definition "Arithmetic
+ * sampling", Sec. 4.2; Eq. 2).  Lanes never communicate (Remark after
+ * Proposition 1).
+ *
+ * Conventions common to every call
+ *   - All functions are extern "C", return an int status (AS_OK = 0, errors < 0)
+ *     and never throw.  as_last_error() gives a text for the calling thread's
+ *     last failure.
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller
+ *     owns every buffer; unless a function's comment says otherwise, nothing is
+ *     allocated and no buffer is kept after the call.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Device-buffer calls only enqueue work on it and return; results are ready
+ *     once the stream has reached that point.  Host-detectable errors return at
+ *     once with nothing enqueued.
+ *   - There is no CPU implementation behind these calls: without a usable CUDA
+ *     device they return AS_ERR_CUDA.
+ *   - Logits are row-major [rows, ld] with ld >= V elements between rows, dtype
+ *     AS_F32 (IEEE binary32) or AS_BF16 (bfloat16 bit patterns).  Rows whose
+ *     address and pitch are multiples of 16 bytes take the bulk-copy path; other
+ *     layouts are accepted and take a slower load path.
+ *   - Codes are fp64 in [0,1).  An input code of exactly 1.0 is read as the
+ *     largest double below 1.  Rescaled codes are clamped to [0, 1 - 2^-53].
+ *
+ * Per-lane conditions found on the device never trap; they are reported through
+ * the optional lane-status array: AS_OK, or AS_ERR_NUMERIC for a NaN or +inf
+ * logit, a row with every logit -inf, or a code outside [0,1] / NaN.  Such a
+ * lane gets token -1 and its code is returned unchanged.
+ *
+ * Readings of the paper fixed by this library (the paper is silent on them):
+ * half-open intervals [F_{i-1}, F_i); modifiers applied as temperature, then
+ * top-k, then softmax over the survivors, then nucleus on that renormalised
+ * distribution, then renormalisation; ties in top-k / nucleus order go to the
+ * lower token index; the nucleus is the smallest probability-sorted prefix with
+ * mass >= top_p; -inf logits are masked out.
+ */
+#ifndef ARITH_SAMPLING_H_
+#define ARITH_SAMPLING_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AS_F32 0
+#define AS_BF16 1
+
+#define AS_OK 0
+#define AS_ERR_INVALID_ARG (-1)  /* NULL pointer, size or parameter out of range */
+#define AS_ERR_UNSUPPORTED (-2)  /* valid request this build cannot serve (e.g. V too large) */
+#define AS_ERR_CUDA (-3)         /* a CUDA runtime call failed (no device, launch error) */
+#define AS_ERR_TIMEOUT (-4)      /* a bounded on-device wait ran out (reported per lane) */
+#define AS_ERR_NUMERIC (-5)      /* per-lane: non-finite logits / empty row / bad code */
+
+/* Largest vocabulary size accepted by as_step / as_decode_bigram*. */
+#define AS_MAX_V (1 << 20)
+
+/*
+ * Optional per-lane diagnostics of as_step; any member may be NULL.
+ *   d_p_tok       [lanes] f64  probability of the chosen token under the modified distribution
+ *   d_cdf_lo      [lanes] f64  F_{i-1}, the lower end of the chosen token's interval
+ *   d_n_kept      [lanes] i32  number of tokens with non-zero probability after the cuts
+ *   d_lane_status [lanes] i32  AS_OK or AS_ERR_NUMERIC / AS_ERR_TIMEOUT
+ */
+typedef struct as_step_diag {
+    double *d_p_tok;
+    double *d_cdf_lo;
+    int32_t *d_n_kept;
+    int32_t *d_lane_status;
+} as_step_diag;
+
+/*
+ * Shifted lattice of codes (Definition "Arithmetic sampling", Sec. 4.2; Eq. 2):
+ *   d_codes[j] = (j + u) / N  (mod 1),  j = 0..N-1,
+ * a lattice of spacing 1/N -- every gap on the circle, the wrap included, is
+ * exactly 1/N -- moved by one shared shift; u is the caller's uniform draw.
+ *   N        number of codes, >= 1
+ *   u        shift in [0,1)
+ *   d_codes  [N] f64 device, written
+ * Errors: AS_ERR_INVALID_ARG for N < 1, u outside [0,1) or NaN, NULL d_codes.
+ */
+int as_lattice_codes(int N, double u, double *d_codes, void *stream);
+
+/*
+ * One decode step for every lane (the loop body of Algorithm 1, with the logit
+ * modifiers named in Sec. 2 and "Top-k sampling", Sec. 5.1):
+ *   x_j = logits[lane, j] / temp; optional top-k and nucleus cuts; p = softmax
+ *   over the kept tokens; F = CDF of p in vocabulary-index order;
+ *   token = the i with F_{i-1} <= c < F_i;  c' = (c - F_{i-1}) / p_i.
+ *   d_logits     [lanes, ld] device, dtype AS_F32 or AS_BF16, read once
+ *   lanes        >= 0 (0 is a no-op);  V in [1, AS_MAX_V];  ld >= V (elements)
+ *   d_codes      [lanes] f64 device, the lanes' current codes
+ *   temp         softmax temperature, > 0 and finite
+ *   top_k        keep the k largest logits; <= 0 or >= V disables
+ *   top_p        nucleus mass; <= 0 or >= 1 disables
+ *   d_tokens     [lanes] i32 device, written
+ *   d_codes_out  [lanes] f64 device, written; may be the same pointer as d_codes
+ *   diag         NULL or a struct of optional device arrays (see as_step_diag)
+ * Errors: AS_ERR_INVALID_ARG (NULL pointers, lanes < 0, V < 1, ld < V, temp not
+ * positive/finite, NaN top_p, unknown dtype, misaligned element pointer),
+ * AS_ERR_UNSUPPORTED (V > AS_MAX_V), AS_ERR_CUDA.
+ */
+int as_step(const void *d_logits, int dtype, int lanes, int V, long long ld,
+            const double *d_codes, double temp, int top_k, double top_p,
+            int32_t *d_tokens, double *d_codes_out, const as_step_diag *diag,
+            void *stream);
+
+/*
+ * Same step with HOST buffers: copies logits and codes to the device, runs
+ * as_step, copies tokens and codes back, and returns after the results are in
+ * the host buffers (it synchronises `stream`).  Pinned host memory makes the
+ * copies fast but is not required.
+ *   h_logits [lanes, ld] host;  h_codes [lanes] host;  h_tokens, h_codes_out
+ *   [lanes] host, written;  h_lane_status NULL or [lanes] host, written.
+ *   d_work   device scratch of at least as_step_host_work_bytes(...) bytes,
+ *            256-byte aligned, owned by the caller; contents undefined after.
+ * Errors: as as_step, plus AS_ERR_INVALID_ARG if work_bytes is too small.
+ */
+int as_step_host(const void *h_logits, int dtype, int lanes, int V, long long ld,
+                 const double *h_codes, double temp, int top_k, double top_p,
+                 int32_t *h_tokens, double *h_codes_out, int32_t *h_lane_status,
+                 void *d_work, size_t work_bytes, void *stream);
+size_t as_step_host_work_bytes(int dtype, int lanes, long long ld);
+
+/*
+ * Full decode loop of Algorithm 1 (REPEAT ... UNTIL X = EOS) over a bigram
+ * model: row table[prev] holds the next-token logits given the previous token.
+ * The code set is the shifted lattice of as_lattice_codes, one copy per start
+ * token: lane = s*N + j decodes code (j+u)/N starting from d_start[s] (the
+ * start token is not part of the output).  Each lane runs up to T steps, stops
+ * after emitting `eos` and pads the rest of its row with -1 (Sec. 3.3: EOS
+ * terminates a sequence, padding makes lengths uniform).
+ *   d_table   [V, ld] device (row index = previous token), read only
+ *   d_start   [S] i32 device, each in [0, V);  S >= 0, N >= 1, u in [0,1)
+ *   T         maximum number of steps, >= 0;  eos: token id, or < 0 for none
+ *   temp, top_k, top_p   as in as_step, the same for every step
+ *   d_seq         [S*N, T] i32 device, written (tokens, then -1 padding)
+ *   d_len         [S*N] i32 device, written: tokens emitted (EOS included)
+ *   d_codes_final NULL or [S*N] f64 device: each lane's code after its last step
+ *   d_lane_status NULL or [S*N] i32 device: AS_OK, or the status that stopped the
+ *                 lane early (a start/previous token outside [0,V) counts as
+ *                 AS_ERR_NUMERIC)
+ * Errors: AS_ERR_INVALID_ARG, AS_ERR_UNSUPPORTED, AS_ERR_CUDA as for as_step.
+ */
+int as_decode_bigram(const void *d_table, int dtype, int V, long long ld,
+                     const int32_t *d_start, int S, int N, double u, int T, int eos,
+                     double temp, int top_k, double top_p,
+                     int32_t *d_seq, int32_t *d_len, double *d_codes_final,
+                     int32_t *d_lane_status, void *stream);
+
+/*
+ * The same loop from caller-supplied per-lane state (Algorithm 1's inputs: a
+ * code point and a prefix): lane i starts from previous token d_prev[i] and
+ * code d_codes_in[i].  With iid uniform codes this is ordinary ancestral
+ * sampling by inverse CDF (Sec. 3.1, last paragraph; Proposition 1); it also
+ * serves to split a decode and resume it (T steps = T1 steps, then T - T1 from
+ * the returned state).
+ */
+int as_decode_bigram_codes(const void *d_table, int dtype, int V, long long ld,
+                           const int32_t *d_prev, const double *d_codes_in, int lanes,
+                           int T, int eos, double temp, int top_k, double top_p,
+                           int32_t *d_seq, int32_t *d_len, double *d_codes_final,
+                           int32_t *d_lane_status, void *stream);
+
+/*
+ * Launch-shape overrides for measurement sweeps (process-wide, not thread-safe;
+ * 0 restores the built-in choice).  Keys:
+ *   AS_TUNE_STEP_PATH     1 = general path only, 2 = staged path wherever it applies
+ *   AS_TUNE_CLUSTER       CTAs per lane for the staged path (1, 2, 4, 8)
+ *   AS_TUNE_CTAS_PER_SM   resident CTAs per SM the grid is sized for
+ * Returns AS_ERR_INVALID_ARG for an unknown key or value.
+ */
+#define AS_TUNE_STEP_PATH 1
+#define AS_TUNE_CLUSTER 2
+#define AS_TUNE_CTAS_PER_SM 3
+int as_tune(int key, int value);
+
+/* Text of the calling thread's most recent error ("" if none). Never NULL. */
+const char *as_last_error(void);
+
+/* Library version: major * 1000 + minor. */
+int as_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ARITH_SAMPLING_H_ */

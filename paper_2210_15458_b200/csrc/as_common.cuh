@@ -1,0 +1,207 @@
+// Shared device helpers: order-preserving integer keys for bf16 / fp32 logits,
+// an fp64 exp for non-positive arguments, warp scans and reductions.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace asx {
+
+constexpr int DT_F32 = 0;
+constexpr int DT_BF16 = 1;
+
+constexpr int ST_OK = 0;
+constexpr int ST_TIMEOUT = -4;
+constexpr int ST_NUMERIC = -5;
+
+// Largest double below 1: rescaled codes are clamped into [0, ONE_BELOW].
+#define ASX_ONE_BELOW 0x1.fffffffffffffp-1
+
+// ---------------------------------------------------------------------------
+// Keys: an unsigned integer whose order equals the order of the stored float.
+// -inf maps to KEY_NINF (masked token); anything below it is a negative NaN,
+// anything >= KEY_PINF is +inf or a positive NaN.
+// ---------------------------------------------------------------------------
+template <int DT> struct Traits;
+
+template <> struct Traits<DT_F32> {
+    static constexpr int E = 4;            // elements per 16-byte vector
+    static constexpr int BYTES = 4;
+    static constexpr int KEYBITS = 32;
+    static constexpr uint32_t KEY_NINF = 0x007FFFFFu;
+    static constexpr uint32_t KEY_PINF = 0xFF800000u;
+    __device__ __forceinline__ static uint32_t key_of(uint32_t bits) {
+        return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+    }
+    __device__ __forceinline__ static float value_f(uint32_t key) {
+        uint32_t bits = (key & 0x80000000u) ? (key ^ 0x80000000u) : ~key;
+        return __uint_as_float(bits);
+    }
+    __device__ __forceinline__ static void unpack(const uint4& q, uint32_t (&k)[4]) {
+        k[0] = key_of(q.x); k[1] = key_of(q.y); k[2] = key_of(q.z); k[3] = key_of(q.w);
+    }
+    __device__ __forceinline__ static uint32_t load_key(const void* row, long long j) {
+        return key_of(reinterpret_cast<const uint32_t*>(row)[j]);
+    }
+};
+
+template <> struct Traits<DT_BF16> {
+    static constexpr int E = 8;
+    static constexpr int BYTES = 2;
+    static constexpr int KEYBITS = 16;
+    static constexpr uint32_t KEY_NINF = 0x007Fu;
+    static constexpr uint32_t KEY_PINF = 0xFF80u;
+    __device__ __forceinline__ static uint32_t key_of(uint32_t b16) {
+        return (b16 & 0x8000u) ? (~b16 & 0xFFFFu) : (b16 | 0x8000u);
+    }
+    __device__ __forceinline__ static float value_f(uint32_t key) {
+        uint32_t bits = (key & 0x8000u) ? (key ^ 0x8000u) : (~key & 0xFFFFu);
+        return __uint_as_float(bits << 16);
+    }
+    __device__ __forceinline__ static void unpack(const uint4& q, uint32_t (&k)[8]) {
+        k[0] = key_of(q.x & 0xFFFFu); k[1] = key_of(q.x >> 16);
+        k[2] = key_of(q.y & 0xFFFFu); k[3] = key_of(q.y >> 16);
+        k[4] = key_of(q.z & 0xFFFFu); k[5] = key_of(q.z >> 16);
+        k[6] = key_of(q.w & 0xFFFFu); k[7] = key_of(q.w >> 16);
+    }
+    __device__ __forceinline__ static uint32_t load_key(const void* row, long long j) {
+        return key_of(reinterpret_cast<const uint16_t*>(row)[j]);
+    }
+};
+
+// Keys of the E elements of vector `vi` of a row (element base vi*E); elements
+// at or past V read as masked.  `vec_ok`: the row start is 16-byte aligned.
+template <int DT>
+__device__ __forceinline__ void load_vec_keys(const void* row, int V, int vi, bool vec_ok,
+                                              uint32_t (&k)[Traits<DT>::E]) {
+    using Tr = Traits<DT>;
+    const int base = vi * Tr::E;
+    if (vec_ok && base + Tr::E <= V) {
+        const uint4 q = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row) +
+                                                        (size_t)base * Tr::BYTES);
+        Tr::unpack(q, k);
+    } else {
+#pragma unroll
+        for (int e = 0; e < Tr::E; ++e)
+            k[e] = (base + e < V) ? Tr::load_key(row, base + e) : Tr::KEY_NINF;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// exp(y) for y <= 0 in fp64: y = (64 n + j) ln2/64 + f, |f| <= ln2/128;
+// exp(y) = 2^n * 2^(j/64) * exp(f), exp(f) by a degree-5 polynomial
+// (truncation ~3e-17).  tbl[j] = 2^(j/64).  Arguments below -700 return 0.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ double exp_nonpos(double y, const double* __restrict__ tbl) {
+    if (!(y >= -700.0)) return 0.0;
+    const double MAGIC = 6755399441055744.0;          // 1.5 * 2^52: rounds to integer
+    double r = fma(y, 0x1.71547652b82fep+6, MAGIC);    // y * 64/ln2
+    const int k = __double2loint(r);
+    r -= MAGIC;
+    double f = fma(r, -0x1.62e42fe000000p-7, y);       // ln2/64, high part (24 low bits zero)
+    f = fma(r, -0x1.f473de6af278fp-36, f);             // ln2/64, low part
+    double p = fma(f, 1.0 / 120.0, 1.0 / 24.0);
+    p = fma(p, f, 1.0 / 6.0);
+    p = fma(p, f, 0.5);
+    p = fma(p, f, 1.0);
+    p = fma(p, f, 1.0);
+    const double v = tbl[k & 63] * p;
+    const int n = k >> 6;                              // floor((64n+j)/64), n in [-1010, 0]
+    return __hiloint2double(__double2hiint(v) + (n << 20), __double2loint(v));
+}
+
+// 2^(j/64), j = 0..63, correctly rounded.
+__device__ const double ASX_T64[64] = {
+    0x1.0000000000000p+0, 0x1.02c9a3e778061p+0, 0x1.059b0d3158574p+0, 0x1.0874518759bc8p+0,
+    0x1.0b5586cf9890fp+0, 0x1.0e3ec32d3d1a2p+0, 0x1.11301d0125b51p+0, 0x1.1429aaea92de0p+0,
+    0x1.172b83c7d517bp+0, 0x1.1a35beb6fcb75p+0, 0x1.1d4873168b9aap+0, 0x1.2063b88628cd6p+0,
+    0x1.2387a6e756238p+0, 0x1.26b4565e27cddp+0, 0x1.29e9df51fdee1p+0, 0x1.2d285a6e4030bp+0,
+    0x1.306fe0a31b715p+0, 0x1.33c08b26416ffp+0, 0x1.371a7373aa9cbp+0, 0x1.3a7db34e59ff7p+0,
+    0x1.3dea64c123422p+0, 0x1.4160a21f72e2ap+0, 0x1.44e086061892dp+0, 0x1.486a2b5c13cd0p+0,
+    0x1.4bfdad5362a27p+0, 0x1.4f9b2769d2ca7p+0, 0x1.5342b569d4f82p+0, 0x1.56f4736b527dap+0,
+    0x1.5ab07dd485429p+0, 0x1.5e76f15ad2148p+0, 0x1.6247eb03a5585p+0, 0x1.6623882552225p+0,
+    0x1.6a09e667f3bcdp+0, 0x1.6dfb23c651a2fp+0, 0x1.71f75e8ec5f74p+0, 0x1.75feb564267c9p+0,
+    0x1.7a11473eb0187p+0, 0x1.7e2f336cf4e62p+0, 0x1.82589994cce13p+0, 0x1.868d99b4492edp+0,
+    0x1.8ace5422aa0dbp+0, 0x1.8f1ae99157736p+0, 0x1.93737b0cdc5e5p+0, 0x1.97d829fde4e50p+0,
+    0x1.9c49182a3f090p+0, 0x1.a0c667b5de565p+0, 0x1.a5503b23e255dp+0, 0x1.a9e6b5579fdbfp+0,
+    0x1.ae89f995ad3adp+0, 0x1.b33a2b84f15fbp+0, 0x1.b7f76f2fb5e47p+0, 0x1.bcc1e904bc1d2p+0,
+    0x1.c199bdd85529cp+0, 0x1.c67f12e57d14bp+0, 0x1.cb720dcef9069p+0, 0x1.d072d4a07897cp+0,
+    0x1.d5818dcfba487p+0, 0x1.da9e603db3285p+0, 0x1.dfc97337b9b5fp+0, 0x1.e502ee78b3ff6p+0,
+    0x1.ea4afa2a490dap+0, 0x1.efa1bee615a27p+0, 0x1.f50765b6e4540p+0, 0x1.fa7c1819e90d8p+0};
+
+// Copies the table into shared memory (divergent indices make a constant-bank
+// read serialise; a shared-memory read does not).  Caller synchronises after.
+__device__ __forceinline__ void fill_exp_table(double* tbl, int tid) {
+    if (tid < 64) tbl[tid] = ASX_T64[tid];
+}
+
+// ---------------------------------------------------------------------------
+// Warp primitives (all 32 lanes active).
+// ---------------------------------------------------------------------------
+constexpr unsigned FULL = 0xFFFFFFFFu;
+
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+    return v;
+}
+__device__ __forceinline__ int warp_sum_i(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+    return v;
+}
+__device__ __forceinline__ unsigned warp_max_u(unsigned v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(FULL, v, o));
+    return v;
+}
+__device__ __forceinline__ unsigned warp_min_u(unsigned v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(FULL, v, o));
+    return v;
+}
+// inclusive scans over lanes 0..31 in lane order
+__device__ __forceinline__ double warp_incl_scan_d(double v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double u = __shfl_up_sync(FULL, v, o);
+        if (lane >= o) v += u;
+    }
+    return v;
+}
+__device__ __forceinline__ int warp_incl_scan_i(int v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(FULL, v, o);
+        if (lane >= o) v += u;
+    }
+    return v;
+}
+// inclusive suffix sums: lane l gets the sum over lanes >= l
+__device__ __forceinline__ double warp_suffix_d(double v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double u = __shfl_down_sync(FULL, v, o);
+        if (lane + o < 32) v += u;
+    }
+    return v;
+}
+__device__ __forceinline__ int warp_suffix_i(int v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_down_sync(FULL, v, o);
+        if (lane + o < 32) v += u;
+    }
+    return v;
+}
+
+// Result of one decode step for one lane, identical in every thread of the CTA.
+struct LaneResult {
+    int token;
+    int status;
+    int n_kept;
+    double code_out;
+    double p_tok;
+    double cdf_lo;
+};
+
+}  // namespace asx
