@@ -1,0 +1,325 @@
+// C-ABI entry points (see include/arith_sampling.h) and the kernels behind them.
+#include "../../include/arith_sampling.h"
+#include "as_generic.cuh"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+namespace asx {
+
+// ---------------------------------------------------------------------------
+// host-side state
+// ---------------------------------------------------------------------------
+static thread_local char g_err[512] = "";
+static int g_tune_path = 0, g_tune_cluster = 0, g_tune_ctas = 0;
+
+static int set_err(int code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+static int cuda_fail(cudaError_t e, const char* what) {
+    return set_err(AS_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+struct DeviceInfo {
+    int sms = 0;
+    bool ok = false;
+};
+static DeviceInfo g_dev[64];
+
+static int device_info(const DeviceInfo** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= 64) return set_err(AS_ERR_CUDA, "device ordinal %d out of range", dev);
+    if (!g_dev[dev].ok) {
+        int sms = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+        g_dev[dev].sms = sms;
+        g_dev[dev].ok = true;
+    }
+    *out = &g_dev[dev];
+    return AS_OK;
+}
+
+struct DiagPtrs {
+    double* p_tok;
+    double* cdf_lo;
+    int* n_kept;
+    int* lane_status;
+};
+
+// ---------------------------------------------------------------------------
+// kernels
+// ---------------------------------------------------------------------------
+constexpr int GEN_NT = 512;
+
+__global__ void lattice_kernel(int N, double u, double* __restrict__ codes) {
+    // Definition "Arithmetic sampling" (Sec. 4.2), spacing 1/N: c_j = (j + u)/N mod 1
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j < N) {
+        double c = ((double)j + u) / (double)N;
+        if (c >= 1.0) c -= 1.0;
+        codes[j] = c;
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(GEN_NT)
+step_generic_kernel(const void* __restrict__ logits, int lanes, int V, long long ld,
+                    const double* codes, double inv_tau, int top_k, double top_p,
+                    int* __restrict__ tokens, double* codes_out, DiagPtrs diag) {
+    __shared__ GenericSmem<GEN_NT> sm;
+    for (int ln = blockIdx.x; ln < lanes; ln += gridDim.x) {
+        const char* row = reinterpret_cast<const char*>(logits) + (size_t)ln * (size_t)ld * Traits<DT>::BYTES;
+        const bool vec_ok = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
+        const double c = codes[ln];
+        GenericLane<DT, GEN_NT> g(sm, row, V, vec_ok);
+        const LaneResult r = g.run(c, inv_tau, top_k, top_p);
+        if (threadIdx.x == 0) {
+            tokens[ln] = r.token;
+            codes_out[ln] = r.code_out;
+            if (diag.p_tok) diag.p_tok[ln] = r.p_tok;
+            if (diag.cdf_lo) diag.cdf_lo[ln] = r.cdf_lo;
+            if (diag.n_kept) diag.n_kept[ln] = r.n_kept;
+            if (diag.lane_status) diag.lane_status[ln] = r.status;
+        }
+    }
+}
+
+// Algorithm 1's REPEAT ... UNTIL loop for one lane per CTA over a bigram table.
+// Lane state comes either from (start, N, u) [codes_in == nullptr] or from
+// (prev, codes_in).
+template <int DT>
+__global__ void __launch_bounds__(GEN_NT)
+decode_generic_kernel(const void* __restrict__ table, int V, long long ld,
+                      const int* __restrict__ start_or_prev, const double* __restrict__ codes_in,
+                      int lanes, int N, double u, int T, int eos, double inv_tau, int top_k,
+                      double top_p, int* __restrict__ seq, int* __restrict__ len,
+                      double* __restrict__ codes_final, int* __restrict__ lane_status) {
+    __shared__ GenericSmem<GEN_NT> sm;
+    for (int ln = blockIdx.x; ln < lanes; ln += gridDim.x) {
+        int prev;
+        double c;
+        if (codes_in) {
+            prev = start_or_prev[ln];
+            c = codes_in[ln];
+        } else {
+            prev = start_or_prev[ln / N];
+            c = ((double)(ln % N) + u) / (double)N;
+            if (c >= 1.0) c -= 1.0;
+        }
+        int n = 0, status = ST_OK;
+        for (int t = 0; t < T; ++t) {
+            if (prev < 0 || prev >= V) { status = ST_NUMERIC; break; }
+            const char* row = reinterpret_cast<const char*>(table) + (size_t)prev * (size_t)ld * Traits<DT>::BYTES;
+            const bool vec_ok = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
+            GenericLane<DT, GEN_NT> g(sm, row, V, vec_ok);
+            const LaneResult r = g.run(c, inv_tau, top_k, top_p);
+            if (r.status != ST_OK) { status = r.status; break; }
+            if (threadIdx.x == 0) seq[(size_t)ln * T + t] = r.token;
+            n = t + 1;
+            c = r.code_out;
+            prev = r.token;
+            if (r.token == eos) break;
+        }
+        for (int t = n + (int)threadIdx.x; t < T; t += GEN_NT) seq[(size_t)ln * T + t] = -1;
+        if (threadIdx.x == 0) {
+            len[ln] = n;
+            if (codes_final) codes_final[ln] = c;
+            if (lane_status) lane_status[ln] = status;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// argument checks
+// ---------------------------------------------------------------------------
+static int check_common(const void* data, int dtype, int V, long long ld, double temp, double top_p) {
+    if (!data) return set_err(AS_ERR_INVALID_ARG, "logits/table pointer is NULL");
+    if (dtype != AS_F32 && dtype != AS_BF16) return set_err(AS_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    if (V < 1) return set_err(AS_ERR_INVALID_ARG, "V = %d must be >= 1", V);
+    if (V > AS_MAX_V) return set_err(AS_ERR_UNSUPPORTED, "V = %d exceeds AS_MAX_V = %d", V, AS_MAX_V);
+    if (ld < V) return set_err(AS_ERR_INVALID_ARG, "ld = %lld is smaller than V = %d", ld, V);
+    if (!(temp > 0.0) || std::isinf(temp)) return set_err(AS_ERR_INVALID_ARG, "temp must be positive and finite");
+    if (std::isnan(top_p)) return set_err(AS_ERR_INVALID_ARG, "top_p is NaN");
+    const uintptr_t a = reinterpret_cast<uintptr_t>(data);
+    if (a % (dtype == AS_F32 ? 4 : 2)) return set_err(AS_ERR_INVALID_ARG, "logits/table pointer is not element-aligned");
+    return AS_OK;
+}
+
+static int grid_for(int lanes, int sms, int per_sm) {
+    const long long cap = (long long)sms * per_sm;
+    return (int)(lanes < cap ? lanes : cap);
+}
+
+}  // namespace asx
+
+using namespace asx;
+
+extern "C" {
+
+int as_version(void) { return 1000; }
+
+const char* as_last_error(void) { return g_err; }
+
+int as_tune(int key, int value) {
+    switch (key) {
+        case AS_TUNE_STEP_PATH:
+            if (value < 0 || value > 2) return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_STEP_PATH takes 0, 1 or 2");
+            g_tune_path = value;
+            return AS_OK;
+        case AS_TUNE_CLUSTER:
+            if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8)
+                return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_CLUSTER takes 0, 1, 2, 4 or 8");
+            g_tune_cluster = value;
+            return AS_OK;
+        case AS_TUNE_CTAS_PER_SM:
+            if (value < 0 || value > 32) return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_CTAS_PER_SM takes 0..32");
+            g_tune_ctas = value;
+            return AS_OK;
+        default:
+            return set_err(AS_ERR_INVALID_ARG, "unknown tuning key %d", key);
+    }
+}
+
+int as_lattice_codes(int N, double u, double* d_codes, void* stream) {
+    if (N < 1) return set_err(AS_ERR_INVALID_ARG, "N = %d must be >= 1", N);
+    if (!(u >= 0.0 && u < 1.0)) return set_err(AS_ERR_INVALID_ARG, "shift u must lie in [0,1)");
+    if (!d_codes) return set_err(AS_ERR_INVALID_ARG, "d_codes is NULL");
+    const DeviceInfo* di;
+    int rc = device_info(&di);
+    if (rc != AS_OK) return rc;
+    lattice_kernel<<<(N + 255) / 256, 256, 0, (cudaStream_t)stream>>>(N, u, d_codes);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "lattice kernel launch");
+    return AS_OK;
+}
+
+int as_step(const void* d_logits, int dtype, int lanes, int V, long long ld, const double* d_codes,
+            double temp, int top_k, double top_p, int32_t* d_tokens, double* d_codes_out,
+            const as_step_diag* diag, void* stream) {
+    if (lanes < 0) return set_err(AS_ERR_INVALID_ARG, "lanes = %d must be >= 0", lanes);
+    int rc = check_common(d_logits, dtype, V, ld, temp, top_p);
+    if (rc != AS_OK) return rc;
+    if (!d_codes || !d_tokens || !d_codes_out) return set_err(AS_ERR_INVALID_ARG, "codes / tokens / codes_out pointer is NULL");
+    if (lanes == 0) return AS_OK;
+    const DeviceInfo* di;
+    rc = device_info(&di);
+    if (rc != AS_OK) return rc;
+    DiagPtrs dp = {nullptr, nullptr, nullptr, nullptr};
+    if (diag) dp = {diag->d_p_tok, diag->d_cdf_lo, diag->d_n_kept, diag->d_lane_status};
+    if (top_k < 0 || top_k >= V) top_k = 0;
+    if (!(top_p > 0.0 && top_p < 1.0)) top_p = 1.0;
+    const double inv_tau = 1.0 / temp;
+    const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == AS_F32)
+        step_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, inv_tau, top_k, top_p, d_tokens, d_codes_out, dp);
+    else
+        step_generic_kernel<DT_BF16><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, inv_tau, top_k, top_p, d_tokens, d_codes_out, dp);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "step kernel launch");
+    return AS_OK;
+}
+
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+size_t as_step_host_work_bytes(int dtype, int lanes, long long ld) {
+    if (lanes < 0 || ld < 0 || (dtype != AS_F32 && dtype != AS_BF16)) return 0;
+    const size_t esz = dtype == AS_F32 ? 4 : 2;
+    return align256((size_t)lanes * (size_t)ld * esz) + 2 * align256((size_t)lanes * 8) +
+           2 * align256((size_t)lanes * 4) + 256;
+}
+
+int as_step_host(const void* h_logits, int dtype, int lanes, int V, long long ld, const double* h_codes,
+                 double temp, int top_k, double top_p, int32_t* h_tokens, double* h_codes_out,
+                 int32_t* h_lane_status, void* d_work, size_t work_bytes, void* stream) {
+    if (lanes < 0) return set_err(AS_ERR_INVALID_ARG, "lanes = %d must be >= 0", lanes);
+    int rc = check_common(h_logits, dtype, V, ld, temp, top_p);
+    if (rc != AS_OK) return rc;
+    if (!h_codes || !h_tokens || !h_codes_out) return set_err(AS_ERR_INVALID_ARG, "host codes / tokens / codes_out pointer is NULL");
+    if (lanes == 0) return AS_OK;
+    if (!d_work || (reinterpret_cast<uintptr_t>(d_work) & 255)) return set_err(AS_ERR_INVALID_ARG, "d_work must be a 256-byte aligned device pointer");
+    if (work_bytes < as_step_host_work_bytes(dtype, lanes, ld)) return set_err(AS_ERR_INVALID_ARG, "work_bytes is smaller than as_step_host_work_bytes()");
+    const size_t esz = dtype == AS_F32 ? 4 : 2;
+    const size_t nlog = (size_t)lanes * (size_t)ld * esz;
+    char* w = reinterpret_cast<char*>(d_work);
+    void* d_logits = w;                 w += align256(nlog);
+    double* d_codes = (double*)w;       w += align256((size_t)lanes * 8);
+    double* d_codes_out = (double*)w;   w += align256((size_t)lanes * 8);
+    int32_t* d_tokens = (int32_t*)w;    w += align256((size_t)lanes * 4);
+    int32_t* d_status = (int32_t*)w;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e;
+    // the last row may be shorter than ld in the caller's buffer: copy lanes-1 full pitches + V
+    const size_t ncopy = ((size_t)(lanes - 1) * (size_t)ld + (size_t)V) * esz;
+    if ((e = cudaMemcpyAsync(d_logits, h_logits, ncopy, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "copy logits to device");
+    if ((e = cudaMemcpyAsync(d_codes, h_codes, (size_t)lanes * 8, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "copy codes to device");
+    as_step_diag dg = {nullptr, nullptr, nullptr, d_status};
+    rc = as_step(d_logits, dtype, lanes, V, ld, d_codes, temp, top_k, top_p, d_tokens, d_codes_out, &dg, stream);
+    if (rc != AS_OK) return rc;
+    if ((e = cudaMemcpyAsync(h_tokens, d_tokens, (size_t)lanes * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "copy tokens to host");
+    if ((e = cudaMemcpyAsync(h_codes_out, d_codes_out, (size_t)lanes * 8, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "copy codes to host");
+    if (h_lane_status && (e = cudaMemcpyAsync(h_lane_status, d_status, (size_t)lanes * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "copy status to host");
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(e, "stream synchronize");
+    return AS_OK;
+}
+
+static int decode_common(const void* d_table, int dtype, int V, long long ld, const int32_t* d_tok,
+                         const double* d_codes_in, int lanes, int N, double u, int T, int eos,
+                         double temp, int top_k, double top_p, int32_t* d_seq, int32_t* d_len,
+                         double* d_codes_final, int32_t* d_lane_status, void* stream) {
+    int rc = check_common(d_table, dtype, V, ld, temp, top_p);
+    if (rc != AS_OK) return rc;
+    if (T < 0) return set_err(AS_ERR_INVALID_ARG, "T = %d must be >= 0", T);
+    if (!d_tok) return set_err(AS_ERR_INVALID_ARG, "start / prev token pointer is NULL");
+    if (!d_len || (!d_seq && T > 0)) return set_err(AS_ERR_INVALID_ARG, "seq / len pointer is NULL");
+    if (lanes == 0) return AS_OK;
+    const DeviceInfo* di;
+    rc = device_info(&di);
+    if (rc != AS_OK) return rc;
+    if (top_k < 0 || top_k >= V) top_k = 0;
+    if (!(top_p > 0.0 && top_p < 1.0)) top_p = 1.0;
+    const double inv_tau = 1.0 / temp;
+    const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == AS_F32)
+        decode_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_table, V, ld, d_tok, d_codes_in, lanes, N, u, T, eos, inv_tau, top_k, top_p, d_seq, d_len, d_codes_final, d_lane_status);
+    else
+        decode_generic_kernel<DT_BF16><<<grid, GEN_NT, 0, st>>>(d_table, V, ld, d_tok, d_codes_in, lanes, N, u, T, eos, inv_tau, top_k, top_p, d_seq, d_len, d_codes_final, d_lane_status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "decode kernel launch");
+    return AS_OK;
+}
+
+int as_decode_bigram(const void* d_table, int dtype, int V, long long ld, const int32_t* d_start, int S,
+                     int N, double u, int T, int eos, double temp, int top_k, double top_p,
+                     int32_t* d_seq, int32_t* d_len, double* d_codes_final, int32_t* d_lane_status,
+                     void* stream) {
+    if (S < 0) return set_err(AS_ERR_INVALID_ARG, "S = %d must be >= 0", S);
+    if (N < 1) return set_err(AS_ERR_INVALID_ARG, "N = %d must be >= 1", N);
+    if (!(u >= 0.0 && u < 1.0)) return set_err(AS_ERR_INVALID_ARG, "shift u must lie in [0,1)");
+    if ((long long)S * N > 0x7FFFFFFFLL) return set_err(AS_ERR_UNSUPPORTED, "S*N exceeds 2^31-1 lanes");
+    return decode_common(d_table, dtype, V, ld, d_start, nullptr, S * N, N, u, T, eos, temp, top_k, top_p,
+                         d_seq, d_len, d_codes_final, d_lane_status, stream);
+}
+
+int as_decode_bigram_codes(const void* d_table, int dtype, int V, long long ld, const int32_t* d_prev,
+                           const double* d_codes_in, int lanes, int T, int eos, double temp, int top_k,
+                           double top_p, int32_t* d_seq, int32_t* d_len, double* d_codes_final,
+                           int32_t* d_lane_status, void* stream) {
+    if (lanes < 0) return set_err(AS_ERR_INVALID_ARG, "lanes = %d must be >= 0", lanes);
+    if (!d_codes_in) return set_err(AS_ERR_INVALID_ARG, "d_codes_in is NULL");
+    return decode_common(d_table, dtype, V, ld, d_prev, d_codes_in, lanes, 1, 0.0, T, eos, temp, top_k, top_p,
+                         d_seq, d_len, d_codes_final, d_lane_status, stream);
+}
+
+}  // extern "C"

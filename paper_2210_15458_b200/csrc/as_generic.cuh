@@ -1,0 +1,478 @@
+// General decode step for one lane, run by one CTA on a row it can address
+// (global or shared memory).  Correct for every input: any V, any top_k /
+// top_p, ties, masked tokens.  All masses are fp64.
+//
+// Steps (Algorithm 1's loop body with the logit modifiers):
+//   1. max key, non-finite detection
+//   2. top-k: exact radix select on the ordered keys -> threshold key T and the
+//      number of elements equal to T that are kept (lowest indices first)
+//   3. Z1 = sum of exp((l - l_max)/temp) over the kept set
+//   4. nucleus: radix select on the keys weighted by mass -> new threshold
+//   5. per-chunk masses in index order, exclusive scan, Z
+//   6. the chunk, then the element, whose interval holds c*Z; rescale
+//
+// The row is cut into chunks of 32*E*R consecutive elements, one warp per chunk
+// at a time, lane l of the warp owning E consecutive elements of each of the R
+// sub-rows, so that (chunk, sub-row, lane, element) order is index order.
+#pragma once
+#include "as_common.cuh"
+#include <limits.h>
+
+namespace asx {
+
+constexpr int MAXCH = 512;  // chunks per row (R grows so that this suffices)
+
+// kept(key) = key > T, or key == T and: eq_mode 1 -> always; eq_mode 2 -> only the
+// first `need` such elements in index order; eq_mode 0 -> never.
+struct Pred {
+    uint32_t T;
+    int need;
+    int eq_mode;
+};
+
+template <int NT>
+struct GenericSmem {
+    double chunk_sum[MAXCH + 1];
+    int chunk_eq[MAXCH + 1];
+    double hist_mass[256];
+    int hist_cnt[256];
+    double red_d[NT / 32];
+    unsigned red_u[NT / 32];
+    unsigned red_u2[NT / 32];
+    int red_i[NT / 32];
+    double exp_tbl[64];
+    double b_d[4];
+    int b_i[4];
+    unsigned b_u[2];
+    LaneResult res;
+};
+
+template <int DT, int NT>
+struct GenericLane {
+    using Tr = Traits<DT>;
+    static constexpr int E = Tr::E;
+    static constexpr int NW = NT / 32;
+
+    GenericSmem<NT>& sm;
+    const void* row;
+    int V;
+    bool vec_ok;
+    int nvec, R, nchunks;
+    int tid, lane, warp;
+    double lmax, inv_tau;
+
+    __device__ GenericLane(GenericSmem<NT>& s, const void* row_, int V_, bool vec_ok_)
+        : sm(s), row(row_), V(V_), vec_ok(vec_ok_) {
+        tid = threadIdx.x;
+        lane = tid & 31;
+        warp = tid >> 5;
+        nvec = (V + E - 1) / E;
+        const int rows32 = (nvec + 31) / 32;
+        R = (rows32 + MAXCH - 1) / MAXCH;
+        nchunks = (rows32 + R - 1) / R;
+    }
+
+    __device__ __forceinline__ void chunk_keys(int ci, int r, uint32_t (&k)[E], int& base) const {
+        const int vi = (ci * R + r) * 32 + lane;
+        base = vi * E;
+        if (vi < nvec) {
+            load_vec_keys<DT>(row, V, vi, vec_ok, k);
+        } else {
+#pragma unroll
+            for (int e = 0; e < E; ++e) k[e] = Tr::KEY_NINF;
+        }
+    }
+
+    // index-order rank, among the elements equal to p.T, of this lane's first one
+    __device__ __forceinline__ int lane_rank0(const uint32_t (&k)[E], const Pred& p, int& tie_run) const {
+        if (p.eq_mode != 2) return 0;
+        int cnt = 0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) cnt += (k[e] == p.T);
+        const int incl = warp_incl_scan_i(cnt, lane);
+        const int rank0 = tie_run + incl - cnt;
+        tie_run += __shfl_sync(FULL, incl, 31);
+        return rank0;
+    }
+
+    __device__ __forceinline__ unsigned kept_bits(const uint32_t (&k)[E], const Pred& p, int rank0) const {
+        unsigned m = 0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            if (k[e] > p.T) {
+                m |= 1u << e;
+            } else if (k[e] == p.T) {
+                if (p.eq_mode == 1 || (p.eq_mode == 2 && rank0 < p.need)) m |= 1u << e;
+                ++rank0;
+            }
+        }
+        return m;
+    }
+
+    __device__ __forceinline__ double mass(uint32_t key) const {
+        return exp_nonpos(((double)Tr::value_f(key) - lmax) * inv_tau, sm.exp_tbl);
+    }
+
+    // exclusive scan of a[0..n) in place by warp 0; a[n] receives the total
+    template <typename T>
+    __device__ void scan_exclusive(T* a, int n) {
+        if (warp == 0) {
+            const int per = (n + 31) / 32;
+            const int b = min(lane * per, n), e = min(b + per, n);
+            T s = 0;
+            for (int i = b; i < e; ++i) s += a[i];
+            T incl = s;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const T u = __shfl_up_sync(FULL, incl, o);
+                if (lane >= o) incl += u;
+            }
+            T run = __shfl_up_sync(FULL, incl, 1);
+            if (lane == 0) run = 0;
+            for (int i = b; i < e; ++i) {
+                const T v = a[i];
+                a[i] = run;
+                run += v;
+            }
+            if (lane == 31) a[n] = incl;
+        }
+        __syncthreads();
+    }
+
+    // chunk_eq[ci] <- number of elements equal to T in chunks before ci
+    __device__ void tie_prepass(uint32_t T) {
+        for (int ci = warp; ci < nchunks; ci += NW) {
+            int cnt = 0;
+            for (int r = 0; r < R; ++r) {
+                uint32_t k[E];
+                int base;
+                chunk_keys(ci, r, k, base);
+#pragma unroll
+                for (int e = 0; e < E; ++e) cnt += (k[e] == T);
+            }
+            cnt = warp_sum_i(cnt);
+            if (lane == 0) sm.chunk_eq[ci] = cnt;
+        }
+        __syncthreads();
+        scan_exclusive(sm.chunk_eq, nchunks);
+    }
+
+    // chunk_sum[ci] <- mass of the kept elements of chunk ci
+    __device__ void sum_pass(const Pred& p) {
+        for (int ci = warp; ci < nchunks; ci += NW) {
+            int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[ci] : 0;
+            double local = 0.0;
+            for (int r = 0; r < R; ++r) {
+                uint32_t k[E];
+                int base;
+                chunk_keys(ci, r, k, base);
+                const int rank0 = lane_rank0(k, p, tie_run);
+                const unsigned bits = kept_bits(k, p, rank0);
+#pragma unroll
+                for (int e = 0; e < E; ++e)
+                    if (bits & (1u << e)) local += mass(k[e]);
+            }
+            local = warp_sum_d(local);
+            if (lane == 0) sm.chunk_sum[ci] = local;
+        }
+        __syncthreads();
+    }
+
+    // histogram of digit (key >> shift) & 255 over kept elements whose key matches
+    // `prefix` on `mask`; counts always, masses if MASS
+    template <bool MASS>
+    __device__ void hist_pass(const Pred& p, uint32_t prefix, uint32_t mask, int shift) {
+        for (int i = tid; i < 256; i += NT) {
+            sm.hist_cnt[i] = 0;
+            sm.hist_mass[i] = 0.0;
+        }
+        __syncthreads();
+        for (int ci = warp; ci < nchunks; ci += NW) {
+            int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[ci] : 0;
+            for (int r = 0; r < R; ++r) {
+                uint32_t k[E];
+                int base;
+                chunk_keys(ci, r, k, base);
+                const int rank0 = lane_rank0(k, p, tie_run);
+                const unsigned bits = kept_bits(k, p, rank0);
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    if ((bits & (1u << e)) && (k[e] & mask) == prefix) {
+                        const int d = (k[e] >> shift) & 255;
+                        atomicAdd(&sm.hist_cnt[d], 1);
+                        if (MASS) atomicAdd(&sm.hist_mass[d], mass(k[e]));
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+
+    // Largest non-empty digit d with (acc + weight of digits >= d) >= target; if none
+    // (rounding), the smallest non-empty digit.  Outputs through shared memory:
+    // b_i[0] = d, b_i[1] = acc_cnt + count(digits > d), b_i[2] = count(d),
+    // b_d[0] = acc_mass + mass(digits > d).
+    template <bool MASS>
+    __device__ void choose_digit(int acc_cnt, double acc_mass, int k_target, double m_target) {
+        if (warp == 0) {
+            int c[8];
+            double m[8];
+            int lc = 0;
+            double lm = 0.0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                c[e] = sm.hist_cnt[lane * 8 + e];
+                m[e] = MASS ? sm.hist_mass[lane * 8 + e] : 0.0;
+                lc += c[e];
+                lm += m[e];
+            }
+            const int suf_c = warp_suffix_i(lc, lane);
+            const double suf_m = MASS ? warp_suffix_d(lm, lane) : 0.0;
+            int above_c = __shfl_down_sync(FULL, suf_c, 1);
+            double above_m = __shfl_down_sync(FULL, suf_m, 1);
+            if (lane == 31) { above_c = 0; above_m = 0.0; }
+            int best = -1, best_above_c = 0, best_c = 0;
+            double best_above_m = 0.0;
+            int low = -1, low_above_c = 0, low_c = 0;
+            double low_above_m = 0.0;
+            int run_c = above_c;
+            double run_m = above_m;
+#pragma unroll
+            for (int e = 7; e >= 0; --e) {
+                if (c[e] > 0) {
+                    const bool ok = MASS ? (acc_mass + (run_m + m[e]) >= m_target)
+                                         : (acc_cnt + run_c + c[e] >= k_target);
+                    if (ok && best < 0) {
+                        best = lane * 8 + e; best_above_c = run_c; best_above_m = run_m; best_c = c[e];
+                    }
+                    low = lane * 8 + e; low_above_c = run_c; low_above_m = run_m; low_c = c[e];
+                }
+                run_c += c[e];
+                run_m += m[e];
+            }
+            const unsigned bal = __ballot_sync(FULL, best >= 0);
+            int src;
+            if (bal) {
+                src = 31 - __clz(bal);
+            } else {
+                const unsigned bal2 = __ballot_sync(FULL, low >= 0);
+                src = bal2 ? (__ffs(bal2) - 1) : 0;
+                best = low; best_above_c = low_above_c; best_above_m = low_above_m; best_c = low_c;
+            }
+            best = __shfl_sync(FULL, best, src);
+            best_above_c = __shfl_sync(FULL, best_above_c, src);
+            best_above_m = __shfl_sync(FULL, best_above_m, src);
+            best_c = __shfl_sync(FULL, best_c, src);
+            if (lane == 0) {
+                sm.b_i[0] = best < 0 ? 0 : best;
+                sm.b_i[1] = acc_cnt + best_above_c;
+                sm.b_i[2] = best_c;
+                sm.b_d[0] = acc_mass + best_above_m;
+            }
+        }
+        __syncthreads();
+    }
+
+    __device__ LaneResult fail(double c_in, int status) {
+        LaneResult r;
+        r.token = -1; r.status = status; r.n_kept = 0; r.code_out = c_in; r.p_tok = 0.0; r.cdf_lo = 0.0;
+        return r;
+    }
+
+    __device__ LaneResult run(double c_in, double inv_tau_, int top_k, double top_p) {
+        inv_tau = inv_tau_;
+        fill_exp_table(sm.exp_tbl, tid);
+        double c = c_in;
+        const bool code_bad = !(c >= 0.0 && c <= 1.0);
+        if (c == 1.0) c = ASX_ONE_BELOW;
+
+        // ---- 1. extremes and finite count
+        unsigned kmax = 0, kmin = 0xFFFFFFFFu;
+        int nfin = 0;
+        for (int vi = tid; vi < nvec; vi += NT) {
+            uint32_t k[E];
+            load_vec_keys<DT>(row, V, vi, vec_ok, k);
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                kmax = max(kmax, k[e]);
+                kmin = min(kmin, k[e]);
+                nfin += (k[e] > Tr::KEY_NINF);
+            }
+        }
+        kmax = warp_max_u(kmax);
+        kmin = warp_min_u(kmin);
+        nfin = warp_sum_i(nfin);
+        if (lane == 0) { sm.red_u[warp] = kmax; sm.red_u2[warp] = kmin; sm.red_i[warp] = nfin; }
+        __syncthreads();
+        kmax = 0; kmin = 0xFFFFFFFFu; nfin = 0;
+        for (int w = 0; w < NW; ++w) {
+            kmax = max(kmax, sm.red_u[w]);
+            kmin = min(kmin, sm.red_u2[w]);
+            nfin += sm.red_i[w];
+        }
+        __syncthreads();
+        if (code_bad || kmin < Tr::KEY_NINF || kmax >= Tr::KEY_PINF || kmax == Tr::KEY_NINF)
+            return fail(c_in, ST_NUMERIC);
+        lmax = (double)Tr::value_f(kmax);
+
+        Pred p;
+        p.T = Tr::KEY_NINF; p.need = 0; p.eq_mode = 0;     // every finite logit
+        int n_kept = nfin;
+
+        // ---- 2. top-k
+        if (top_k > 0 && top_k < nfin) {
+            uint32_t prefix = 0, mask = 0;
+            int acc = 0, eq = 0;
+            for (int shift = Tr::KEYBITS - 8; shift >= 0; shift -= 8) {
+                hist_pass<false>(p, prefix, mask, shift);
+                choose_digit<false>(acc, 0.0, top_k, 0.0);
+                prefix |= (uint32_t)sm.b_i[0] << shift;
+                mask |= 0xFFu << shift;
+                acc = sm.b_i[1];
+                eq = sm.b_i[2];
+                __syncthreads();
+            }
+            p.T = prefix;
+            p.need = top_k - acc;
+            p.eq_mode = (p.need < eq) ? 2 : 1;
+            n_kept = top_k;
+            if (p.eq_mode == 2) tie_prepass(p.T);
+        }
+
+        // ---- 3. masses of the kept set
+        sum_pass(p);
+        scan_exclusive(sm.chunk_sum, nchunks);
+
+        // ---- 4. nucleus on the distribution renormalised over the survivors
+        if (top_p > 0.0 && top_p < 1.0) {
+            const double target = top_p * sm.chunk_sum[nchunks];
+            __syncthreads();
+            uint32_t prefix = 0, mask = 0;
+            int acc_c = 0, eq = 0;
+            double acc_m = 0.0;
+            for (int shift = Tr::KEYBITS - 8; shift >= 0; shift -= 8) {
+                hist_pass<true>(p, prefix, mask, shift);
+                choose_digit<true>(acc_c, acc_m, 0, target);
+                prefix |= (uint32_t)sm.b_i[0] << shift;
+                mask |= 0xFFu << shift;
+                acc_c = sm.b_i[1];
+                eq = sm.b_i[2];
+                acc_m = sm.b_d[0];
+                __syncthreads();
+            }
+            // `eq` kept elements share the threshold key and the same mass e_P: take the
+            // fewest of them (lowest indices) that bring the mass to the target
+            const double e_P = mass(prefix);
+            long long r = (long long)ceil((target - acc_m) / e_P);
+            if (r < 1) r = 1;
+            if (r > eq) r = eq;
+            while (r > 1 && acc_m + (double)(r - 1) * e_P >= target) --r;
+            while (r < eq && acc_m + (double)r * e_P < target) ++r;
+            const int n_new = acc_c + (int)r;
+            if (n_new != n_kept) {
+                const bool same_ranked = (prefix == p.T && p.eq_mode == 2);
+                if ((int)r < eq) {
+                    p.eq_mode = 2;
+                    p.need = (int)r;
+                } else if (prefix != p.T) {
+                    p.eq_mode = 1;
+                }
+                p.T = prefix;
+                n_kept = n_new;
+                if (p.eq_mode == 2 && !same_ranked) tie_prepass(p.T);
+                sum_pass(p);
+                scan_exclusive(sm.chunk_sum, nchunks);
+            }
+        }
+
+        // ---- 5/6. locate the chunk, then the element
+        const double Z = sm.chunk_sum[nchunks];
+        const double t = c * Z;
+        if (tid == 0) { sm.b_i[0] = INT_MAX; sm.b_i[1] = -1; }
+        __syncthreads();
+        for (int ci = tid; ci < nchunks; ci += NT) {
+            const double excl = sm.chunk_sum[ci], incl = sm.chunk_sum[ci + 1];
+            if (incl > excl) {
+                atomicMax(&sm.b_i[1], ci);
+                if (t < incl) atomicMin(&sm.b_i[0], ci);
+            }
+        }
+        __syncthreads();
+        const bool force_last = (sm.b_i[0] == INT_MAX);
+        const int cstar = force_last ? sm.b_i[1] : sm.b_i[0];
+
+        if (warp == 0) {
+            double run = sm.chunk_sum[cstar];
+            int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[cstar] : 0;
+            int last_idx = -1;
+            double last_S = 0.0, last_e = 1.0;
+            int tok = -1;
+            double tok_S = 0.0, tok_e = 1.0;
+            for (int r = 0; r < R && tok < 0; ++r) {
+                uint32_t k[E];
+                int base;
+                chunk_keys(cstar, r, k, base);
+                const int rank0 = lane_rank0(k, p, tie_run);
+                const unsigned bits = kept_bits(k, p, rank0);
+                double ev[E];
+                double local = 0.0;
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    ev[e] = (bits & (1u << e)) ? mass(k[e]) : 0.0;
+                    local += ev[e];
+                }
+                const double incl = warp_incl_scan_d(local, lane);
+                double excl = __shfl_up_sync(FULL, incl, 1);
+                if (lane == 0) excl = 0.0;
+                int pick = -1;
+                double pick_S = 0.0, pick_e = 1.0;
+                if (bits) {
+                    double S = run + excl;
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        if (bits & (1u << e)) {
+                            if (pick < 0 && t < S + ev[e]) { pick = base + e; pick_S = S; pick_e = ev[e]; }
+                            last_idx = base + e; last_S = S; last_e = ev[e];
+                            S += ev[e];
+                        }
+                    }
+                }
+                const bool cross = !force_last && bits && (t < run + incl);
+                const unsigned bal = __ballot_sync(FULL, cross);
+                if (bal) {
+                    const int L = __ffs(bal) - 1;
+                    if (pick < 0) { pick = last_idx; pick_S = last_S; pick_e = last_e; }
+                    tok = __shfl_sync(FULL, pick, L);
+                    tok_S = __shfl_sync(FULL, pick_S, L);
+                    tok_e = __shfl_sync(FULL, pick_e, L);
+                }
+                run += __shfl_sync(FULL, incl, 31);
+            }
+            if (tok < 0) {   // rounding at the top end: the last kept element of the chunk
+                const unsigned best = warp_max_u((unsigned)(last_idx + 1));
+                const unsigned bal = __ballot_sync(FULL, (unsigned)(last_idx + 1) == best);
+                const int L = __ffs(bal) - 1;
+                tok = __shfl_sync(FULL, last_idx, L);
+                tok_S = __shfl_sync(FULL, last_S, L);
+                tok_e = __shfl_sync(FULL, last_e, L);
+            }
+            if (lane == 0) {
+                double cn = (t - tok_S) / tok_e;
+                if (!(cn >= 0.0)) cn = 0.0;
+                if (cn > ASX_ONE_BELOW) cn = ASX_ONE_BELOW;
+                LaneResult r;
+                r.token = tok; r.status = tok < 0 ? ST_NUMERIC : ST_OK; r.n_kept = n_kept;
+                r.code_out = tok < 0 ? c_in : cn;
+                r.p_tok = tok_e / Z;
+                r.cdf_lo = tok_S / Z;
+                sm.res = r;
+            }
+        }
+        __syncthreads();
+        const LaneResult out = sm.res;
+        __syncthreads();
+        return out;
+    }
+};
+
+}  // namespace asx

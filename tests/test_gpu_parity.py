@@ -1,0 +1,356 @@
+"""CUDA path vs CPU oracle, element by element, through the C-ABI binding (needs a B200)."""
+import numpy as np
+import pytest
+
+from tests.parity import compare_step
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+F32, BF16 = 0, 1
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2210_15458_b200 import binding
+    binding.lib()
+    return binding
+
+
+def to_dev(arr, dtype):
+    if dtype == BF16:
+        return torch.from_numpy(np.ascontiguousarray(arr).view(np.int16)).cuda().view(torch.bfloat16)
+    return torch.from_numpy(np.ascontiguousarray(arr)).cuda()
+
+
+def gpu_step(B, arr, dtype, codes, temp, top_k, top_p, V=None):
+    d = {}
+    tok, c2 = B.as_step(to_dev(arr, dtype), torch.from_numpy(codes).cuda(), temp, top_k, top_p, diag=d, V=V)
+    torch.cuda.synchronize()
+    return (tok.cpu().numpy(), c2.cpu().numpy(), d["p_tok"].cpu().numpy(), d["n_kept"].cpu().numpy(),
+            d["lane_status"].cpu().numpy())
+
+
+def check(B, orc, arr, dtype, codes, temp, top_k, top_p, V=None, what="", threads=8):
+    ref = orc.step(arr, dtype, codes, temp, top_k, top_p, V=V, threads=threads)
+    tok, c2, p, nk, st = gpu_step(B, arr, dtype, codes, temp, top_k, top_p, V=V)
+    return compare_step(ref, tok, c2, p, nk, st, what=what)
+
+
+MODS = [(1.0, 0, 1.0), (0.7, 5, 1.0), (1.3, 0, 0.9), (0.8, 7, 0.6), (0.5, 1, 1.0), (1.0, 0, 1e-6),
+        (2.0, 1000000, 0.999)]
+
+
+def _store(x, dtype):
+    from paper_2210_15458_b200 import synth
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    return synth.f32_to_bf16_bits(x) if dtype == BF16 else x
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+@pytest.mark.parametrize("V", [1, 2, 3, 5, 17, 33, 255, 1000, 4099, 9001])
+def test_step_small_shapes_all_modifiers(B, orc, dtype, V):
+    rng = np.random.default_rng(1000 + V)
+    lanes = 37
+    arr = _store(rng.normal(0, 3, (lanes, V)), dtype)
+    codes = rng.random(lanes)
+    codes[0] = 0.0
+    codes[1] = 1.0
+    codes[2] = 1.0 - 2.0 ** -53
+    for temp, k, p in MODS:
+        check(B, orc, arr, dtype, codes, temp, k, p, what="V=%d dt=%d mods=%s" % (V, dtype, (temp, k, p)))
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_step_heavy_ties(B, orc, dtype):
+    # integer-valued logits: most elements tie at every threshold, so top-k and the nucleus
+    # both cut inside groups of equal values (lowest indices win)
+    rng = np.random.default_rng(77)
+    for V in (64, 700, 5000):
+        arr = _store(rng.integers(-3, 4, (29, V)), dtype)
+        codes = rng.random(29)
+        for temp, k, p in [(1.0, 10, 1.0), (0.9, 0, 0.5), (1.1, V // 2, 0.7), (1.0, 3, 0.99), (1.0, V - 1, 1.0)]:
+            check(B, orc, arr, dtype, codes, temp, k, p, what="ties V=%d %s" % (V, (temp, k, p)))
+    flat = _store(np.zeros((8, 3000)), dtype)                 # one value only
+    check(B, orc, flat, dtype, rng.random(8), 1.0, 100, 0.5, what="flat row")
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_step_masked_and_nonfinite_lanes(B, orc, dtype):
+    rng = np.random.default_rng(5)
+    V = 777
+    x = rng.normal(0, 2, (10, V)).astype(np.float32)
+    x[0, ::2] = -np.inf
+    x[1, :] = -np.inf
+    x[1, 500] = 0.25                      # a single live token
+    x[2, 3] = np.nan
+    x[3, 700] = np.inf
+    x[4, :] = -np.inf                     # empty row
+    x[5, 10] = -np.nan
+    arr = _store(x, dtype)
+    codes = rng.random(10)
+    codes[6] = 1.5
+    codes[7] = np.nan
+    codes[8] = -0.1
+    for temp, k, p in [(1.0, 0, 1.0), (0.7, 4, 0.9)]:
+        r = check(B, orc, arr, dtype, codes, temp, k, p, what="nonfinite")
+    ref = orc.step(arr, dtype, codes)
+    assert (ref.status[[2, 3, 4, 5, 6, 7, 8]] == orc.ERR_NUMERIC).all() and ref.status[[0, 1, 9]].tolist() == [0, 0, 0]
+    tok, c2, *_ = gpu_step(B, arr, dtype, codes, 1.0, 0, 1.0)
+    assert tok[1] == 500 and c2[6] == 1.5                      # code returned unchanged on failure
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_step_padded_and_unaligned_rows(B, orc, dtype):
+    # ld > V, odd pitches (rows not 16-byte aligned) and a view that starts off-alignment
+    rng = np.random.default_rng(9)
+    for V, ld in [(1000, 1001), (1000, 1024), (33, 37), (4099, 4101)]:
+        full = _store(rng.normal(0, 3, (21, ld)), dtype)
+        codes = rng.random(21)
+        check(B, orc, full, dtype, codes, 0.9, 6, 0.95, V=V, what="ld=%d" % ld)
+    big = _store(rng.normal(0, 3, (12, 2051)), dtype)
+    dev = to_dev(big, dtype)[:, 3:2003]                        # offset view, pitch 2051
+    ref = orc.step(np.ascontiguousarray(big[:, 3:2003]), dtype, rng.random(12) * 0 + 0.37, 1.0, 9, 1.0)
+    tok, c2 = B.as_step(dev, torch.full((12,), 0.37, dtype=torch.float64, device="cuda"), 1.0, 9, 1.0)
+    compare_step(ref, tok.cpu().numpy(), c2.cpu().numpy(), what="offset view")
+
+
+def test_step_in_place_and_deterministic(B, orc):
+    from paper_2210_15458_b200 import synth
+    w = synth.c2()
+    arr = w.logits(64)
+    dev = to_dev(arr, BF16)
+    codes = torch.from_numpy(orc.lattice_codes(64, 0.3)).cuda()
+    t1, c1 = B.as_step(dev, codes, w.temp, w.top_k, w.top_p)
+    t2, c2 = B.as_step(dev, codes, w.temp, w.top_k, w.top_p)
+    assert torch.equal(t1, t2) and torch.equal(c1, c2)
+    alias = codes.clone()
+    t3, c3 = B.as_step(dev, alias, w.temp, w.top_k, w.top_p, codes_out=alias)
+    assert torch.equal(t1, t3) and torch.equal(c1, alias)
+    assert B.as_step(dev[:0], codes[:0], 1.0)[0].numel() == 0   # zero lanes is a no-op
+
+
+def test_lattice_codes_bit_exact(B, orc):
+    for N, u in [(1, 0.0), (7, 0.5), (256, 0.999999999), (1024, 1.0 - 2.0 ** -53), (100003, 0.123456789)]:
+        got = B.as_lattice_codes(N, u).cpu().numpy()
+        np.testing.assert_array_equal(got, orc.lattice_codes(N, u))
+    with pytest.raises(B.AsError):
+        B.as_lattice_codes(8, 1.0)
+
+
+# --------------------------------------------------------------------------- the measured configurations
+def test_c2_full(B, orc):
+    from paper_2210_15458_b200 import synth
+    w = synth.c2()
+    arr = w.logits()
+    codes = orc.lattice_codes(w.N, w.shift())
+    r = check(B, orc, arr, BF16, codes, w.temp, w.top_k, w.top_p, what="c2")
+    assert r["compared"] > 0.95 * w.lanes
+    iid = synth.iid_codes(w.lanes, 123)                      # ordinary ancestral sampling, same path
+    check(B, orc, arr, BF16, iid, w.temp, w.top_k, w.top_p, what="c2 iid")
+
+
+def _sampled_full_size(B, orc, w, sample, seed):
+    arr = w.logits()
+    codes = orc.lattice_codes(w.N, w.shift())[: w.lanes]
+    tok, c2, p, nk, st = gpu_step(B, arr, w.dtype, codes, w.temp, w.top_k, w.top_p)
+    idx = np.sort(np.random.default_rng(seed).choice(w.lanes, sample, replace=False))
+    ref = orc.step(np.ascontiguousarray(arr[idx]), w.dtype, codes[idx], w.temp, w.top_k, w.top_p, threads=8)
+    r = compare_step(ref, tok[idx], c2[idx], p[idx], nk[idx], st[idx], what=w.name)
+    assert (st == 0).all() and (tok >= 0).all() and (tok < w.V).all()
+    assert (c2 >= 0).all() and (c2 < 1).all() and (nk >= 1).all()
+    if w.top_k:
+        assert (nk <= w.top_k).all()
+    return r
+
+
+def test_c3_full_size_sampled(B, orc):
+    from paper_2210_15458_b200 import synth
+    r = _sampled_full_size(B, orc, synth.c3(), 64, 1)
+    assert r["compared"] >= 56
+
+
+def test_c5_full_size_sampled(B, orc):
+    from paper_2210_15458_b200 import synth
+    r = _sampled_full_size(B, orc, synth.c5(1024), 48, 2)
+    assert r["compared"] >= 40
+
+
+# --------------------------------------------------------------------------- bigram decode loop
+def _teacher_forced(B, orc, table, dtype, dev_table, prev, codes, T, eos, temp, top_k, top_p):
+    """Oracle decodes freely and records each step's input state; the GPU then takes every
+    recorded (previous token, code) as a one-step decode and must reproduce that step."""
+    ref = orc.decode_bigram_codes(table, dtype, prev, codes, T, eos, temp, top_k, top_p, trace=True, threads=8)
+    lanes = len(prev)
+    ts = [(i, t) for i in range(lanes) for t in range(ref.len[i])]
+    p_in = np.array([prev[i] if t == 0 else ref.seq[i, t - 1] for i, t in ts], np.int32)
+    c_in = np.array([ref.trace_code_in[i, t] for i, t in ts])
+    seq, ln = B.as_decode_bigram_codes(dev_table, torch.from_numpy(p_in).cuda(), torch.from_numpy(c_in).cuda(),
+                                       1, eos, temp, top_k, top_p,
+                                       codes_final=(cf := torch.empty(len(ts), dtype=torch.float64, device="cuda")))
+    torch.cuda.synchronize()
+    want_tok = np.array([ref.seq[i, t] for i, t in ts])
+    want_c = np.array([ref.trace_code_out[i, t] for i, t in ts])
+    d_tok = np.array([ref.trace_d_tok[i, t] for i, t in ts])
+    safe = d_tok > 1e-5
+    got = seq.cpu().numpy()[:, 0]
+    assert (ln.cpu().numpy() == 1).all()
+    assert (got[safe] == want_tok[safe]).all()
+    np.testing.assert_allclose(cf.cpu().numpy()[safe], want_c[safe], rtol=1e-6, atol=1e-12)
+    return ref, int(safe.sum()), len(ts)
+
+
+def _comparable_prefix(ref, i):
+    """Number of leading steps of lane i on which a free-running decode must still equal the
+    oracle's: before the first step inside the boundary band, and while the rounding error of
+    the code (~1e-16, multiplied by 1/p at every step) is still far below that band."""
+    n = int(ref.len[i])
+    amp = 1e-15
+    for t in range(n):
+        if not (ref.trace_d_tok[i, t] > 1e-5) or amp > 1e-8:
+            return t
+        amp /= ref.trace_p_tok[i, t]
+    return n
+
+
+def test_c1_decode(B, orc):
+    from paper_2210_15458_b200 import synth
+    w = synth.c1()
+    table = w.table()
+    dev = to_dev(table, F32)
+    starts = w.starts()
+    u = w.shift()
+    st = torch.empty(w.lanes, dtype=torch.int32, device="cuda")
+    cf = torch.empty(w.lanes, dtype=torch.float64, device="cuda")
+    seq, ln = B.as_decode_bigram(dev, torch.from_numpy(starts).cuda(), w.N, u, w.T, w.eos, w.temp,
+                                 codes_final=cf, lane_status=st)
+    torch.cuda.synchronize()
+    prev = np.repeat(starts, w.N).astype(np.int32)
+    codes = np.tile(orc.lattice_codes(w.N, u), w.S)
+    ref, nsafe, nsteps = _teacher_forced(B, orc, table, F32, dev, prev, codes, w.T, w.eos, w.temp, 0, 1.0)
+    assert nsafe > 0.98 * nsteps
+    seq, ln = seq.cpu().numpy(), ln.cpu().numpy()
+    assert (st.cpu().numpy() == 0).all()
+    # free-running sequences agree up to the first step that sits in the boundary band
+    compared = 0
+    for i in range(w.lanes):
+        upto = _comparable_prefix(ref, i)
+        assert (seq[i, :upto] == ref.seq[i, :upto]).all()
+        compared += upto
+        assert (seq[i, ln[i]:] == -1).all() and (seq[i, :ln[i]] >= 0).all()
+        if ln[i] < w.T:
+            assert seq[i, ln[i] - 1] == w.eos
+    assert compared >= 3 * w.lanes
+    # split and resume: 16 steps == 8 + 8 from the returned state
+    a_cf = torch.empty(w.lanes, dtype=torch.float64, device="cuda")
+    a_seq, a_len = B.as_decode_bigram_codes(dev, torch.from_numpy(prev).cuda(), torch.from_numpy(codes).cuda(),
+                                            8, w.eos, w.temp, codes_final=a_cf)
+    alive = (a_len == 8) & (a_seq[:, 7] != w.eos)
+    idx = torch.nonzero(alive)[:, 0]
+    b_seq, b_len = B.as_decode_bigram_codes(dev, a_seq[idx, 7].contiguous(), a_cf[idx].contiguous(), 8, w.eos, w.temp)
+    torch.cuda.synchronize()
+    assert (b_seq.cpu().numpy() == seq[idx.cpu().numpy(), 8:]).all()
+
+
+def test_decode_small_models_with_cuts_and_eos(B, orc):
+    rng = np.random.default_rng(31)
+    for dtype, V, eos, temp, k, p in [(F32, 50, 3, 1.0, 0, 1.0), (BF16, 300, 0, 0.8, 10, 1.0),
+                                      (F32, 1000, 7, 1.2, 0, 0.8), (BF16, 2000, -1, 0.7, 20, 0.9)]:
+        x = rng.normal(0, 2, (V, V)).astype(np.float32)
+        if eos >= 0:
+            x[:, eos] += 3.0                              # frequent EOS -> ragged lengths
+        table = _store(x, dtype)
+        dev = to_dev(table, dtype)
+        prev = rng.integers(0, V, 96).astype(np.int32)
+        codes = rng.random(96)
+        ref, nsafe, nsteps = _teacher_forced(B, orc, table, dtype, dev, prev, codes, 12, eos, temp, k, p)
+        assert nsafe > 0.9 * nsteps
+        seq, ln = B.as_decode_bigram_codes(dev, torch.from_numpy(prev).cuda(), torch.from_numpy(codes).cuda(),
+                                           12, eos, temp, k, p)
+        seq, ln = seq.cpu().numpy(), ln.cpu().numpy()
+        compared = 0
+        for i in range(96):
+            upto = _comparable_prefix(ref, i)
+            assert (seq[i, :upto] == ref.seq[i, :upto]).all()
+            if upto == ref.len[i]:
+                assert ln[i] == ref.len[i] and (seq[i, upto:] == -1).all()
+            compared += upto
+        assert compared >= 96
+    # T = 0 and an out-of-range start token
+    seq, ln = B.as_decode_bigram_codes(dev, torch.tensor([1], dtype=torch.int32, device="cuda"),
+                                       torch.tensor([0.5], dtype=torch.float64, device="cuda"), 0, -1)
+    assert ln.cpu().item() == 0
+    st = torch.empty(2, dtype=torch.int32, device="cuda")
+    seq, ln = B.as_decode_bigram_codes(dev, torch.tensor([1, V + 5], dtype=torch.int32, device="cuda"),
+                                       torch.tensor([0.5, 0.5], dtype=torch.float64, device="cuda"), 3, -1,
+                                       lane_status=st)
+    assert st.cpu().tolist() == [0, B.ERR_NUMERIC] and ln.cpu().tolist() == [3, 0]
+    assert (seq[1].cpu().numpy() == -1).all()
+
+
+def test_decode_lattice_properties_on_gpu_output(B, orc):
+    # Sec. 4.3 on the GPU's own output: sorted codes give dictionary-ordered sequences, and a
+    # first token of probability P is produced by floor(NP) or ceil(NP) lanes of a group.
+    from paper_2210_15458_b200 import synth
+    w = synth.c1()
+    table = w.table()
+    starts = w.starts()
+    u = w.shift()
+    seq, ln = B.as_decode_bigram(to_dev(table, F32), torch.from_numpy(starts).cuda(), w.N, u, w.T, w.eos, w.temp)
+    seq = seq.cpu().numpy()
+    for s in range(w.S):
+        grp = [tuple(r) for r in seq[s * w.N:(s + 1) * w.N]]
+        # codes of a group increase with j except for the wrap; after rotating, order is kept
+        codes = orc.lattice_codes(w.N, u)
+        order = np.argsort(codes, kind="stable")
+        keyed = [tuple(np.where(np.array(grp[j]) < 0, 10 ** 6, np.array(grp[j]))) for j in order]
+        # padded (-1) positions sort after every token except EOS itself, which ends the sequence
+        firsts = [g[0] for g in keyed]
+        assert firsts == sorted(firsts)
+        row = table[starts[s]].astype(np.float64)
+        pr = np.exp(row - row.max())
+        pr /= pr.sum()
+        cnt = np.bincount([g[0] for g in grp], minlength=w.V)
+        assert (cnt >= np.floor(w.N * pr - 1e-9)).all() and (cnt <= np.ceil(w.N * pr + 1e-9)).all()
+
+
+def test_c4_shape_reduced_table(B, orc):
+    # c4's recipe (bf16 table, Zipf-like column bias, temperature 0.8, EOS id 1) on a 4096-token
+    # vocabulary so that the whole loop runs in seconds; the full 32128 x 32128 table is
+    # covered by test_c4_full_size_sampled.
+    from paper_2210_15458_b200 import synth
+    w = synth.c4(V=4096, S=16, T=48)
+    table = w.table()
+    dev = to_dev(table, BF16)
+    prev = np.repeat(w.starts(), w.N).astype(np.int32)
+    codes = np.tile(orc.lattice_codes(w.N, w.shift()), w.S)
+    ref, nsafe, nsteps = _teacher_forced(B, orc, table, BF16, dev, prev, codes, w.T, w.eos, w.temp, 0, 1.0)
+    assert nsafe > 0.97 * nsteps
+
+
+def test_c4_full_size_sampled(B, orc):
+    from paper_2210_15458_b200 import synth
+    w = synth.c4()
+    table = w.table()
+    dev = to_dev(table, BF16)
+    starts = w.starts()
+    u = w.shift()
+    st = torch.empty(w.lanes, dtype=torch.int32, device="cuda")
+    seq, ln = B.as_decode_bigram(dev, torch.from_numpy(starts).cuda(), w.N, u, w.T, w.eos, w.temp, lane_status=st)
+    torch.cuda.synchronize()
+    seq, ln = seq.cpu().numpy(), ln.cpu().numpy()
+    assert (st.cpu().numpy() == 0).all() and (seq[np.arange(w.lanes), 0] >= 0).all()
+    assert (seq < w.V).all()
+    lanes = np.sort(np.random.default_rng(4).choice(w.lanes, 24, replace=False))
+    prev = np.repeat(starts, w.N).astype(np.int32)[lanes]
+    codes = np.tile(orc.lattice_codes(w.N, u), w.S)[lanes]
+    ref, nsafe, nsteps = _teacher_forced(B, orc, table, BF16, dev, prev, codes, 24, w.eos, w.temp, 0, 1.0)
+    assert nsafe > 0.97 * nsteps
+    compared = 0
+    for n, i in enumerate(lanes):
+        upto = _comparable_prefix(ref, n)
+        assert (seq[i, :upto] == ref.seq[n, :upto]).all()
+        compared += upto
+    assert compared >= 5 * len(lanes)
