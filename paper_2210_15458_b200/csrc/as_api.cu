@@ -142,14 +142,18 @@ decode_generic_kernel(const void* __restrict__ table, int V, long long ld,
 // ---------------------------------------------------------------------------
 // argument checks
 // ---------------------------------------------------------------------------
-static int check_common(const void* data, int dtype, int V, long long ld, double temp, double top_p) {
-    if (!data) return set_err(AS_ERR_INVALID_ARG, "logits/table pointer is NULL");
+static int check_scalars(int dtype, int V, long long ld, double temp, double top_p) {
     if (dtype != AS_F32 && dtype != AS_BF16) return set_err(AS_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     if (V < 1) return set_err(AS_ERR_INVALID_ARG, "V = %d must be >= 1", V);
     if (V > AS_MAX_V) return set_err(AS_ERR_UNSUPPORTED, "V = %d exceeds AS_MAX_V = %d", V, AS_MAX_V);
     if (ld < V) return set_err(AS_ERR_INVALID_ARG, "ld = %lld is smaller than V = %d", ld, V);
     if (!(temp > 0.0) || std::isinf(temp)) return set_err(AS_ERR_INVALID_ARG, "temp must be positive and finite");
     if (std::isnan(top_p)) return set_err(AS_ERR_INVALID_ARG, "top_p is NaN");
+    return AS_OK;
+}
+
+static int check_data(const void* data, int dtype) {
+    if (!data) return set_err(AS_ERR_INVALID_ARG, "logits/table pointer is NULL");
     const uintptr_t a = reinterpret_cast<uintptr_t>(data);
     if (a % (dtype == AS_F32 ? 4 : 2)) return set_err(AS_ERR_INVALID_ARG, "logits/table pointer is not element-aligned");
     return AS_OK;
@@ -207,10 +211,11 @@ int as_step(const void* d_logits, int dtype, int lanes, int V, long long ld, con
             double temp, int top_k, double top_p, int32_t* d_tokens, double* d_codes_out,
             const as_step_diag* diag, void* stream) {
     if (lanes < 0) return set_err(AS_ERR_INVALID_ARG, "lanes = %d must be >= 0", lanes);
-    int rc = check_common(d_logits, dtype, V, ld, temp, top_p);
+    int rc = check_scalars(dtype, V, ld, temp, top_p);
     if (rc != AS_OK) return rc;
-    if (!d_codes || !d_tokens || !d_codes_out) return set_err(AS_ERR_INVALID_ARG, "codes / tokens / codes_out pointer is NULL");
     if (lanes == 0) return AS_OK;
+    if ((rc = check_data(d_logits, dtype)) != AS_OK) return rc;
+    if (!d_codes || !d_tokens || !d_codes_out) return set_err(AS_ERR_INVALID_ARG, "codes / tokens / codes_out pointer is NULL");
     const DeviceInfo* di;
     rc = device_info(&di);
     if (rc != AS_OK) return rc;
@@ -243,10 +248,11 @@ int as_step_host(const void* h_logits, int dtype, int lanes, int V, long long ld
                  double temp, int top_k, double top_p, int32_t* h_tokens, double* h_codes_out,
                  int32_t* h_lane_status, void* d_work, size_t work_bytes, void* stream) {
     if (lanes < 0) return set_err(AS_ERR_INVALID_ARG, "lanes = %d must be >= 0", lanes);
-    int rc = check_common(h_logits, dtype, V, ld, temp, top_p);
+    int rc = check_scalars(dtype, V, ld, temp, top_p);
     if (rc != AS_OK) return rc;
-    if (!h_codes || !h_tokens || !h_codes_out) return set_err(AS_ERR_INVALID_ARG, "host codes / tokens / codes_out pointer is NULL");
     if (lanes == 0) return AS_OK;
+    if ((rc = check_data(h_logits, dtype)) != AS_OK) return rc;
+    if (!h_codes || !h_tokens || !h_codes_out) return set_err(AS_ERR_INVALID_ARG, "host codes / tokens / codes_out pointer is NULL");
     if (!d_work || (reinterpret_cast<uintptr_t>(d_work) & 255)) return set_err(AS_ERR_INVALID_ARG, "d_work must be a 256-byte aligned device pointer");
     if (work_bytes < as_step_host_work_bytes(dtype, lanes, ld)) return set_err(AS_ERR_INVALID_ARG, "work_bytes is smaller than as_step_host_work_bytes()");
     const size_t esz = dtype == AS_F32 ? 4 : 2;
@@ -277,12 +283,13 @@ static int decode_common(const void* d_table, int dtype, int V, long long ld, co
                          const double* d_codes_in, int lanes, int N, double u, int T, int eos,
                          double temp, int top_k, double top_p, int32_t* d_seq, int32_t* d_len,
                          double* d_codes_final, int32_t* d_lane_status, void* stream) {
-    int rc = check_common(d_table, dtype, V, ld, temp, top_p);
+    int rc = check_scalars(dtype, V, ld, temp, top_p);
     if (rc != AS_OK) return rc;
     if (T < 0) return set_err(AS_ERR_INVALID_ARG, "T = %d must be >= 0", T);
+    if (lanes == 0) return AS_OK;
+    if ((rc = check_data(d_table, dtype)) != AS_OK) return rc;
     if (!d_tok) return set_err(AS_ERR_INVALID_ARG, "start / prev token pointer is NULL");
     if (!d_len || (!d_seq && T > 0)) return set_err(AS_ERR_INVALID_ARG, "seq / len pointer is NULL");
-    if (lanes == 0) return AS_OK;
     const DeviceInfo* di;
     rc = device_info(&di);
     if (rc != AS_OK) return rc;

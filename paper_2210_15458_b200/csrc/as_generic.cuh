@@ -113,7 +113,7 @@ struct GenericLane {
         return exp_nonpos(((double)Tr::value_f(key) - lmax) * inv_tau, sm.exp_tbl);
     }
 
-    // exclusive scan of a[0..n) in place by warp 0; a[n] receives the total
+    // exclusive scan of a[0..n), n >= 1, in place by warp 0; a[n] receives the total
     template <typename T>
     __device__ void scan_exclusive(T* a, int n) {
         if (warp == 0) {
@@ -134,7 +134,9 @@ struct GenericLane {
                 a[i] = run;
                 run += v;
             }
-            if (lane == 31) a[n] = incl;
+            // the total continues the same running sum as the prefixes, so that
+            // a[i+1] > a[i] exactly when element i added something
+            if (e == n && b < n) a[n] = run;
         }
         __syncthreads();
     }
