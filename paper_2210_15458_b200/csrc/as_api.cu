@@ -1,6 +1,6 @@
 // C-ABI entry points (see include/arith_sampling.h) and the kernels behind them.
 #include "../../include/arith_sampling.h"
-#include "as_generic.cuh"
+#include "as_staged.cuh"
 
 #include <cmath>
 #include <cstdarg>
@@ -49,12 +49,70 @@ static int device_info(const DeviceInfo** out) {
     return AS_OK;
 }
 
-struct DiagPtrs {
-    double* p_tok;
-    double* cdf_lo;
-    int* n_kept;
-    int* lane_status;
-};
+using DiagPtrs = DiagOut;
+
+// ---------------------------------------------------------------------------
+// staged step kernel: launch shape
+// ---------------------------------------------------------------------------
+constexpr size_t SMEM_OPTIN_MAX = 232448;   // 227 KB per CTA on sm_100
+
+static size_t staged_fixed_bytes() { return (sizeof(StagedSmem<ST_NT>) + 127) & ~(size_t)127; }
+
+template <int DT, int CS>
+static int launch_staged(const StepArgs& a, size_t smem, int sms, int want_per_sm, cudaStream_t st) {
+    static size_t attr_set[64] = {0};
+    static int max_clusters[64] = {0};
+    static size_t max_clusters_smem[64] = {0};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    auto kern = step_staged_kernel<DT, CS>;
+    cudaError_t e;
+    if (attr_set[dev] < smem) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_OPTIN_MAX - 1024));
+        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(max dynamic shared memory)");
+        attr_set[dev] = SMEM_OPTIN_MAX;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(ST_NT);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (max_clusters_smem[dev] != smem) {       // resident clusters for this shape (cached)
+        cfg.gridDim = dim3(CS * sms);
+        int n = 0;
+        e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaOccupancyMaxActiveClusters");
+        if (n < 1) return set_err(AS_ERR_CUDA, "staged kernel does not fit (cluster %d, %zu bytes shared)", CS, smem);
+        max_clusters[dev] = n;
+        max_clusters_smem[dev] = smem;
+    }
+    int nclusters = max_clusters[dev];
+    if (want_per_sm > 0) {
+        const long long cap = (long long)want_per_sm * sms / CS;
+        if (cap >= 1 && cap < nclusters) nclusters = (int)cap;
+    }
+    if (nclusters > a.lanes) nclusters = a.lanes;
+    cfg.gridDim = dim3(nclusters * CS);
+    e = cudaLaunchKernelEx(&cfg, kern, a);
+    if (e != cudaSuccess) return cuda_fail(e, "staged step kernel launch");
+    return AS_OK;
+}
+
+template <int DT>
+static int launch_staged_cs(int cs, const StepArgs& a, size_t smem, int sms, int per_sm, cudaStream_t st) {
+    switch (cs) {
+        case 1: return launch_staged<DT, 1>(a, smem, sms, per_sm, st);
+        case 2: return launch_staged<DT, 2>(a, smem, sms, per_sm, st);
+        case 4: return launch_staged<DT, 4>(a, smem, sms, per_sm, st);
+        default: return launch_staged<DT, 8>(a, smem, sms, per_sm, st);
+    }
+}
 
 // ---------------------------------------------------------------------------
 // kernels
@@ -224,8 +282,26 @@ int as_step(const void* d_logits, int dtype, int lanes, int V, long long ld, con
     if (top_k < 0 || top_k >= V) top_k = 0;
     if (!(top_p > 0.0 && top_p < 1.0)) top_p = 1.0;
     const double inv_tau = 1.0 / temp;
-    const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
     cudaStream_t st = (cudaStream_t)stream;
+    // staged path: the row (or a 1/CS slice of it per CTA of a cluster) must fit in shared memory
+    const int E = dtype == AS_F32 ? 4 : 8;
+    const size_t row_bytes = (size_t)((V + E - 1) / E) * 16;
+    int cs = g_tune_cluster;
+    if (cs == 0) cs = row_bytes <= 80 * 1024 ? 1 : row_bytes <= 160 * 1024 ? 2 : row_bytes <= 320 * 1024 ? 4 : 8;
+    const size_t slice_bytes = (((row_bytes / 16) + cs - 1) / cs) * 16;
+    const size_t smem = staged_fixed_bytes() + slice_bytes + 16;
+    const bool staged = g_tune_path != 1 && smem <= SMEM_OPTIN_MAX - 1024 &&
+                        slice_bytes <= (size_t)ST_MAXCHUNK * ST_CHUNK_BYTES;
+    if (staged) {
+        StepArgs a;
+        a.logits = d_logits; a.codes = d_codes; a.tokens = d_tokens; a.codes_out = d_codes_out; a.diag = dp;
+        a.ld = ld; a.inv_tau = inv_tau; a.top_p = top_p; a.scale2 = (float)(1.4426950408889634 / temp);
+        a.lanes = lanes; a.V = V; a.top_k = top_k;
+        a.fast = (top_k > 0 && top_k <= 300) || (top_k == 0 && top_p < 1.0);
+        return dtype == AS_F32 ? launch_staged_cs<DT_F32>(cs, a, smem, di->sms, g_tune_ctas, st)
+                               : launch_staged_cs<DT_BF16>(cs, a, smem, di->sms, g_tune_ctas, st);
+    }
+    const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
     if (dtype == AS_F32)
         step_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, inv_tau, top_k, top_p, d_tokens, d_codes_out, dp);
     else

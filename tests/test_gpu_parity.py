@@ -354,3 +354,49 @@ def test_c4_full_size_sampled(B, orc):
         assert (seq[i, :upto] == ref.seq[n, :upto]).all()
         compared += upto
     assert compared >= 5 * len(lanes)
+
+
+# --------------------------------------------------------------------------- launch shapes
+@pytest.mark.parametrize("cluster", [1, 2, 4, 8])
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_step_every_cluster_size(B, orc, dtype, cluster):
+    # the same lanes through 1, 2, 4 and 8 CTAs per lane (row slices in distributed shared
+    # memory), with ragged tails, ties, and more lanes than resident clusters
+    rng = np.random.default_rng(500 + cluster)
+    try:
+        B.as_tune(B.TUNE_CLUSTER, cluster)
+        for V, lanes in [(9001, 45), (40000, 300), (777, 20), (65536 + 24, 33)]:
+            x = rng.normal(0, 3, (lanes, V)).astype(np.float32)
+            x[:, : V // 3] = np.round(x[:, : V // 3])           # a third of the row is tie-prone
+            arr = _store(x, dtype)
+            codes = rng.random(lanes)
+            for temp, k, p in [(0.7, 40, 1.0), (1.0, 0, 0.9), (0.8, 64, 0.95), (1.0, 0, 1.0), (1.0, 290, 0.5)]:
+                check(B, orc, arr, dtype, codes, temp, k, p, what="cluster=%d V=%d %s" % (cluster, V, (temp, k, p)))
+    finally:
+        B.as_tune(B.TUNE_CLUSTER, 0)
+
+
+def test_step_general_path_only(B, orc):
+    from paper_2210_15458_b200 import synth
+    w = synth.c2()
+    arr = w.logits(96)
+    codes = orc.lattice_codes(96, 0.77)
+    try:
+        B.as_tune(B.TUNE_STEP_PATH, 1)
+        check(B, orc, arr, BF16, codes, w.temp, w.top_k, 0.9, what="general path")
+    finally:
+        B.as_tune(B.TUNE_STEP_PATH, 0)
+
+
+def test_step_flat_and_adversarial_rows_fall_back(B, orc):
+    # rows the compaction cannot serve: everything ties with the maximum, a nucleus that needs
+    # most of the vocabulary, top-k larger than the candidate capacity
+    rng = np.random.default_rng(600)
+    V = 20000
+    flat = _store(np.zeros((6, V)), BF16)
+    check(B, orc, flat, BF16, rng.random(6), 1.0, 40, 1.0, what="flat top-k")
+    check(B, orc, flat, BF16, rng.random(6), 1.0, 0, 0.9, what="flat nucleus")
+    wide = _store(rng.normal(0, 0.05, (6, V)), F32)
+    check(B, orc, wide, F32, rng.random(6), 1.0, 0, 0.97, what="wide nucleus")
+    check(B, orc, wide, F32, rng.random(6), 1.0, 5000, 1.0, what="large top-k")
+    check(B, orc, wide, F32, rng.random(6), 1.0, 5000, 0.3, what="large top-k + nucleus")
