@@ -71,12 +71,18 @@ extern "C" {
  *   d_cdf_lo      [lanes] f64  F_{i-1}, the lower end of the chosen token's interval
  *   d_n_kept      [lanes] i32  number of tokens with non-zero probability after the cuts
  *   d_lane_status [lanes] i32  AS_OK or AS_ERR_NUMERIC / AS_ERR_TIMEOUT
+ *   d_path        [lanes] i32  which routine decided the lane: AS_PATH_COMPACT (candidate
+ *                              compaction from shared memory) or AS_PATH_GENERAL (full-row
+ *                              fp64 routine; slower, serves every input)
  */
+#define AS_PATH_COMPACT 0
+#define AS_PATH_GENERAL 1
 typedef struct as_step_diag {
     double *d_p_tok;
     double *d_cdf_lo;
     int32_t *d_n_kept;
     int32_t *d_lane_status;
+    int32_t *d_path;
 } as_step_diag;
 
 /*
@@ -175,14 +181,18 @@ int as_decode_bigram_codes(const void *d_table, int dtype, int V, long long ld,
 /*
  * Launch-shape overrides for measurement sweeps (process-wide, not thread-safe;
  * 0 restores the built-in choice).  Keys:
- *   AS_TUNE_STEP_PATH     1 = general path only, 2 = staged path wherever it applies
- *   AS_TUNE_CLUSTER       CTAs per lane for the staged path (1, 2, 4, 8)
+ *   AS_TUNE_STEP_PATH     0 = streaming kernel (one CTA per lane), 1 = general kernel only,
+ *                         2 = cluster kernel (row split over the CTAs of a cluster)
+ *   AS_TUNE_CLUSTER       CTAs per lane for the cluster kernel (1, 2, 4, 8)
  *   AS_TUNE_CTAS_PER_SM   resident CTAs per SM the grid is sized for
+ *   AS_TUNE_STAGES        16 KB ring stages of the streaming kernel for rows that do not
+ *                         fit the ring (2..12)
  * Returns AS_ERR_INVALID_ARG for an unknown key or value.
  */
 #define AS_TUNE_STEP_PATH 1
 #define AS_TUNE_CLUSTER 2
 #define AS_TUNE_CTAS_PER_SM 3
+#define AS_TUNE_STAGES 4
 int as_tune(int key, int value);
 
 /* Text of the calling thread's most recent error ("" if none). Never NULL. */

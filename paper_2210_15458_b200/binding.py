@@ -25,9 +25,13 @@ ERR_CUDA = -3
 ERR_TIMEOUT = -4
 ERR_NUMERIC = -5
 
+PATH_COMPACT = 0
+PATH_GENERAL = 1
+
 TUNE_STEP_PATH = 1
 TUNE_CLUSTER = 2
 TUNE_CTAS_PER_SM = 3
+TUNE_STAGES = 4
 
 EXPORTS = ["as_lattice_codes", "as_step", "as_step_host", "as_step_host_work_bytes", "as_decode_bigram",
            "as_decode_bigram_codes", "as_tune", "as_last_error", "as_version"]
@@ -41,7 +45,8 @@ class AsError(RuntimeError):
 
 class as_step_diag(ctypes.Structure):
     _fields_ = [("d_p_tok", ctypes.c_void_p), ("d_cdf_lo", ctypes.c_void_p),
-                ("d_n_kept", ctypes.c_void_p), ("d_lane_status", ctypes.c_void_p)]
+                ("d_n_kept", ctypes.c_void_p), ("d_lane_status", ctypes.c_void_p),
+                ("d_path", ctypes.c_void_p)]
 
 
 _lib = None
@@ -126,7 +131,7 @@ def as_step(logits: torch.Tensor, codes: torch.Tensor, temp: float = 1.0, top_k:
             codes_out: Optional[torch.Tensor] = None, diag: Optional[dict] = None, V: Optional[int] = None,
             stream=None):
     """tokens, codes' = one decode step.  `diag`, if a dict, receives the tensors p_tok,
-    cdf_lo, n_kept, lane_status (allocated here unless already present)."""
+    cdf_lo, n_kept, lane_status, path (allocated here unless already present)."""
     lanes, width, ld = _logits_layout(logits)
     V = width if V is None else V
     dev = logits.device
@@ -142,8 +147,9 @@ def as_step(logits: torch.Tensor, codes: torch.Tensor, temp: float = 1.0, top_k:
         diag.setdefault("cdf_lo", torch.empty(lanes, dtype=torch.float64, device=dev))
         diag.setdefault("n_kept", torch.empty(lanes, dtype=torch.int32, device=dev))
         diag.setdefault("lane_status", torch.empty(lanes, dtype=torch.int32, device=dev))
+        diag.setdefault("path", torch.empty(lanes, dtype=torch.int32, device=dev))
         dg = as_step_diag(_ptr(diag["p_tok"]), _ptr(diag["cdf_lo"]), _ptr(diag["n_kept"]),
-                          _ptr(diag["lane_status"]))
+                          _ptr(diag["lane_status"]), _ptr(diag["path"]))
     _check(lib().as_step(_ptr(logits), _logits_dtype(logits), lanes, V, ld, _ptr(codes), temp, top_k, top_p,
                          _ptr(tokens), _ptr(codes_out), ctypes.byref(dg) if dg is not None else None,
                          _stream(stream)))

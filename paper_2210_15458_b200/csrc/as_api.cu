@@ -1,6 +1,6 @@
 // C-ABI entry points (see include/arith_sampling.h) and the kernels behind them.
 #include "../../include/arith_sampling.h"
-#include "as_staged.cuh"
+#include "as_stream.cuh"
 
 #include <cmath>
 #include <cstdarg>
@@ -13,7 +13,7 @@ namespace asx {
 // host-side state
 // ---------------------------------------------------------------------------
 static thread_local char g_err[512] = "";
-static int g_tune_path = 0, g_tune_cluster = 0, g_tune_ctas = 0;
+static int g_tune_path = 0, g_tune_cluster = 0, g_tune_ctas = 0, g_tune_stages = 0;
 
 static int set_err(int code, const char* fmt, ...) {
     va_list ap;
@@ -104,6 +104,39 @@ static int launch_staged(const StepArgs& a, size_t smem, int sms, int want_per_s
     return AS_OK;
 }
 
+static size_t stream_fixed_bytes() { return (sizeof(StreamSmem) + 127) & ~(size_t)127; }
+
+template <int DT>
+static int launch_stream(const StepArgs& a, int stages, int sms, int want_per_sm, cudaStream_t st) {
+    static bool attr_set[64] = {false};
+    static int per_sm_cache[64][SK_MAXSTAGES + 1] = {{0}};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    auto kern = step_stream_kernel<DT>;
+    cudaError_t e;
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_OPTIN_MAX - 1024));
+        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(max dynamic shared memory)");
+        attr_set[dev] = true;
+    }
+    const size_t smem = stream_fixed_bytes() + (size_t)stages * SK_STAGE_BYTES;
+    if (per_sm_cache[dev][stages] == 0) {
+        int n = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, SK_THREADS, smem);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaOccupancyMaxActiveBlocksPerMultiprocessor");
+        if (n < 1) return set_err(AS_ERR_CUDA, "streaming kernel does not fit (%zu bytes shared)", smem);
+        per_sm_cache[dev][stages] = n;
+    }
+    int per_sm = per_sm_cache[dev][stages];
+    if (want_per_sm > 0 && want_per_sm < per_sm) per_sm = want_per_sm;
+    long long grid = (long long)per_sm * sms;
+    if (grid > a.lanes) grid = a.lanes;
+    kern<<<(unsigned)grid, SK_THREADS, smem, st>>>(a, stages);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "streaming step kernel launch");
+    return AS_OK;
+}
+
 template <int DT>
 static int launch_staged_cs(int cs, const StepArgs& a, size_t smem, int sms, int per_sm, cudaStream_t st) {
     switch (cs) {
@@ -148,6 +181,7 @@ step_generic_kernel(const void* __restrict__ logits, int lanes, int V, long long
             if (diag.cdf_lo) diag.cdf_lo[ln] = r.cdf_lo;
             if (diag.n_kept) diag.n_kept[ln] = r.n_kept;
             if (diag.lane_status) diag.lane_status[ln] = r.status;
+            if (diag.path) diag.path[ln] = PATH_GENERAL;
         }
     }
 }
@@ -230,6 +264,13 @@ extern "C" {
 
 int as_version(void) { return 1000; }
 
+#ifdef ASX_PROFILE
+// profiling builds only: copies CTA 0's phase timestamps of the last staged launch
+int as_debug_marks(long long* h_out) {
+    return cudaMemcpyFromSymbol(h_out, g_asx_marks, sizeof(long long) * 32) == cudaSuccess ? AS_OK : AS_ERR_CUDA;
+}
+#endif
+
 const char* as_last_error(void) { return g_err; }
 
 int as_tune(int key, int value) {
@@ -246,6 +287,10 @@ int as_tune(int key, int value) {
         case AS_TUNE_CTAS_PER_SM:
             if (value < 0 || value > 32) return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_CTAS_PER_SM takes 0..32");
             g_tune_ctas = value;
+            return AS_OK;
+        case AS_TUNE_STAGES:
+            if (value < 0 || value == 1 || value > SK_MAXSTAGES) return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_STAGES takes 0 or 2..12");
+            g_tune_stages = value;
             return AS_OK;
         default:
             return set_err(AS_ERR_INVALID_ARG, "unknown tuning key %d", key);
@@ -277,29 +322,41 @@ int as_step(const void* d_logits, int dtype, int lanes, int V, long long ld, con
     const DeviceInfo* di;
     rc = device_info(&di);
     if (rc != AS_OK) return rc;
-    DiagPtrs dp = {nullptr, nullptr, nullptr, nullptr};
-    if (diag) dp = {diag->d_p_tok, diag->d_cdf_lo, diag->d_n_kept, diag->d_lane_status};
+    DiagPtrs dp = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    if (diag) dp = {diag->d_p_tok, diag->d_cdf_lo, diag->d_n_kept, diag->d_lane_status, diag->d_path};
     if (top_k < 0 || top_k >= V) top_k = 0;
     if (!(top_p > 0.0 && top_p < 1.0)) top_p = 1.0;
     const double inv_tau = 1.0 / temp;
     cudaStream_t st = (cudaStream_t)stream;
-    // staged path: the row (or a 1/CS slice of it per CTA of a cluster) must fit in shared memory
+    StepArgs a;
+    a.logits = d_logits; a.codes = d_codes; a.tokens = d_tokens; a.codes_out = d_codes_out; a.diag = dp;
+    a.ld = ld; a.inv_tau = inv_tau; a.top_p = top_p; a.scale2 = (float)(1.4426950408889634 / temp);
+    a.lanes = lanes; a.V = V; a.top_k = top_k;
     const int E = dtype == AS_F32 ? 4 : 8;
     const size_t row_bytes = (size_t)((V + E - 1) / E) * 16;
-    int cs = g_tune_cluster;
-    if (cs == 0) cs = row_bytes <= 80 * 1024 ? 1 : row_bytes <= 160 * 1024 ? 2 : row_bytes <= 320 * 1024 ? 4 : 8;
-    const size_t slice_bytes = (((row_bytes / 16) + cs - 1) / cs) * 16;
-    const size_t smem = staged_fixed_bytes() + slice_bytes + 16;
-    const bool staged = g_tune_path != 1 && smem <= SMEM_OPTIN_MAX - 1024 &&
-                        slice_bytes <= (size_t)ST_MAXCHUNK * ST_CHUNK_BYTES;
-    if (staged) {
-        StepArgs a;
-        a.logits = d_logits; a.codes = d_codes; a.tokens = d_tokens; a.codes_out = d_codes_out; a.diag = dp;
-        a.ld = ld; a.inv_tau = inv_tau; a.top_p = top_p; a.scale2 = (float)(1.4426950408889634 / temp);
-        a.lanes = lanes; a.V = V; a.top_k = top_k;
-        a.fast = (top_k > 0 && top_k <= 300) || (top_k == 0 && top_p < 1.0);
-        return dtype == AS_F32 ? launch_staged_cs<DT_F32>(cs, a, smem, di->sms, g_tune_ctas, st)
-                               : launch_staged_cs<DT_BF16>(cs, a, smem, di->sms, g_tune_ctas, st);
+    if (g_tune_path == 0) {
+        // streaming kernel: one CTA per lane; rows of up to 6 stages (96 KB) stay resident in the ring
+        const int nsl = (int)((row_bytes + SK_STAGE_BYTES - 1) / SK_STAGE_BYTES);
+        const bool resident = nsl <= 6;
+        a.fast = (top_k > 0 && top_k <= SK_K0_MAX) || (top_k == 0 && top_p < 1.0);
+        if (resident || a.fast) {
+            int stages = resident ? (nsl < 1 ? 1 : nsl) : (g_tune_stages > 0 ? g_tune_stages : 3);
+            if (!resident && stages >= nsl) stages = nsl - 1;
+            return dtype == AS_F32 ? launch_stream<DT_F32>(a, stages, di->sms, g_tune_ctas, st)
+                                   : launch_stream<DT_BF16>(a, stages, di->sms, g_tune_ctas, st);
+        }
+    }
+    if (g_tune_path == 2) {
+        // cluster kernel: the row split over CS CTAs' shared memory
+        int cs = g_tune_cluster;
+        if (cs == 0) cs = row_bytes <= 80 * 1024 ? 1 : row_bytes <= 160 * 1024 ? 2 : row_bytes <= 320 * 1024 ? 4 : 8;
+        const size_t slice_bytes = (((row_bytes / 16) + cs - 1) / cs) * 16;
+        const size_t smem = staged_fixed_bytes() + slice_bytes + 16;
+        if (smem <= SMEM_OPTIN_MAX - 1024 && slice_bytes <= (size_t)ST_MAXCHUNK * ST_CHUNK_BYTES) {
+            a.fast = (top_k > 0 && top_k <= 300) || (top_k == 0 && top_p < 1.0);
+            return dtype == AS_F32 ? launch_staged_cs<DT_F32>(cs, a, smem, di->sms, g_tune_ctas, st)
+                                   : launch_staged_cs<DT_BF16>(cs, a, smem, di->sms, g_tune_ctas, st);
+        }
     }
     const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
     if (dtype == AS_F32)
@@ -345,7 +402,7 @@ int as_step_host(const void* h_logits, int dtype, int lanes, int V, long long ld
     const size_t ncopy = ((size_t)(lanes - 1) * (size_t)ld + (size_t)V) * esz;
     if ((e = cudaMemcpyAsync(d_logits, h_logits, ncopy, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "copy logits to device");
     if ((e = cudaMemcpyAsync(d_codes, h_codes, (size_t)lanes * 8, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "copy codes to device");
-    as_step_diag dg = {nullptr, nullptr, nullptr, d_status};
+    as_step_diag dg = {nullptr, nullptr, nullptr, d_status, nullptr};
     rc = as_step(d_logits, dtype, lanes, V, ld, d_codes, temp, top_k, top_p, d_tokens, d_codes_out, &dg, stream);
     if (rc != AS_OK) return rc;
     if ((e = cudaMemcpyAsync(h_tokens, d_tokens, (size_t)lanes * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "copy tokens to host");

@@ -47,7 +47,19 @@ struct GenericSmem {
     LaneResult res;
 };
 
-template <int DT, int NT>
+// Barrier over the NT threads that run a lane: the whole CTA, or (in kernels with a
+// separate copy-issuing warp) the consumer warps only, through named barrier 1.
+struct SyncAll {
+    __device__ __forceinline__ static void sync() { __syncthreads(); }
+};
+template <int NTHREADS>
+struct SyncNamed {
+    __device__ __forceinline__ static void sync() {
+        asm volatile("bar.sync 1, %0;" ::"n"(NTHREADS) : "memory");
+    }
+};
+
+template <int DT, int NT, class Sync = SyncAll>
 struct GenericLane {
     using Tr = Traits<DT>;
     static constexpr int E = Tr::E;
@@ -138,7 +150,7 @@ struct GenericLane {
             // a[i+1] > a[i] exactly when element i added something
             if (e == n && b < n) a[n] = run;
         }
-        __syncthreads();
+        Sync::sync();
     }
 
     // chunk_eq[ci] <- number of elements equal to T in chunks before ci
@@ -155,7 +167,7 @@ struct GenericLane {
             cnt = warp_sum_i(cnt);
             if (lane == 0) sm.chunk_eq[ci] = cnt;
         }
-        __syncthreads();
+        Sync::sync();
         scan_exclusive(sm.chunk_eq, nchunks);
     }
 
@@ -177,7 +189,7 @@ struct GenericLane {
             local = warp_sum_d(local);
             if (lane == 0) sm.chunk_sum[ci] = local;
         }
-        __syncthreads();
+        Sync::sync();
     }
 
     // histogram of digit (key >> shift) & 255 over kept elements whose key matches
@@ -188,7 +200,7 @@ struct GenericLane {
             sm.hist_cnt[i] = 0;
             sm.hist_mass[i] = 0.0;
         }
-        __syncthreads();
+        Sync::sync();
         for (int ci = warp; ci < nchunks; ci += NW) {
             int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[ci] : 0;
             for (int r = 0; r < R; ++r) {
@@ -207,7 +219,7 @@ struct GenericLane {
                 }
             }
         }
-        __syncthreads();
+        Sync::sync();
     }
 
     // Largest non-empty digit d with (acc + weight of digits >= d) >= target; if none
@@ -272,7 +284,7 @@ struct GenericLane {
                 sm.b_d[0] = acc_mass + best_above_m;
             }
         }
-        __syncthreads();
+        Sync::sync();
     }
 
     __device__ LaneResult fail(double c_in, int status) {
@@ -305,14 +317,14 @@ struct GenericLane {
         kmin = warp_min_u(kmin);
         nfin = warp_sum_i(nfin);
         if (lane == 0) { sm.red_u[warp] = kmax; sm.red_u2[warp] = kmin; sm.red_i[warp] = nfin; }
-        __syncthreads();
+        Sync::sync();
         kmax = 0; kmin = 0xFFFFFFFFu; nfin = 0;
         for (int w = 0; w < NW; ++w) {
             kmax = max(kmax, sm.red_u[w]);
             kmin = min(kmin, sm.red_u2[w]);
             nfin += sm.red_i[w];
         }
-        __syncthreads();
+        Sync::sync();
         if (code_bad || kmin < Tr::KEY_NINF || kmax >= Tr::KEY_PINF || kmax == Tr::KEY_NINF)
             return fail(c_in, ST_NUMERIC);
         lmax = (double)Tr::value_f(kmax);
@@ -332,7 +344,7 @@ struct GenericLane {
                 mask |= 0xFFu << shift;
                 acc = sm.b_i[1];
                 eq = sm.b_i[2];
-                __syncthreads();
+                Sync::sync();
             }
             p.T = prefix;
             p.need = top_k - acc;
@@ -348,7 +360,7 @@ struct GenericLane {
         // ---- 4. nucleus on the distribution renormalised over the survivors
         if (top_p > 0.0 && top_p < 1.0) {
             const double target = top_p * sm.chunk_sum[nchunks];
-            __syncthreads();
+            Sync::sync();
             uint32_t prefix = 0, mask = 0;
             int acc_c = 0, eq = 0;
             double acc_m = 0.0;
@@ -360,7 +372,7 @@ struct GenericLane {
                 acc_c = sm.b_i[1];
                 eq = sm.b_i[2];
                 acc_m = sm.b_d[0];
-                __syncthreads();
+                Sync::sync();
             }
             // `eq` kept elements share the threshold key and the same mass e_P: take the
             // fewest of them (lowest indices) that bring the mass to the target
@@ -391,7 +403,7 @@ struct GenericLane {
         const double Z = sm.chunk_sum[nchunks];
         const double t = c * Z;
         if (tid == 0) { sm.b_i[0] = INT_MAX; sm.b_i[1] = -1; }
-        __syncthreads();
+        Sync::sync();
         for (int ci = tid; ci < nchunks; ci += NT) {
             const double excl = sm.chunk_sum[ci], incl = sm.chunk_sum[ci + 1];
             if (incl > excl) {
@@ -399,7 +411,7 @@ struct GenericLane {
                 if (t < incl) atomicMin(&sm.b_i[0], ci);
             }
         }
-        __syncthreads();
+        Sync::sync();
         const bool force_last = (sm.b_i[0] == INT_MAX);
         const int cstar = force_last ? sm.b_i[1] : sm.b_i[0];
 
@@ -470,9 +482,9 @@ struct GenericLane {
                 sm.res = r;
             }
         }
-        __syncthreads();
+        Sync::sync();
         const LaneResult out = sm.res;
-        __syncthreads();
+        Sync::sync();
         return out;
     }
 };

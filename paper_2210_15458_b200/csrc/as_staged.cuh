@@ -40,12 +40,23 @@ constexpr int ST_M = 2 * ST_NT;        // subset maxima per CTA
 constexpr int ST_KP = 256;             // candidates aimed at for nucleus-only lanes
 constexpr long long ST_WAIT_CYCLES = 4000000000LL;   // ~2 s: bound on any mbarrier wait
 
+// Phase timestamps of CTA 0 for profiling builds (-DASX_PROFILE); compiled out otherwise.
+#ifdef ASX_PROFILE
+__device__ long long g_asx_marks[32];
+#define ASX_MARK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_asx_marks[i] = clock64(); } while (0)
+#else
+#define ASX_MARK(i) do {} while (0)
+#endif
+
 struct DiagOut {
     double* p_tok;
     double* cdf_lo;
     int* n_kept;
     int* lane_status;
+    int* path;
 };
+constexpr int PATH_COMPACT = 0;
+constexpr int PATH_GENERAL = 1;
 
 struct StepArgs {
     const void* logits;
@@ -196,7 +207,8 @@ template <> struct Pass<DT_F32> {
     __device__ static uint32_t key_of_f(float x) { return Traits<DT_F32>::key_of(__float_as_uint(x)); }
 };
 
-__device__ __forceinline__ void write_result(const StepArgs& a, int ln, const LaneResult& r) {
+__device__ __forceinline__ void write_result(const StepArgs& a, int ln, const LaneResult& r, int path) {
+    if (a.diag.path) a.diag.path[ln] = path;
     a.tokens[ln] = r.token;
     a.codes_out[ln] = r.code_out;
     if (a.diag.p_tok) a.diag.p_tok[ln] = r.p_tok;
@@ -270,12 +282,14 @@ __device__ bool epilogue(StagedSmem<NT>& sm, int C, double c, double c_in, doubl
         ep.order[r] = (unsigned short)i;
     }
     __syncthreads();
+    ASX_MARK(8);
     const int kmax = (top_k > 0 && top_k < C) ? top_k : C;
     for (int r = tid; r < kmax; r += NT) {
         const uint32_t key = (uint32_t)(sm.cand[ep.order[r]] >> 32);
         ep.e[r] = exp_nonpos(((double)Tr::value_f(key) - lmax) * inv_tau, sm.exp_tbl);
     }
     __syncthreads();
+    ASX_MARK(9);
     // nucleus on the distribution renormalised over the survivors: prefix masses in rank order
     if (warp == 0) {
         const int per = (kmax + 31) / 32;
@@ -304,6 +318,7 @@ __device__ bool epilogue(StagedSmem<NT>& sm, int C, double c, double c_in, doubl
         if (lane == 0) { sm.b_i[0] = n_final; sm.b_i[1] = ok; }
     }
     __syncthreads();
+    ASX_MARK(10);
     const int n_final = sm.b_i[0];
     if (!sm.b_i[1]) return false;
     // index order among the kept
@@ -315,6 +330,7 @@ __device__ bool epilogue(StagedSmem<NT>& sm, int C, double c, double c_in, doubl
         ep.tok_idx[ir] = (int)idx;
     }
     __syncthreads();
+    ASX_MARK(11);
     if (warp == 0) {
         const int per = (n_final + 31) / 32;
         const int b = min(lane * per, n_final), e = min(b + per, n_final);
@@ -445,13 +461,14 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
             if (is_leader) {
                 GenericLane<DT, NT> g(sm.u.gen, row_of(ln), V, false);
                 const LaneResult r = g.run(c_in, a.inv_tau, a.top_k, a.top_p);
-                if (tid == 0) write_result(a, ln, r);
+                if (tid == 0) write_result(a, ln, r, PATH_GENERAL);
             }
             if (nxt < a.lanes && staged_ok(nxt)) issue(nxt);
             continue;
         }
 
         // ---------------- pass 1: max, as the copies land
+        ASX_MARK(0);
         typename P::Acc acc = P::init();
         bool timed_out = poisoned;
         for (int i = 0; i < nchunk; ++i) {
@@ -460,6 +477,7 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
             if (v < bulk_vec) P::fold(acc, rowv[v]);
         }
         ++phase;
+        ASX_MARK(1);
         if (tail_elems > 0 && tid == 0) P::fold(acc, rowv[bulk_vec]);
         uint32_t k0, k1;
         P::keys(acc, k0, k1);
@@ -473,12 +491,14 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
         cmax = 0;
         for (int w = 0; w < NT / 32; ++w) cmax = max(cmax, sm.red_u[w]);
         const bool cut = a.fast && (a.top_k > 0 || a.top_p < 1.0);
+        ASX_MARK(2);
         uint32_t t0key = Tr::KEY_NINF;
         if (cut) {
             const int K0 = a.top_k > 0 ? a.top_k : ST_KP;
             const int K0r = (K0 + CS - 1) / CS;
             if (K0r <= ST_M) t0key = P::key_from16(select_kth16<DT, NT>(sm, K0r));
         }
+        ASX_MARK(3);
         int flag = sm.b_i[3];
         __syncthreads();
         if (tid == 0) sm.b_i[3] = 0;
@@ -503,12 +523,13 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
         }
         if (flag || code_bad || gmax >= Tr::KEY_PINF || gmax <= Tr::KEY_NINF) {
             // timeout, bad code, NaN / +inf (NaN-propagating max), or nothing but -inf
-            if (is_leader && tid == 0) write_result(a, ln, failed_lane(c_in, flag ? ST_TIMEOUT : ST_NUMERIC));
+            if (is_leader && tid == 0) write_result(a, ln, failed_lane(c_in, flag ? ST_TIMEOUT : ST_NUMERIC), PATH_COMPACT);
             if (CS > 1) cluster.sync();          // peers are done with this row's exchange slots
             else __syncthreads();
             if (nxt < a.lanes && staged_ok(nxt)) issue(nxt);
             continue;
         }
+        ASX_MARK(4);
         const double lmax = (double)Tr::value_f(gmax);
         gt0 = max(gt0, Tr::KEY_NINF);            // a bound below every finite key means "all of them"
 
@@ -517,13 +538,13 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
             if (CS == 1) {
                 GenericLane<DT, NT> g(sm.u.gen, rowbuf, V, true);
                 const LaneResult r = g.run(c_in, a.inv_tau, a.top_k, a.top_p);
-                if (tid == 0) write_result(a, ln, r);
+                if (tid == 0) write_result(a, ln, r, PATH_GENERAL);
             } else {
                 cluster.sync();
                 if (is_leader) {
                     GenericLane<DT, NT> g(sm.u.gen, row_of(ln), V, true);
                     const LaneResult r = g.run(c_in, a.inv_tau, a.top_k, a.top_p);
-                    if (tid == 0) write_result(a, ln, r);
+                    if (tid == 0) write_result(a, ln, r, PATH_GENERAL);
                 }
             }
             if (nxt < a.lanes && staged_ok(nxt)) issue(nxt);
@@ -572,6 +593,7 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
                 }
             }
         }
+        ASX_MARK(5);
         if (want_tail) {
             double td = warp_sum_d((double)tail);
             if (lane == 0) sm.red_d[warp] = td;
@@ -586,7 +608,9 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
         else __syncthreads();
 
         // ---------------- next lane's copies overlap the epilogue
+        ASX_MARK(6);
         if (nxt < a.lanes && staged_ok(nxt)) issue(nxt);
+        ASX_MARK(7);
 
         // ---------------- epilogue on the leader
         if (is_leader) {
@@ -602,9 +626,10 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
                 GenericLane<DT, NT> g(sm.u.gen, row_of(ln), V, true);
                 r = g.run(c_in, a.inv_tau, a.top_k, a.top_p);
             }
-            if (tid == 0) write_result(a, ln, r);
+            if (tid == 0) write_result(a, ln, r, done ? PATH_COMPACT : PATH_GENERAL);
             __syncthreads();
         }
+        ASX_MARK(12);
     }
     if (poisoned && tid == 0) {
         // copies issued before the wait ran out may still be in flight: give them one more bounded wait

@@ -364,6 +364,7 @@ def test_step_every_cluster_size(B, orc, dtype, cluster):
     # memory), with ragged tails, ties, and more lanes than resident clusters
     rng = np.random.default_rng(500 + cluster)
     try:
+        B.as_tune(B.TUNE_STEP_PATH, 2)
         B.as_tune(B.TUNE_CLUSTER, cluster)
         for V, lanes in [(9001, 45), (40000, 300), (777, 20), (65536 + 24, 33)]:
             x = rng.normal(0, 3, (lanes, V)).astype(np.float32)
@@ -374,6 +375,27 @@ def test_step_every_cluster_size(B, orc, dtype, cluster):
                 check(B, orc, arr, dtype, codes, temp, k, p, what="cluster=%d V=%d %s" % (cluster, V, (temp, k, p)))
     finally:
         B.as_tune(B.TUNE_CLUSTER, 0)
+        B.as_tune(B.TUNE_STEP_PATH, 0)
+
+
+@pytest.mark.parametrize("stages", [2, 3, 5])
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_step_streamed_rows(B, orc, dtype, stages):
+    # rows longer than the shared-memory ring: slices stream through 2, 3 or 5 stages, the
+    # threshold is refreshed at slices 0, 1, 2, 4, ..., ragged last slice and ragged last vector
+    rng = np.random.default_rng(700 + stages)
+    try:
+        B.as_tune(B.TUNE_STAGES, stages)
+        for V, lanes in [(70001, 40), (131072, 12), (200003, 9)]:
+            x = rng.normal(0, 3, (lanes, V)).astype(np.float32)
+            x[:, ::3] = np.round(x[:, ::3])
+            x[: lanes // 2] += np.linspace(0, 6, V, dtype=np.float32)[None, :]   # the best tokens come last
+            arr = _store(x, dtype)
+            codes = rng.random(lanes)
+            for temp, k, p in [(0.7, 40, 1.0), (1.0, 0, 0.9), (0.8, 64, 0.95), (1.0, 128, 0.5), (1.0, 1, 1.0)]:
+                check(B, orc, arr, dtype, codes, temp, k, p, what="stages=%d V=%d %s" % (stages, V, (temp, k, p)))
+    finally:
+        B.as_tune(B.TUNE_STAGES, 0)
 
 
 def test_step_general_path_only(B, orc):
