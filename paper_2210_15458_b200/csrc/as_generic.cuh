@@ -293,7 +293,7 @@ struct GenericLane {
         return r;
     }
 
-    __device__ LaneResult run(double c_in, double inv_tau_, int top_k, double top_p) {
+    __device__ __noinline__ LaneResult run(double c_in, double inv_tau_, int top_k, double top_p) {
         inv_tau = inv_tau_;
         fill_exp_table(sm.exp_tbl, tid);
         double c = c_in;

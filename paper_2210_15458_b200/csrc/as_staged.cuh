@@ -164,6 +164,15 @@ template <> struct Pass<DT_BF16> {
     __device__ static void fold(Acc& a, const uint4& q) {
         a.m = max_nan_bf16x2(a.m, max_nan_bf16x2(max_nan_bf16x2(q.x, q.y), max_nan_bf16x2(q.z, q.w)));
     }
+    // NaN-propagating max of one vector, kept packed; merged into the running max and
+    // reused for the "any element >= threshold" test
+    __device__ static Acc reduce(const uint4& q) {
+        return Acc{max_nan_bf16x2(max_nan_bf16x2(q.x, q.y), max_nan_bf16x2(q.z, q.w))};
+    }
+    __device__ static void merge(Acc& a, const Acc& b) { a.m = max_nan_bf16x2(a.m, b.m); }
+    __device__ static float part_max(const Acc& b) {
+        return fmaxf(__uint_as_float(b.m << 16), __uint_as_float(b.m & 0xFFFF0000u));
+    }
     __device__ static void keys(const Acc& a, uint32_t& k0, uint32_t& k1) {
         k0 = Traits<DT_BF16>::key_of(a.m & 0xFFFFu);
         k1 = Traits<DT_BF16>::key_of(a.m >> 16);
@@ -190,6 +199,12 @@ template <> struct Pass<DT_F32> {
         s.a = max_nan_f32(s.a, max_nan_f32(__uint_as_float(q.x), __uint_as_float(q.z)));
         s.b = max_nan_f32(s.b, max_nan_f32(__uint_as_float(q.y), __uint_as_float(q.w)));
     }
+    __device__ static Acc reduce(const uint4& q) {
+        return Acc{max_nan_f32(__uint_as_float(q.x), __uint_as_float(q.z)),
+                   max_nan_f32(__uint_as_float(q.y), __uint_as_float(q.w))};
+    }
+    __device__ static void merge(Acc& s, const Acc& b) { s.a = max_nan_f32(s.a, b.a); s.b = max_nan_f32(s.b, b.b); }
+    __device__ static float part_max(const Acc& b) { return fmaxf(b.a, b.b); }
     __device__ static void keys(const Acc& s, uint32_t& k0, uint32_t& k1) {
         k0 = Traits<DT_F32>::key_of(__float_as_uint(s.a));
         k1 = Traits<DT_F32>::key_of(__float_as_uint(s.b));

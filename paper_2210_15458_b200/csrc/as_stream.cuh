@@ -8,22 +8,25 @@
 // wait for compute.  Consumers see each row exactly once (Algorithm 1 needs every
 // conditional probability once):
 //   resident rows (row <= ring): all stages land, one NaN-propagating max pass,
-//       one threshold T0, one compaction pass from shared memory;
+//       one threshold T0, one hit pass from shared memory;
 //   streamed rows (row > ring): each 16 KB slice goes shared memory -> registers,
 //       the stage is released at once, the slice is folded into the running
-//       max and compacted against the current T0; T0 is recomputed at slices
+//       max and tested against the current T0; T0 is recomputed at slices
 //       0, 1, 2, 4, 8, ... and only ever rises.
 // T0 is a lower bound on the K0-th largest logit: each warp takes the m-th
-// largest (m = ceil(K0 / 8)) of its 64 per-thread subset maxima by a 16-step
-// ballot search, and T0 is the smallest of the 8 warp values, so at least K0
-// elements are >= T0.  Every element >= T0 is appended to a candidate list.
-// The epilogue is exact and fp64 on that list only: bitonic sort by (value desc,
-// index asc), top-k, masses, nucleus prefix, sort by index, CDF prefix,
-// crossing, rescale (Algorithm 1: w_i, (m, M), c <- (c - m)/(M - m)).
-// For nucleus-only lanes the masses of non-candidates are summed in fp32 (they
-// only enter the nucleus target top_p * Z1).  Lanes the list cannot decide
-// (too many candidates, nucleus deeper than the list, unaligned rows) go to
-// GenericLane, which reads the row from global memory (L2).
+// largest (m = ceil(K0 / 8)) of its 64 per-thread subset maxima by a ballot
+// search, and T0 is the smallest of the 8 warp values, so at least K0 elements
+// are >= T0.  The hot loop costs one packed max and one compare per 16-byte
+// vector; a vector holding an element >= T0 is copied (warp-aggregated, one
+// atomic per warp) to a small list.  Once per row the listed vectors are
+// searched for elements >= the FINAL T0, which also discards what earlier,
+// lower thresholds let in.  The epilogue is exact and fp64 on those candidates
+// only: rank by (value desc, index asc), top-k, masses, nucleus prefix, index
+// order, CDF prefix, crossing, rescale (Algorithm 1: w_i, (m, M),
+// c <- (c - m)/(M - m)).  For nucleus-only lanes the masses of everything else
+// are summed in fp32 (they only enter the nucleus target top_p * Z1).  Lanes the
+// list cannot decide (too many hits, nucleus deeper than the exact depth,
+// unaligned rows) go to GenericLane, which reads the row from global memory (L2).
 #pragma once
 #include "as_staged.cuh"
 
@@ -32,12 +35,14 @@ namespace asx {
 constexpr int SK_NT = 256;                 // consumer threads
 constexpr int SK_NW = SK_NT / 32;          // consumer warps
 constexpr int SK_THREADS = SK_NT + 32;     // + producer warp
-constexpr int SK_CAP = 1024;               // candidate capacity per lane
+constexpr int SK_CAPV = 1024;              // hit-vector capacity per lane
+constexpr int SK_CAP = 512;                // candidate (element) capacity per lane
 constexpr int SK_STAGE_VEC = 1024;         // 16-byte vectors per stage (16 KB)
 constexpr int SK_STAGE_BYTES = SK_STAGE_VEC * 16;
 constexpr int SK_VPT = SK_STAGE_VEC / SK_NT;   // vectors per consumer thread per slice
 constexpr int SK_MAXSTAGES = 12;
-constexpr int SK_K0_MAX = 128;             // largest top_k served by the candidate list
+constexpr int SK_K0_RESIDENT = 256;        // largest top_k served by the list, resident rows
+constexpr int SK_K0_STREAMED = 96;         // ... streamed rows (hits grow like K0 ln(V / K0))
 constexpr int SK_KP = 96;                  // K0 for nucleus-only lanes
 
 using SyncC = SyncNamed<SK_NT>;
@@ -47,16 +52,23 @@ struct StreamSmem {
     unsigned long long empty_bar[SK_MAXSTAGES];
     union {
         struct {
-            unsigned long long cand[SK_CAP];    // (key << 32) | ~index
-            unsigned long long isort[SK_CAP];   // (index << 32) | rank
-            double e[SK_CAP];                   // mass by rank
+            union {
+                uint4 cvec[SK_CAPV];                       // hit vectors (dead once extracted)
+                struct {
+                    unsigned long long srt[SK_CAP + 4];    // candidates by rank
+                    double e[SK_CAP];                      // mass by rank
+                } rk;
+            } v;
+            int cidx[SK_CAPV];                             // vector index of each hit vector
+            unsigned long long cand[SK_CAP + 4];           // (key << 32) | ~index, any order
         } ep;
         GenericSmem<SK_NT> gen;
     } u;
     double exp_tbl[64];
     double red_d[SK_NW];
-    unsigned wmax[SK_NW];
-    unsigned wsel[SK_NW];
+    unsigned wmax[2][SK_NW];
+    unsigned wsel[2][SK_NW];
+    int vec_count;
     int cand_count;
     int poisoned;        // a bounded wait ran out: stop issuing / stop waiting
     int b_i[4];
@@ -67,66 +79,57 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-// m-th largest (1-based) of the 64 16-bit keys held two per lane, by binary search on the
-// value: the largest v with count(keys >= v) >= m.
+// m-th largest (1-based) of the 64 16-bit keys held two per lane, by a search on the value, two
+// bits per step: the largest v with count(keys >= v) >= m (0 if fewer than m keys are positive).
 __device__ __forceinline__ uint32_t warp_select16(uint32_t a16, uint32_t b16, int m) {
     uint32_t res = 0;
-#pragma unroll
-    for (int bit = 15; bit >= 0; --bit) {
-        const uint32_t cand = res | (1u << bit);
-        const int cnt = __popc(__ballot_sync(FULL, a16 >= cand)) + __popc(__ballot_sync(FULL, b16 >= cand));
-        if (cnt >= m) res = cand;
+#pragma unroll 1
+    for (int bit = 14; bit >= 0; bit -= 2) {
+        const uint32_t c1 = res | (1u << bit), c2 = res | (2u << bit), c3 = res | (3u << bit);
+        const int n1 = __popc(__ballot_sync(FULL, a16 >= c1)) + __popc(__ballot_sync(FULL, b16 >= c1));
+        const int n2 = __popc(__ballot_sync(FULL, a16 >= c2)) + __popc(__ballot_sync(FULL, b16 >= c2));
+        const int n3 = __popc(__ballot_sync(FULL, a16 >= c3)) + __popc(__ballot_sync(FULL, b16 >= c3));
+        res = n3 >= m ? c3 : n2 >= m ? c2 : n1 >= m ? c1 : res;
     }
     return res;
 }
 
-// bitonic sort of a[0..P) (P a power of two) by NT threads; DESC: largest first
-template <int NT, class Sync, bool DESC>
-__device__ void bitonic_sort(unsigned long long* a, int P, int tid) {
-    for (int k = 2; k <= P; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = tid; i < P; i += NT) {
-                const int ixj = i ^ j;
-                if (ixj > i) {
-                    const unsigned long long x = a[i], y = a[ixj];
-                    const bool first_big = ((i & k) == 0) == DESC;   // this pair wants the larger first
-                    if ((x < y) == first_big) { a[i] = y; a[ixj] = x; }
-                }
-            }
-            Sync::sync();
-        }
-    }
-}
-
-// Exact decode on the candidate list.  t0_final: every element of the row with key >= t0_final is
-// in the list, so ranks are exact down to that key.  Returns false if the list cannot decide.
+// Exact decode on a candidate list src[0..C) (composites, any order); dst is scratch of C + 4
+// entries.  depth_key: every element of the row with key >= depth_key is in the list, so ranks
+// are exact down to that key.  Returns false if the list cannot decide the lane.
 template <int DT, int NT, class Sync>
-__device__ bool epilogue_sorted(StreamSmem& sm, int C, uint32_t t0_final, double c, double lmax,
-                                double inv_tau, int top_k, double top_p, double tail, LaneResult& out) {
+__device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long* src, unsigned long long* dst,
+                                             double* e, int C, uint32_t depth_key, double c, double lmax,
+                                             double inv_tau, int top_k, double top_p, double tail,
+                                             LaneResult& out) {
     using Tr = Traits<DT>;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    unsigned long long* cand = sm.u.ep.cand;
-    unsigned long long* isort = sm.u.ep.isort;
-    double* e = sm.u.ep.e;
-    int P = 32;
-    while (P < C) P <<= 1;
-    for (int i = C + tid; i < P; i += NT) cand[i] = 0ull;     // sorts after every real candidate
+    if (tid < 4) src[C + tid] = 0ull;             // padding for the 4-wide rank loop
     Sync::sync();
-    bitonic_sort<NT, Sync, true>(cand, P, tid);
+    // ---- ranks by (value desc, index asc): composites are distinct -> a permutation
+    for (int i = tid; i < C; i += NT) {
+        const unsigned long long ci = src[i];
+        int r = 0;
+#pragma unroll 1
+        for (int j = 0; j < C; j += 4)
+            r += (src[j] > ci) + (src[j + 1] > ci) + (src[j + 2] > ci) + (src[j + 3] > ci);
+        dst[r] = ci;
+    }
+    Sync::sync();
     const int kmax = (top_k > 0 && top_k < C) ? top_k : C;
     for (int r = tid; r < kmax; r += NT)
-        e[r] = exp_nonpos(((double)Tr::value_f((uint32_t)(cand[r] >> 32)) - lmax) * inv_tau, sm.exp_tbl);
+        e[r] = exp_nonpos(((double)Tr::value_f((uint32_t)(dst[r] >> 32)) - lmax) * inv_tau, sm.exp_tbl);
     Sync::sync();
     if (warp == 0) {
         // prefix masses in rank order: nucleus on the distribution renormalised over the survivors
-        const int per = (kmax + 31) / 32;
-        const int b = min(lane * per, kmax), en = min(b + per, kmax);
-        double s = 0.0;
-        for (int r = b; r < en; ++r) s += e[r];
-        const double incl = warp_incl_scan_d(s, lane);
-        const double total = __shfl_sync(FULL, incl, 31);
         int n_final = kmax, ok = 1;
         if (top_p < 1.0) {
+            const int per = (kmax + 31) / 32;
+            const int b = min(lane * per, kmax), en = min(b + per, kmax);
+            double s = 0.0;
+            for (int r = b; r < en; ++r) s += e[r];
+            const double incl = warp_incl_scan_d(s, lane);
+            const double total = __shfl_sync(FULL, incl, 31);
             const double target = top_p * (total + tail);
             double run = __shfl_up_sync(FULL, incl, 1);
             if (lane == 0) run = 0.0;
@@ -139,63 +142,76 @@ __device__ bool epilogue_sorted(StreamSmem& sm, int C, uint32_t t0_final, double
                 n_final = below + 1;
             }
         }
+        if (ok && (uint32_t)(dst[n_final - 1] >> 32) < depth_key) ok = 0;   // cut below the exact depth
         if (lane == 0) { sm.b_i[0] = n_final; sm.b_i[1] = ok; }
     }
     Sync::sync();
     const int n_final = sm.b_i[0];
-    if (!sm.b_i[1]) return false;
-    if ((uint32_t)(cand[n_final - 1] >> 32) < t0_final) return false;   // cut below the exact depth
-    int P2 = 32;
-    while (P2 < n_final) P2 <<= 1;
-    for (int i = tid; i < P2; i += NT)
-        isort[i] = i < n_final ? (((unsigned long long)(~(uint32_t)cand[i])) << 32) | (uint32_t)i : ~0ull;
-    Sync::sync();
-    bitonic_sort<NT, Sync, false>(isort, P2, tid);
-    if (warp == 0) {
-        const int per = (n_final + 31) / 32;
-        const int b = min(lane * per, n_final), en = min(b + per, n_final);
-        double s = 0.0;
-        for (int i = b; i < en; ++i) s += e[(uint32_t)isort[i]];
-        const double incl = warp_incl_scan_d(s, lane);
-        double run = __shfl_up_sync(FULL, incl, 1);
-        if (lane == 0) run = 0.0;
-        double zrun = run;                       // Z continues the same running sum as the prefixes
-        for (int i = b; i < en; ++i) zrun += e[(uint32_t)isort[i]];
-        const double Z = __shfl_sync(FULL, zrun, (n_final - 1) / per);
-        const double t = c * Z;
-        int pick = -1;
-        double pS = 0.0, pe = 1.0;
-        for (int i = b; i < en; ++i) {
-            const double ev = e[(uint32_t)isort[i]];
-            if (pick < 0 && (t < run + ev || i == n_final - 1)) { pick = i; pS = run; pe = ev; }
-            run += ev;
+    if (sm.b_i[1]) {
+        // ---- index order among the kept: src is free now, it receives (index << 32) | rank
+        if (tid < 4) dst[n_final + tid] = 0ull;    // ~0 = index 0xFFFFFFFF: never "smaller"
+        Sync::sync();
+        for (int r = tid; r < n_final; r += NT) {
+            const uint32_t idx = ~(uint32_t)dst[r];
+            int ir = 0;
+#pragma unroll 1
+            for (int q = 0; q < n_final; q += 4)
+                ir += (~(uint32_t)dst[q] < idx) + (~(uint32_t)dst[q + 1] < idx) +
+                      (~(uint32_t)dst[q + 2] < idx) + (~(uint32_t)dst[q + 3] < idx);
+            src[ir] = ((unsigned long long)idx << 32) | (uint32_t)r;
         }
-        const unsigned bal = __ballot_sync(FULL, pick >= 0);
-        const int L = __ffs(bal) - 1;
-        pick = __shfl_sync(FULL, pick, L);
-        pS = __shfl_sync(FULL, pS, L);
-        pe = __shfl_sync(FULL, pe, L);
-        if (lane == 0) {
-            double cn = (t - pS) / pe;
-            if (!(cn >= 0.0)) cn = 0.0;
-            if (cn > ASX_ONE_BELOW) cn = ASX_ONE_BELOW;
-            LaneResult r;
-            r.token = (int)(isort[pick] >> 32); r.status = ST_OK; r.n_kept = n_final; r.code_out = cn;
-            r.p_tok = pe / Z; r.cdf_lo = pS / Z;
-            sm.res = r;
+        Sync::sync();
+        if (warp == 0) {
+            const int per = (n_final + 31) / 32;
+            const int b = min(lane * per, n_final), en = min(b + per, n_final);
+            double s = 0.0;
+            for (int i = b; i < en; ++i) s += e[(uint32_t)src[i]];
+            const double incl = warp_incl_scan_d(s, lane);
+            double run = __shfl_up_sync(FULL, incl, 1);
+            if (lane == 0) run = 0.0;
+            double zrun = run;                   // Z continues the same running sum as the prefixes
+            for (int i = b; i < en; ++i) zrun += e[(uint32_t)src[i]];
+            const double Z = __shfl_sync(FULL, zrun, (n_final - 1) / per);
+            const double tt = c * Z;
+            int pick = -1;
+            double pS = 0.0, pe = 1.0;
+            for (int i = b; i < en; ++i) {
+                const double ev = e[(uint32_t)src[i]];
+                if (pick < 0 && (tt < run + ev || i == n_final - 1)) { pick = i; pS = run; pe = ev; }
+                run += ev;
+            }
+            const unsigned bal = __ballot_sync(FULL, pick >= 0);
+            const int L = __ffs(bal) - 1;
+            pick = __shfl_sync(FULL, pick, L);
+            pS = __shfl_sync(FULL, pS, L);
+            pe = __shfl_sync(FULL, pe, L);
+            // the three divisions on three lanes
+            const double num = lane == 0 ? (tt - pS) : lane == 1 ? pe : pS;
+            const double den = lane == 0 ? pe : Z;
+            const double quo = num / den;
+            const double p_tok = __shfl_sync(FULL, quo, 1), cdf_lo = __shfl_sync(FULL, quo, 2);
+            if (lane == 0) {
+                double cn = quo;
+                if (!(cn >= 0.0)) cn = 0.0;
+                if (cn > ASX_ONE_BELOW) cn = ASX_ONE_BELOW;
+                LaneResult r;
+                r.token = (int)(src[pick] >> 32); r.status = ST_OK; r.n_kept = n_final; r.code_out = cn;
+                r.p_tok = p_tok; r.cdf_lo = cdf_lo;
+                sm.res = r;
+            }
         }
     }
     Sync::sync();
     out = sm.res;
-    return true;
+    return sm.b_i[1] != 0;
 }
 
 template <int DT>
-__global__ void __launch_bounds__(SK_THREADS) step_stream_kernel(const StepArgs a, const int stages) {
+__global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepArgs a, const int stages) {
     using Tr = Traits<DT>;
     using P = Pass<DT>;
-    constexpr int E = Tr::E;
     constexpr int NT = SK_NT;
+    constexpr int E = Tr::E;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     StreamSmem& sm = *reinterpret_cast<StreamSmem*>(smem_raw);
     unsigned char* ring = smem_raw + ((sizeof(StreamSmem) + 127) & ~(size_t)127);
@@ -245,7 +261,6 @@ __global__ void __launch_bounds__(SK_THREADS) step_stream_kernel(const StepArgs 
                     }
                     const uint32_t bytes = (uint32_t)min(SK_STAGE_BYTES, bulk_bytes - s * SK_STAGE_BYTES);
                     const uint32_t bar = smem_u32(&sm.full_bar[st]);
-                    fence_proxy_async();
                     mbar_expect_tx(bar, bytes);
                     bulk_g2s(smem_u32(ring + (size_t)st * SK_STAGE_BYTES), src + (size_t)s * SK_STAGE_BYTES, bytes, bar);
                 }
@@ -258,58 +273,68 @@ __global__ void __launch_bounds__(SK_THREADS) step_stream_kernel(const StepArgs 
     const bool want_tail = (a.top_k == 0);        // nucleus-only: masses of non-candidates in fp32
     const int K0 = a.top_k > 0 ? a.top_k : SK_KP;
     const int m_sel = (K0 + SK_NW - 1) / SK_NW;
+    const float scale2 = a.scale2;
+    const uint32_t ninf_word = (DT == DT_BF16) ? 0xFF80FF80u : 0xFF800000u;
     unsigned g = 0;
+    int thr_calls = 0;
 
-    // block step: max so far and threshold from the subset maxima held in `acc`
-    auto threshold = [&](const typename P::Acc& acc, uint32_t& gmax, uint32_t& t0key) {
+    // block step: max so far and (optionally) threshold from the subset maxima held in `acc`;
+    // one barrier: the exchange slots are double-buffered between consecutive calls
+    auto threshold = [&](const typename P::Acc& acc, uint32_t& gmax, uint32_t& t0key, bool want_sel) {
         uint32_t k0, k1;
         P::keys(acc, k0, k1);
         const uint32_t wm = warp_max_u(max(k0, k1));
-        const uint32_t ws = warp_select16(P::key16(k0), P::key16(k1), m_sel);
-        SyncC::sync();                           // previous readers of wmax / wsel are done
-        if (lane == 0) { sm.wmax[warp] = wm; sm.wsel[warp] = ws; }
+        const uint32_t ws = want_sel ? warp_select16(P::key16(k0), P::key16(k1), m_sel) : 0u;
+        const int buf = thr_calls & 1;
+        ++thr_calls;
+        if (lane == 0) { sm.wmax[buf][warp] = wm; sm.wsel[buf][warp] = ws; }
         SyncC::sync();
         gmax = 0;
         uint32_t t16 = 0xFFFFFFFFu;
 #pragma unroll
-        for (int w = 0; w < SK_NW; ++w) { gmax = max(gmax, sm.wmax[w]); t16 = min(t16, sm.wsel[w]); }
+        for (int w = 0; w < SK_NW; ++w) { gmax = max(gmax, sm.wmax[buf][w]); t16 = min(t16, sm.wsel[buf][w]); }
         t0key = max(P::key_from16(t16), Tr::KEY_NINF);
     };
-    // compaction of one vector: candidates to the list, the rest to the fp32 tail
-    auto compact = [&](const uint4& q, int vec_index, uint32_t t0key, float t0f, float ref, float& tail) {
-        if (!want_tail) {
-            if (P::vmax(q) >= t0f) {
-                float x[E];
-                P::floats(q, x);
+    // SK_VPT vectors of one thread against the threshold.  Per vector: one packed max (shared with
+    // the running max when do_merge) and one compare.  Hit vectors are copied to the list: one
+    // ballot per vector position, one atomic per warp and position that has hits.  Nucleus-only
+    // lanes also sum 2^((x - ref) * scale2) over the vectors that are not listed.
+    auto slice_pass = [&](const uint4 (&q)[SK_VPT], int vec0, unsigned valid, bool do_merge, typename P::Acc& acc,
+                          float t0f, float ref, float& tail) {
+        unsigned hm = 0;
 #pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    if (x[e] >= t0f) {
-                        const uint32_t key = P::key_of_f(x[e]);
-                        if (key >= t0key && key > Tr::KEY_NINF) {
-                            const int slot = atomicAdd(&sm.cand_count, 1);
-                            if (slot < SK_CAP)
-                                sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)(vec_index * E + e);
+        for (int j = 0; j < SK_VPT; ++j) {
+            const typename P::Acc part = P::reduce(q[j]);
+            if (do_merge) P::merge(acc, part);
+            const bool hit = ((valid >> j) & 1u) && P::part_max(part) >= t0f;
+            hm |= (hit ? 1u : 0u) << j;
+            if (want_tail) {
+                float x[E];
+                P::floats(q[j], x);
+                float sacc = 0.f;
+#pragma unroll
+                for (int e = 0; e < E; ++e) sacc += ex2_approx((x[e] - ref) * scale2);
+                tail += hit ? 0.f : sacc;
+            }
+        }
+        if (__any_sync(FULL, hm != 0)) {
+#pragma unroll
+            for (int j = 0; j < SK_VPT; ++j) {
+                const bool hit = (hm >> j) & 1u;
+                const unsigned bal = __ballot_sync(FULL, hit);
+                if (bal) {
+                    const int leader = __ffs(bal) - 1;
+                    int base = 0;
+                    if (lane == leader) base = atomicAdd(&sm.vec_count, __popc(bal));
+                    base = __shfl_sync(FULL, base, leader);
+                    if (hit) {
+                        const int slot = base + __popc(bal & ((1u << lane) - 1u));
+                        if (slot < SK_CAPV) {
+                            sm.u.ep.v.cvec[slot] = q[j];
+                            sm.u.ep.cidx[slot] = vec0 + j * NT;
                         }
                     }
                 }
-            }
-        } else {
-            float x[E];
-            P::floats(q, x);
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-                const float ev = ex2_approx((x[e] - ref) * a.scale2);
-                bool pushed = false;
-                if (x[e] >= t0f) {
-                    const uint32_t key = P::key_of_f(x[e]);
-                    if (key >= t0key && key > Tr::KEY_NINF) {
-                        pushed = true;
-                        const int slot = atomicAdd(&sm.cand_count, 1);
-                        if (slot < SK_CAP)
-                            sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)(vec_index * E + e);
-                    }
-                }
-                tail += pushed ? 0.f : ev;
             }
         }
     };
@@ -321,17 +346,24 @@ __global__ void __launch_bounds__(SK_THREADS) step_stream_kernel(const StepArgs 
         if (c == 1.0) c = ASX_ONE_BELOW;
         const char* row = row_of(ln);
 
+        // Lanes the candidate list cannot decide end in ONE call of the general routine (kept out
+        // of line so that the hot path stays small).
+        const void* general_row = nullptr;      // set = run the general routine on this row
+        bool general_vec_ok = true;
+        bool general_release = false;           // resident row in the ring: release its stages after
+        LaneResult r;
+        int path = PATH_COMPACT;
+        bool decided = false;
+
         if (!staged_ok(ln)) {        // unaligned row: general routine from global memory
-            GenericLane<DT, NT, SyncC> gl(sm.u.gen, row, V, false);
-            const LaneResult r = gl.run(c_in, a.inv_tau, a.top_k, a.top_p);
-            if (tid == 0) write_result(a, ln, r, PATH_GENERAL);
-            continue;
+            general_row = row;
+            general_vec_ok = false;
         }
-        if (tid == 0) sm.cand_count = 0;
+        if (tid == 0) { sm.vec_count = 0; sm.cand_count = 0; }
 
         // ragged end of the row (< 16 bytes): one padded vector read straight from global memory
-        uint4 qt = make_uint4(0, 0, 0, 0);
-        if (tail_elems > 0 && tid == 0) {
+        uint4 qt = make_uint4(ninf_word, ninf_word, ninf_word, ninf_word);
+        if (tail_elems > 0 && tid == 0 && !general_row) {
             uint32_t w[4];
             if (DT == DT_BF16) {
                 const unsigned short* src = reinterpret_cast<const unsigned short*>(row + bulk_bytes);
@@ -353,161 +385,208 @@ __global__ void __launch_bounds__(SK_THREADS) step_stream_kernel(const StepArgs 
         uint32_t gmax = 0, t0key = Tr::KEY_NINF;
         float tail = 0.f;
         float ref = 0.f;             // exponent reference of the fp32 tail
-        bool timed_out = false;
+        float t0f = 0.f;
         const bool cut = a.fast && (a.top_k > 0 || a.top_p < 1.0);
 
         auto wait_full = [&](unsigned gg) {
-            if (*(volatile int*)&sm.poisoned) { timed_out = true; return; }
-            if (!mbar_wait_bounded(smem_u32(&sm.full_bar[gg % S]), (gg / S) & 1)) {
-                timed_out = true;
-                *(volatile int*)&sm.poisoned = 1;
-            }
+            if (*(volatile int*)&sm.poisoned) return;
+            if (!mbar_wait_bounded(smem_u32(&sm.full_bar[gg % S]), (gg / S) & 1)) *(volatile int*)&sm.poisoned = 1;
         };
         auto release = [&](unsigned gg) {
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sm.empty_bar[gg % S]));
         };
+        auto load_slice = [&](const uint4* sv, int nv, uint4 (&q)[SK_VPT]) -> unsigned {
+            unsigned valid = 0;
+#pragma unroll
+            for (int j = 0; j < SK_VPT; ++j) {
+                const int v = j * NT + tid;
+                const bool ok = v < nv;
+                valid |= (ok ? 1u : 0u) << j;
+                q[j] = ok ? sv[v] : make_uint4(ninf_word, ninf_word, ninf_word, ninf_word);
+            }
+            return valid;
+        };
 
-        if (resident) {
+        ASX_MARK(0);
+        if (general_row) {
+            // nothing was staged for this lane
+        } else if (resident) {
             // ---- all stages land; max pass from shared memory
+#pragma unroll 1
             for (int s = 0; s < nsl; ++s) {
                 wait_full(g + s);
-                const int nv = min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC);
-                const uint4* sv = ringv + (size_t)((g + s) % S) * SK_STAGE_VEC;
+                ASX_MARK(1);
+                uint4 q[SK_VPT];
+                load_slice(ringv + (size_t)((g + s) % S) * SK_STAGE_VEC, min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC), q);
 #pragma unroll
-                for (int j = 0; j < SK_VPT; ++j) {
-                    const int v = j * NT + tid;
-                    if (v < nv) P::fold(acc, sv[v]);
-                }
+                for (int j = 0; j < SK_VPT; ++j) P::merge(acc, P::reduce(q[j]));
             }
-            if (tail_elems > 0 && tid == 0) P::fold(acc, qt);
-            threshold(acc, gmax, t0key);
+            if (tid == 0) P::merge(acc, P::reduce(qt));
+            ASX_MARK(2);
+            threshold(acc, gmax, t0key, cut);
+            ASX_MARK(3);
             const bool bad = code_bad || gmax >= Tr::KEY_PINF || gmax <= Tr::KEY_NINF;
-            if (bad || !cut) {
-                LaneResult r;
-                if (bad) {
-                    r = failed_lane(c_in, ST_NUMERIC);
-                } else {
-                    // no cut: every token is kept; the general routine scans the row in shared memory
-                    if (tail_elems > 0 && tid < tail_elems) {
-                        if (DT == DT_BF16)
-                            reinterpret_cast<unsigned short*>(ring + bulk_bytes)[tid] =
-                                reinterpret_cast<const unsigned short*>(row + bulk_bytes)[tid];
-                        else
-                            reinterpret_cast<uint32_t*>(ring + bulk_bytes)[tid] =
-                                reinterpret_cast<const uint32_t*>(row + bulk_bytes)[tid];
-                    }
-                    SyncC::sync();
-                    GenericLane<DT, NT, SyncC> gl(sm.u.gen, ring, V, true);
-                    r = gl.run(c_in, a.inv_tau, a.top_k, a.top_p);
-                }
+            if (bad) {
+                r = failed_lane(c_in, ST_NUMERIC);
+                decided = true;
                 for (int s = 0; s < nsl; ++s) release(g + s);
-                g += nsl;
-                if (tid == 0) write_result(a, ln, r, bad ? PATH_COMPACT : PATH_GENERAL);
-                continue;
-            }
-            ref = Tr::value_f(gmax);
-            const float t0f = Tr::value_f(t0key);
-            for (int s = 0; s < nsl; ++s) {
-                const int nv = min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC);
-                const uint4* sv = ringv + (size_t)((g + s) % S) * SK_STAGE_VEC;
-#pragma unroll
-                for (int j = 0; j < SK_VPT; ++j) {
-                    const int v = j * NT + tid;
-                    if (v < nv) compact(sv[v], s * SK_STAGE_VEC + v, t0key, t0f, ref, tail);
+            } else if (!cut) {
+                // no cut: every token is kept; the general routine scans the row in shared memory
+                if (tail_elems > 0 && tid < tail_elems) {
+                    if (DT == DT_BF16)
+                        reinterpret_cast<unsigned short*>(ring + bulk_bytes)[tid] =
+                            reinterpret_cast<const unsigned short*>(row + bulk_bytes)[tid];
+                    else
+                        reinterpret_cast<uint32_t*>(ring + bulk_bytes)[tid] =
+                            reinterpret_cast<const uint32_t*>(row + bulk_bytes)[tid];
                 }
+                general_row = ring;
+                general_release = true;
+            } else {
+                ref = Tr::value_f(gmax);
+                t0f = Tr::value_f(t0key);
+#pragma unroll 1
+                for (int s = 0; s < nsl; ++s) {
+                    uint4 q[SK_VPT];
+                    const unsigned valid = load_slice(ringv + (size_t)((g + s) % S) * SK_STAGE_VEC,
+                                                      min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC), q);
+                    slice_pass(q, s * SK_STAGE_VEC + tid, valid, false, acc, t0f, ref, tail);
+                }
+                for (int s = 0; s < nsl; ++s) release(g + s);     // the producer may refill: next row
             }
-            if (tail_elems > 0 && tid == 0) compact(qt, bulk_vec, t0key, t0f, ref, tail);
-            for (int s = 0; s < nsl; ++s) release(g + s);     // the producer may refill: next row
-            g += nsl;
         } else {
             // ---- streamed: slice -> registers -> stage released; T0 at slices 0, 1, 2, 4, 8, ...
             int refresh_at = 1;
-            float t0f = 0.f;
+#ifdef ASX_PROFILE
+            long long pw = 0, pl = 0, pt = 0, pc = 0, tt0;
+#define ASX_ACC(var) do { const long long tt1 = clock64(); var += tt1 - tt0; tt0 = tt1; } while (0)
+            tt0 = clock64();
+#else
+#define ASX_ACC(var) do {} while (0)
+#endif
+#pragma unroll 1
             for (int s = 0; s < nsl; ++s, ++g) {
                 wait_full(g);
-                const int nv = min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC);
-                const uint4* sv = ringv + (size_t)(g % S) * SK_STAGE_VEC;
+                ASX_ACC(pw);
                 uint4 q[SK_VPT];
-#pragma unroll
-                for (int j = 0; j < SK_VPT; ++j) {
-                    const int v = j * NT + tid;
-                    q[j] = (v < nv) ? sv[v] : make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
-                }
-                if (DT == DT_F32) {
-#pragma unroll
-                    for (int j = 0; j < SK_VPT; ++j)
-                        if (j * NT + tid >= nv) q[j] = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
-                }
+                const unsigned valid = load_slice(ringv + (size_t)(g % S) * SK_STAGE_VEC,
+                                                  min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC), q);
                 release(g);
+                ASX_ACC(pl);
                 if (s == 0) {
 #pragma unroll
-                    for (int j = 0; j < SK_VPT; ++j) P::fold(acc, q[j]);
+                    for (int j = 0; j < SK_VPT; ++j) P::merge(acc, P::reduce(q[j]));
                 }
                 if (s == 0 || s == refresh_at) {
                     uint32_t gm, t0new;
-                    threshold(acc, gm, t0new);
+                    threshold(acc, gm, t0new, true);
                     t0key = max(t0key, t0new);
                     t0f = Tr::value_f(t0key);
                     if (s == 0) ref = Tr::value_f(min(max(gm, Tr::KEY_NINF + 1), Tr::KEY_PINF - 1));
                     if (s == refresh_at) refresh_at <<= 1;
                 }
-                if (s > 0) {
-#pragma unroll
-                    for (int j = 0; j < SK_VPT; ++j) P::fold(acc, q[j]);
-                }
-#pragma unroll
-                for (int j = 0; j < SK_VPT; ++j) {
-                    const int v = j * NT + tid;
-                    if (v < nv) compact(q[j], s * SK_STAGE_VEC + v, t0key, t0f, ref, tail);
-                }
+                ASX_ACC(pt);
+                slice_pass(q, s * SK_STAGE_VEC + tid, valid, s > 0, acc, t0f, ref, tail);
+                ASX_ACC(pc);
             }
-            if (tail_elems > 0 && tid == 0) {
-                P::fold(acc, qt);
-                compact(qt, bulk_vec, t0key, t0f, ref, tail);
-            }
+#ifdef ASX_PROFILE
+            if (blockIdx.x == 0 && tid == 0) { g_asx_marks[24] = pw; g_asx_marks[25] = pl; g_asx_marks[26] = pt; g_asx_marks[27] = pc; }
+#endif
+            if (tid == 0) P::merge(acc, P::reduce(qt));
             uint32_t t0unused;
-            threshold(acc, gmax, t0unused);       // final max (t0key keeps the value candidates were taken with)
+            threshold(acc, gmax, t0unused, false);   // final max (t0key keeps the value the hits were taken with)
             const bool bad = code_bad || gmax >= Tr::KEY_PINF || gmax <= Tr::KEY_NINF;
             if (bad) {
-                if (tid == 0) write_result(a, ln, failed_lane(c_in, ST_NUMERIC), PATH_COMPACT);
-                continue;
+                r = failed_lane(c_in, ST_NUMERIC);
+                decided = true;
             }
         }
 
-        // ---- candidate list complete: tail mass, then the exact epilogue
+        // ---- hit vectors -> candidates >= the final threshold; the rest of them joins the tail
+        ASX_MARK(4);
+        SyncC::sync();
+        const int nvh = sm.vec_count;
+        bool list_ok = !decided && !general_row && nvh <= SK_CAPV;
+        if (list_ok) {
+            for (int i = tid; i < nvh; i += NT) {
+                const uint4 q = sm.u.ep.v.cvec[i];
+                const int base = sm.u.ep.cidx[i] * E;
+                float x[E];
+                P::floats(q, x);
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    bool hit = false;
+                    if (x[e] >= t0f) {
+                        const uint32_t key = P::key_of_f(x[e]);
+                        if (key >= t0key && key > Tr::KEY_NINF) {
+                            hit = true;
+                            const int slot = atomicAdd(&sm.cand_count, 1);
+                            if (slot < SK_CAP)
+                                sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)(base + e);
+                        }
+                    }
+                    if (want_tail && !hit) tail += ex2_approx((x[e] - ref) * scale2);
+                }
+            }
+            if (tail_elems > 0 && tid == 0) {      // the ragged last vector lives in thread 0's registers
+                float x[E];
+                P::floats(qt, x);
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    bool hit = false;
+                    if (x[e] >= t0f) {
+                        const uint32_t key = P::key_of_f(x[e]);
+                        if (key >= t0key && key > Tr::KEY_NINF) {
+                            hit = true;
+                            const int slot = atomicAdd(&sm.cand_count, 1);
+                            if (slot < SK_CAP)
+                                sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)(bulk_vec * E + e);
+                        }
+                    }
+                    if (want_tail && !hit) tail += ex2_approx((x[e] - ref) * scale2);
+                }
+            }
+        }
         double tailsum = 0.0;
         if (want_tail) {
             const double td = warp_sum_d((double)tail);
-            SyncC::sync();
             if (lane == 0) sm.red_d[warp] = td;
-            SyncC::sync();
+        }
+        SyncC::sync();                      // candidates complete; cvec is dead from here on
+        if (want_tail) {
 #pragma unroll
             for (int w = 0; w < SK_NW; ++w) tailsum += sm.red_d[w];
-        } else {
-            SyncC::sync();
         }
-        (void)timed_out;                          // a wait that ran out has set sm.poisoned
+        const int C = sm.cand_count;
+        list_ok = list_ok && C > 0 && C <= SK_CAP;
         const double lmax = (double)Tr::value_f(gmax);
         // the tail was summed against `ref` (<= lmax); bring it to the true maximum
         if (want_tail) tailsum *= exp_nonpos(((double)ref - lmax) * a.inv_tau, sm.exp_tbl);
-        const int C = sm.cand_count;
-        LaneResult r;
-        bool done = false;
+        ASX_MARK(5);
+#ifdef ASX_PROFILE
+        if (blockIdx.x == 0 && tid == 0) { g_asx_marks[20] = nvh; g_asx_marks[21] = C; }
+#endif
         if (*(volatile int*)&sm.poisoned) {
             r = failed_lane(c_in, ST_TIMEOUT);
-            done = true;
-        } else if (C > 0 && C <= SK_CAP && (!want_tail || (tailsum == tailsum && tailsum < 1e300))) {
-            done = epilogue_sorted<DT, NT, SyncC>(sm, C, t0key, c, lmax, a.inv_tau, a.top_k, a.top_p, tailsum, r);
+            decided = true;
+        } else if (list_ok && (!want_tail || (tailsum == tailsum && tailsum < 1e300))) {
+            decided = epilogue_ranked<DT, NT, SyncC>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, t0key, c,
+                                                     lmax, a.inv_tau, a.top_k, a.top_p, tailsum, r);
         }
-        const int path = done ? PATH_COMPACT : PATH_GENERAL;
-        if (!done) {
+        if (!decided) {
+            if (!general_row) general_row = row;          // the row again, from global memory (L2)
             SyncC::sync();
-            GenericLane<DT, NT, SyncC> gl(sm.u.gen, row, V, true);
+            GenericLane<DT, NT, SyncC> gl(sm.u.gen, general_row, V, general_vec_ok);
             r = gl.run(c_in, a.inv_tau, a.top_k, a.top_p);
+            path = PATH_GENERAL;
+            if (general_release)
+                for (int s = 0; s < nsl; ++s) release(g + s);
         }
+        if (resident && staged_ok(ln)) g += nsl;
         if (tid == 0) write_result(a, ln, r, path);
         SyncC::sync();
+        ASX_MARK(12);
     }
 }
 
