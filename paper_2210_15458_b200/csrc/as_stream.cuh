@@ -82,6 +82,23 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // m-th largest (1-based) of the 64 16-bit keys held two per lane, by a search on the value, two
 // bits per step: the largest v with count(keys >= v) >= m (0 if fewer than m keys are positive).
 __device__ __forceinline__ uint32_t warp_select16(uint32_t a16, uint32_t b16, int m) {
+    if (m <= 6) {
+        // few steps: take the maximum m times, removing one occurrence each time
+        const int lane = threadIdx.x & 31;
+        uint32_t cur = 0;
+#pragma unroll 1
+        for (int it = 0; it < m; ++it) {
+            cur = warp_max_u(max(a16, b16));
+            const unsigned ba = __ballot_sync(FULL, a16 == cur);
+            if (ba) {
+                if (lane == __ffs(ba) - 1) a16 = 0;
+            } else {
+                const unsigned bb = __ballot_sync(FULL, b16 == cur);
+                if (lane == __ffs(bb) - 1) b16 = 0;
+            }
+        }
+        return cur;
+    }
     uint32_t res = 0;
 #pragma unroll 1
     for (int bit = 14; bit >= 0; bit -= 2) {
@@ -104,9 +121,9 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
                                              LaneResult& out) {
     using Tr = Traits<DT>;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid < 4) src[C + tid] = 0ull;             // padding for the 4-wide rank loop
-    Sync::sync();
-    // ---- ranks by (value desc, index asc): composites are distinct -> a permutation
+    // (src[C..C+3] are zero: the caller zero-fills the array before collecting candidates)
+    // ---- ranks by (value desc, index asc): composites are distinct -> a permutation; each
+    //      thread also computes the mass of its own candidate and stores it by rank
     for (int i = tid; i < C; i += NT) {
         const unsigned long long ci = src[i];
         int r = 0;
@@ -114,16 +131,15 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
         for (int j = 0; j < C; j += 4)
             r += (src[j] > ci) + (src[j + 1] > ci) + (src[j + 2] > ci) + (src[j + 3] > ci);
         dst[r] = ci;
+        e[r] = exp_nonpos(((double)Tr::value_f((uint32_t)(ci >> 32)) - lmax) * inv_tau, sm.exp_tbl);
     }
-    Sync::sync();
     const int kmax = (top_k > 0 && top_k < C) ? top_k : C;
-    for (int r = tid; r < kmax; r += NT)
-        e[r] = exp_nonpos(((double)Tr::value_f((uint32_t)(dst[r] >> 32)) - lmax) * inv_tau, sm.exp_tbl);
+    if (tid < 4) dst[C + tid] = 0ull;             // ~0 = index 0xFFFFFFFF: never "smaller"
     Sync::sync();
-    if (warp == 0) {
-        // prefix masses in rank order: nucleus on the distribution renormalised over the survivors
-        int n_final = kmax, ok = 1;
-        if (top_p < 1.0) {
+    if (top_p < 1.0) {
+        if (warp == 0) {
+            // prefix masses in rank order: nucleus on the distribution renormalised over the survivors
+            int n_final = kmax, ok = 1;
             const int per = (kmax + 31) / 32;
             const int b = min(lane * per, kmax), en = min(b + per, kmax);
             double s = 0.0;
@@ -141,16 +157,27 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
             } else {
                 n_final = below + 1;
             }
+            if (ok && (uint32_t)(dst[n_final - 1] >> 32) < depth_key) ok = 0;   // cut below the exact depth
+            __syncwarp();
+            if (lane == 0) {
+                sm.b_i[0] = n_final; sm.b_i[1] = ok;
+                // entries past the kept ranks must not count in the index loop
+                if (n_final < C) { dst[n_final] = 0ull; dst[n_final + 1] = 0ull; dst[n_final + 2] = 0ull; dst[n_final + 3] = 0ull; }
+            }
         }
-        if (ok && (uint32_t)(dst[n_final - 1] >> 32) < depth_key) ok = 0;   // cut below the exact depth
-        if (lane == 0) { sm.b_i[0] = n_final; sm.b_i[1] = ok; }
+        Sync::sync();
+    } else {
+        // top-k only: the answer follows from kmax alone
+        if (tid == 0) { sm.b_i[0] = kmax; sm.b_i[1] = ((uint32_t)(dst[kmax - 1] >> 32) >= depth_key) ? 1 : 0; }
+        if (kmax < C) {
+            Sync::sync();
+            if (tid < 4) dst[kmax + tid] = 0ull;  // entries past the kept ranks must not count below
+        }
+        Sync::sync();
     }
-    Sync::sync();
     const int n_final = sm.b_i[0];
     if (sm.b_i[1]) {
         // ---- index order among the kept: src is free now, it receives (index << 32) | rank
-        if (tid < 4) dst[n_final + tid] = 0ull;    // ~0 = index 0xFFFFFFFF: never "smaller"
-        Sync::sync();
         for (int r = tid; r < n_final; r += NT) {
             const uint32_t idx = ~(uint32_t)dst[r];
             int ir = 0;
@@ -360,6 +387,9 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
             general_vec_ok = false;
         }
         if (tid == 0) { sm.vec_count = 0; sm.cand_count = 0; }
+        // the candidate array starts zeroed: entries past the count rank below every candidate,
+        // which the epilogue's 4-wide rank loop relies on
+        for (int i = tid; i < SK_CAP + 4; i += NT) sm.u.ep.cand[i] = 0ull;
 
         // ragged end of the row (< 16 bytes): one padded vector read straight from global memory
         uint4 qt = make_uint4(ninf_word, ninf_word, ninf_word, ninf_word);
