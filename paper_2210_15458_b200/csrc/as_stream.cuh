@@ -41,6 +41,7 @@ constexpr int SK_STAGE_VEC = 1024;         // 16-byte vectors per stage (16 KB)
 constexpr int SK_STAGE_BYTES = SK_STAGE_VEC * 16;
 constexpr int SK_VPT = SK_STAGE_VEC / SK_NT;   // vectors per consumer thread per slice
 constexpr int SK_MAXSTAGES = 12;
+constexpr int SK_RES_STAGES = 6;           // rows of up to this many stages (96 KB) stay resident
 constexpr int SK_K0_RESIDENT = 256;        // largest top_k served by the list, resident rows
 constexpr int SK_K0_STREAMED = 96;         // ... streamed rows (hits grow like K0 ln(V / K0))
 constexpr int SK_KP = 96;                  // K0 for nucleus-only lanes
@@ -442,15 +443,26 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
         if (general_row) {
             // nothing was staged for this lane
         } else if (resident) {
-            // ---- all stages land; max pass from shared memory
-#pragma unroll 1
-            for (int s = 0; s < nsl; ++s) {
-                wait_full(g + s);
-                ASX_MARK(1);
-                uint4 q[SK_VPT];
-                load_slice(ringv + (size_t)((g + s) % S) * SK_STAGE_VEC, min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC), q);
+            // ---- all stages land; max pass from shared memory.  Each vector's own maximum stays
+            //      in a register, so the hit test after the threshold needs no second pass.
+            float pm[SK_RES_STAGES * SK_VPT];
 #pragma unroll
-                for (int j = 0; j < SK_VPT; ++j) P::merge(acc, P::reduce(q[j]));
+            for (int s = 0; s < SK_RES_STAGES; ++s) {
+                if (s < nsl) {
+                    wait_full(g + s);
+                    ASX_MARK(1);
+                    uint4 q[SK_VPT];
+                    load_slice(ringv + (size_t)((g + s) % S) * SK_STAGE_VEC, min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC), q);
+#pragma unroll
+                    for (int j = 0; j < SK_VPT; ++j) {
+                        const typename P::Acc part = P::reduce(q[j]);
+                        P::merge(acc, part);
+                        pm[s * SK_VPT + j] = P::part_max(part);      // -inf for vectors past the row
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < SK_VPT; ++j) pm[s * SK_VPT + j] = __uint_as_float(0xFF800000u);
+                }
             }
             if (tid == 0) P::merge(acc, P::reduce(qt));
             ASX_MARK(2);
@@ -476,12 +488,41 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
             } else {
                 ref = Tr::value_f(gmax);
                 t0f = Tr::value_f(t0key);
+                if (!want_tail) {
+                    // the threshold is final here: vectors whose maximum passes give their elements
+                    // straight to the candidate list
+                    unsigned hm = 0;
+#pragma unroll
+                    for (int i = 0; i < SK_RES_STAGES * SK_VPT; ++i) hm |= (pm[i] >= t0f ? 1u : 0u) << i;
 #pragma unroll 1
-                for (int s = 0; s < nsl; ++s) {
-                    uint4 q[SK_VPT];
-                    const unsigned valid = load_slice(ringv + (size_t)((g + s) % S) * SK_STAGE_VEC,
-                                                      min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC), q);
-                    slice_pass(q, s * SK_STAGE_VEC + tid, valid, false, acc, t0f, ref, tail);
+                    while (hm) {
+                        const int i = __ffs(hm) - 1;
+                        hm &= hm - 1;
+                        const int s = i / SK_VPT, v = (i % SK_VPT) * NT + tid;
+                        const uint4 q = ringv[(size_t)((g + s) % S) * SK_STAGE_VEC + v];
+                        float x[E];
+                        P::floats(q, x);
+#pragma unroll
+                        for (int e = 0; e < E; ++e) {
+                            if (x[e] >= t0f) {
+                                const uint32_t key = P::key_of_f(x[e]);
+                                if (key >= t0key && key > Tr::KEY_NINF) {
+                                    const int slot = atomicAdd(&sm.cand_count, 1);
+                                    if (slot < SK_CAP)
+                                        sm.u.ep.cand[slot] = ((unsigned long long)key << 32) |
+                                                             (uint32_t)~(uint32_t)((s * SK_STAGE_VEC + v) * E + e);
+                                }
+                            }
+                        }
+                    }
+                } else {
+#pragma unroll 1
+                    for (int s = 0; s < nsl; ++s) {
+                        uint4 q[SK_VPT];
+                        const unsigned valid = load_slice(ringv + (size_t)((g + s) % S) * SK_STAGE_VEC,
+                                                          min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC), q);
+                        slice_pass(q, s * SK_STAGE_VEC + tid, valid, false, acc, t0f, ref, tail);
+                    }
                 }
                 for (int s = 0; s < nsl; ++s) release(g + s);     // the producer may refill: next row
             }
