@@ -134,6 +134,7 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
         dst[r] = ci;
         e[r] = exp_nonpos(((double)Tr::value_f((uint32_t)(ci >> 32)) - lmax) * inv_tau, sm.exp_tbl);
     }
+    ASX_MARK(6);
     const int kmax = (top_k > 0 && top_k < C) ? top_k : C;
     if (tid < 4) dst[C + tid] = 0ull;             // ~0 = index 0xFFFFFFFF: never "smaller"
     Sync::sync();
@@ -176,6 +177,7 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
         }
         Sync::sync();
     }
+    ASX_MARK(7);
     const int n_final = sm.b_i[0];
     if (sm.b_i[1]) {
         // ---- index order among the kept: src is free now, it receives (index << 32) | rank
@@ -189,24 +191,50 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
             src[ir] = ((unsigned long long)idx << 32) | (uint32_t)r;
         }
         Sync::sync();
+        ASX_MARK(8);
         if (warp == 0) {
+            // lane l owns index-order positions [b, en); up to 4 masses are kept in registers
             const int per = (n_final + 31) / 32;
             const int b = min(lane * per, n_final), en = min(b + per, n_final);
+            double ev4[4] = {0.0, 0.0, 0.0, 0.0};
             double s = 0.0;
-            for (int i = b; i < en; ++i) s += e[(uint32_t)src[i]];
+            if (per <= 4) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (b + k < en) { ev4[k] = e[(uint32_t)src[b + k]]; s += ev4[k]; }
+            } else {
+                for (int i = b; i < en; ++i) s += e[(uint32_t)src[i]];
+            }
             const double incl = warp_incl_scan_d(s, lane);
             double run = __shfl_up_sync(FULL, incl, 1);
             if (lane == 0) run = 0.0;
-            double zrun = run;                   // Z continues the same running sum as the prefixes
-            for (int i = b; i < en; ++i) zrun += e[(uint32_t)src[i]];
+            // Z continues the same running sum as the prefixes: run + (elements in order)
+            double zrun = run;
+            if (per <= 4) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) if (b + k < en) zrun += ev4[k];
+            } else {
+                for (int i = b; i < en; ++i) zrun += e[(uint32_t)src[i]];
+            }
             const double Z = __shfl_sync(FULL, zrun, (n_final - 1) / per);
             const double tt = c * Z;
             int pick = -1;
             double pS = 0.0, pe = 1.0;
-            for (int i = b; i < en; ++i) {
-                const double ev = e[(uint32_t)src[i]];
-                if (pick < 0 && (tt < run + ev || i == n_final - 1)) { pick = i; pS = run; pe = ev; }
-                run += ev;
+            if (per <= 4) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if (b + k < en) {
+                        const double ev = ev4[k];
+                        if (pick < 0 && (tt < run + ev || b + k == n_final - 1)) { pick = b + k; pS = run; pe = ev; }
+                        run += ev;
+                    }
+                }
+            } else {
+                for (int i = b; i < en; ++i) {
+                    const double ev = e[(uint32_t)src[i]];
+                    if (pick < 0 && (tt < run + ev || i == n_final - 1)) { pick = i; pS = run; pe = ev; }
+                    run += ev;
+                }
             }
             const unsigned bal = __ballot_sync(FULL, pick >= 0);
             const int L = __ffs(bal) - 1;
@@ -229,7 +257,9 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
             }
         }
     }
+    ASX_MARK(9);
     Sync::sync();
+    ASX_MARK(10);
     out = sm.res;
     return sm.b_i[1] != 0;
 }
@@ -246,6 +276,7 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
     const uint4* ringv = reinterpret_cast<const uint4*>(ring);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    ASX_MARK(13);
     const int V = a.V;
     const int row_bytes = V * Tr::BYTES;
     const int bulk_bytes = row_bytes & ~15;
@@ -255,48 +286,57 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
     const bool resident = nsl <= stages;
     const int S = resident ? max(nsl, 1) : stages;                     // ring length in use
 
-    if (tid == 0) {
-        for (int i = 0; i < SK_MAXSTAGES; ++i) {
-            mbar_init(smem_u32(&sm.full_bar[i]), 1);
-            mbar_init(smem_u32(&sm.empty_bar[i]), SK_NW);
-        }
-        fence_mbar_init();
-        sm.poisoned = 0;
-    }
-    fill_exp_table(sm.exp_tbl, tid);
-    __syncthreads();
-
     auto row_of = [&](int ln) -> const char* {
         return reinterpret_cast<const char*>(a.logits) + (size_t)ln * (size_t)a.ld * Tr::BYTES;
     };
     auto staged_ok = [&](int ln) -> bool { return (reinterpret_cast<uintptr_t>(row_of(ln)) & 15) == 0; };
 
+    // The producer lane initialises the barriers of the stages in use and starts the first copies
+    // before the block-wide barrier, so the first row is in flight while the rest of the CTA sets up.
+    const bool is_producer = (warp == SK_NW && lane == 0);
+    unsigned g_issued = 0;                        // producer: slices issued so far
+    int ln_issue = blockIdx.x;                    // producer: lane whose slices come next
+    int s_issue = 0;
+    auto issue_some = [&](bool first_row_only) -> bool {   // false: a bounded wait ran out
+        for (; ln_issue < a.lanes; ln_issue += gridDim.x, s_issue = 0) {
+            if (!staged_ok(ln_issue)) continue;
+            const char* src = row_of(ln_issue);
+            for (; s_issue < nsl; ++s_issue, ++g_issued) {
+                const int st = g_issued % S;
+                if (g_issued >= (unsigned)S) {    // the stage must have been drained by every consumer warp
+                    if (first_row_only) return true;
+                    if (*(volatile int*)&sm.poisoned) return false;
+                    if (!mbar_wait_bounded(smem_u32(&sm.empty_bar[st]), ((g_issued / S) - 1) & 1)) {
+                        *(volatile int*)&sm.poisoned = 1;
+                        return false;
+                    }
+                }
+                const uint32_t bytes = (uint32_t)min(SK_STAGE_BYTES, bulk_bytes - s_issue * SK_STAGE_BYTES);
+                const uint32_t bar = smem_u32(&sm.full_bar[st]);
+                mbar_expect_tx(bar, bytes);
+                bulk_g2s(smem_u32(ring + (size_t)st * SK_STAGE_BYTES), src + (size_t)s_issue * SK_STAGE_BYTES, bytes, bar);
+            }
+            if (first_row_only) { ln_issue += gridDim.x; s_issue = 0; return true; }
+        }
+        return true;
+    };
+    if (is_producer) {
+        for (int i = 0; i < S; ++i) {
+            mbar_init(smem_u32(&sm.full_bar[i]), 1);
+            mbar_init(smem_u32(&sm.empty_bar[i]), SK_NW);
+        }
+        fence_mbar_init();
+        sm.poisoned = 0;
+        issue_some(true);                         // fills the ring without waiting
+    }
+    fill_exp_table(sm.exp_tbl, tid);
+    __syncthreads();
+
     // =========================== producer warp ===========================
     if (warp == SK_NW) {
-        if (lane == 0) {
-            unsigned g = 0;                       // slices issued so far (ring position)
-            for (int ln = blockIdx.x; ln < a.lanes; ln += gridDim.x) {
-                if (!staged_ok(ln)) continue;
-                const char* src = row_of(ln);
-                for (int s = 0; s < nsl; ++s, ++g) {
-                    const int st = g % S;
-                    if (g >= (unsigned)S) {       // the stage must have been drained by every consumer warp
-                        if (*(volatile int*)&sm.poisoned) return;
-                        if (!mbar_wait_bounded(smem_u32(&sm.empty_bar[st]), ((g / S) - 1) & 1)) {
-                            *(volatile int*)&sm.poisoned = 1;
-                            return;
-                        }
-                    }
-                    const uint32_t bytes = (uint32_t)min(SK_STAGE_BYTES, bulk_bytes - s * SK_STAGE_BYTES);
-                    const uint32_t bar = smem_u32(&sm.full_bar[st]);
-                    mbar_expect_tx(bar, bytes);
-                    bulk_g2s(smem_u32(ring + (size_t)st * SK_STAGE_BYTES), src + (size_t)s * SK_STAGE_BYTES, bytes, bar);
-                }
-            }
-        }
+        if (lane == 0) issue_some(false);
         return;
     }
-
     // =========================== consumer warps ===========================
     const bool want_tail = (a.top_k == 0);        // nucleus-only: masses of non-candidates in fp32
     const int K0 = a.top_k > 0 ? a.top_k : SK_KP;
@@ -659,6 +699,7 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
         SyncC::sync();
         ASX_MARK(12);
     }
+    ASX_MARK(14);
 }
 
 }  // namespace asx
