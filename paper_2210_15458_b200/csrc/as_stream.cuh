@@ -69,6 +69,7 @@ struct StreamSmem {
     double red_d[SK_NW];
     unsigned wmax[2][SK_NW];
     unsigned wsel[2][SK_NW];
+    double list_mass;    // epilogue: total mass of the ranked list (nucleus lanes)
     int vec_count;
     int cand_count;
     int poisoned;        // a bounded wait ran out: stop issuing / stop waiting
@@ -148,6 +149,7 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
             for (int r = b; r < en; ++r) s += e[r];
             const double incl = warp_incl_scan_d(s, lane);
             const double total = __shfl_sync(FULL, incl, 31);
+            if (lane == 0) sm.list_mass = total;
             const double target = top_p * (total + tail);
             double run = __shfl_up_sync(FULL, incl, 1);
             if (lane == 0) run = 0.0;
@@ -262,6 +264,122 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
     ASX_MARK(10);
     out = sm.res;
     return sm.b_i[1] != 0;
+}
+
+// Nucleus-only lane whose nucleus reaches below the exact depth of the list (key >= t0key).
+// The row is read again from global memory (it was just streamed, so mostly from L2):
+//   1. masses and counts of the elements below the old threshold go into a histogram over
+//      y = (x - max) * scale2, 64 bins per unit of log2 mass, 16 units deep;
+//   2. the bins are taken from the top until their mass covers what the nucleus still lacks
+//      (with a margin for the fp32 sums): that gives a lower threshold t1 below which no
+//      nucleus token can lie, if the candidates still fit the list;
+//   3. everything >= t1 is collected afresh, the rest summed in fp32, and the exact epilogue
+//      runs again.  Returns false if the window or the list capacity does not suffice.
+constexpr int DP_NB = 1024;
+constexpr float DP_BINS_PER_UNIT = 64.f;
+template <int DT>
+__device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, const StepArgs& a, const char* row, uint32_t gmax,
+                                            float t0f, double tailsum, double c, LaneResult& r) {
+    using Tr = Traits<DT>;
+    using P = Pass<DT>;
+    constexpr int E = Tr::E;
+    constexpr int NT = SK_NT;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int V = a.V;
+    const int nvec_full = (V * Tr::BYTES) >> 4;           // whole 16-byte vectors
+    const float lmaxf = Tr::value_f(gmax);
+    const float scale2 = a.scale2;
+    const float y0 = (t0f - lmaxf) * scale2;
+    float* hmass = reinterpret_cast<float*>(sm.u.ep.v.cvec);
+    int* hcnt = reinterpret_cast<int*>(hmass + DP_NB);
+    const double list_mass = sm.list_mass;
+    SyncC::sync();                                         // the epilogue's arrays are dead
+    for (int i = tid; i < DP_NB; i += NT) { hmass[i] = 0.f; hcnt[i] = 0; }
+    if (tid == 0) sm.cand_count = 0;
+    for (int i = tid; i < SK_CAP + 4; i += NT) sm.u.ep.cand[i] = 0ull;
+    SyncC::sync();
+    auto visit = [&](auto&& f) {                           // f(x, index) over the whole row
+        for (int v = tid; v < nvec_full; v += NT) {
+            const uint4 q = __ldg(reinterpret_cast<const uint4*>(row) + v);
+            float x[E];
+            P::floats(q, x);
+#pragma unroll
+            for (int e = 0; e < E; ++e) f(x[e], v * E + e);
+        }
+        for (int j = nvec_full * E + tid; j < V; j += NT) f(Tr::value_f(Tr::load_key(row, j)), j);
+    };
+    // ---- 1. histogram below the old threshold
+    visit([&](float x, int) {
+        if (x < t0f) {
+            const float y = (x - lmaxf) * scale2;
+            const float d = (y0 - y) * DP_BINS_PER_UNIT;
+            if (d < (float)DP_NB) {
+                const int bin = (int)d;
+                atomicAdd(&hcnt[bin], 1);
+                atomicAdd(&hmass[bin], ex2_approx(y));
+            }
+        }
+    });
+    SyncC::sync();
+    // ---- 2. lowest bin needed
+    if (warp == 0) {
+        const double target = a.top_p * (list_mass + tailsum);
+        const double need = (target - list_mass) * 1.002 + 1e-7 * target;
+        constexpr int PER = DP_NB / 32;
+        double m = 0.0;
+        int n = 0;
+        for (int i = 0; i < PER; ++i) { m += (double)hmass[lane * PER + i]; n += hcnt[lane * PER + i]; }
+        const double mi = warp_incl_scan_d(m, lane);
+        const int ni = warp_incl_scan_i(n, lane);
+        double run = mi - m;
+        int cnt = ni - n;
+        int found = -1, found_cnt = 0;
+        for (int i = 0; i < PER; ++i) {
+            run += (double)hmass[lane * PER + i];
+            cnt += hcnt[lane * PER + i];
+            if (found < 0 && run >= need) { found = lane * PER + i; found_cnt = cnt; }
+        }
+        const unsigned bal = __ballot_sync(FULL, found >= 0);
+        int bin = -1, below = 0;
+        if (bal) {
+            const int L = __ffs(bal) - 1;
+            bin = __shfl_sync(FULL, found, L);
+            below = __shfl_sync(FULL, found_cnt, L);
+        }
+        if (lane == 0) { sm.b_i[0] = bin; sm.b_i[1] = below; }
+    }
+    SyncC::sync();
+    const int bin = sm.b_i[0];
+    const int old_count = sm.b_i[2];
+    if (bin < 0 || sm.b_i[1] + old_count > SK_CAP - 8) return false;
+    const float t1f = lmaxf + (y0 - (float)(bin + 1) / DP_BINS_PER_UNIT - 2e-3f) / scale2;
+    uint32_t depth_key = P::key_of_f(t1f);
+    if (Tr::value_f(depth_key) < t1f) depth_key += 1;     // smallest key whose value is >= t1
+    SyncC::sync();
+    // ---- 3. collect afresh
+    float tail = 0.f;
+    visit([&](float x, int j) {
+        bool hit = false;
+        if (x >= t1f) {
+            const uint32_t key = P::key_of_f(x);
+            if (key > Tr::KEY_NINF) {
+                hit = true;
+                const int slot = atomicAdd(&sm.cand_count, 1);
+                if (slot < SK_CAP) sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)j;
+            }
+        }
+        if (!hit) tail += ex2_approx((x - lmaxf) * scale2);
+    });
+    const double td = warp_sum_d((double)tail);
+    if (lane == 0) sm.red_d[warp] = td;
+    SyncC::sync();
+    double tsum = 0.0;
+#pragma unroll
+    for (int w = 0; w < SK_NW; ++w) tsum += sm.red_d[w];
+    const int C = sm.cand_count;
+    if (C <= 0 || C > SK_CAP || !(tsum == tsum) || !(tsum < 1e300)) return false;
+    return epilogue_ranked<DT, NT, SyncC>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, depth_key, c,
+                                          (double)lmaxf, a.inv_tau, a.top_k, a.top_p, tsum, r);
 }
 
 template <int DT>
@@ -684,6 +802,11 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
         } else if (list_ok && (!want_tail || (tailsum == tailsum && tailsum < 1e300))) {
             decided = epilogue_ranked<DT, NT, SyncC>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, t0key, c,
                                                      lmax, a.inv_tau, a.top_k, a.top_p, tailsum, r);
+        }
+        if (!decided && want_tail && list_ok && !*(volatile int*)&sm.poisoned) {
+            // the nucleus reaches below the exact depth of the list: lower the threshold once
+            if (tid == 0) sm.b_i[2] = C;
+            decided = deepen_nucleus<DT>(sm, a, row, gmax, t0f, tailsum, c, r);
         }
         if (!decided) {
             if (!general_row) general_row = row;          // the row again, from global memory (L2)
