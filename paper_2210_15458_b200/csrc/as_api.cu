@@ -269,6 +269,9 @@ int as_version(void) { return 1000; }
 int as_debug_marks(long long* h_out) {
     return cudaMemcpyFromSymbol(h_out, g_asx_marks, sizeof(long long) * 32) == cudaSuccess ? AS_OK : AS_ERR_CUDA;
 }
+int as_debug_counts(unsigned long long* h_out) {
+    return cudaMemcpyFromSymbol(h_out, g_asx_counts, sizeof(unsigned long long) * 16) == cudaSuccess ? AS_OK : AS_ERR_CUDA;
+}
 #endif
 
 const char* as_last_error(void) { return g_err; }

@@ -43,9 +43,12 @@ constexpr long long ST_WAIT_CYCLES = 4000000000LL;   // ~2 s: bound on any mbarr
 // Phase timestamps of CTA 0 for profiling builds (-DASX_PROFILE); compiled out otherwise.
 #ifdef ASX_PROFILE
 __device__ long long g_asx_marks[32];
+__device__ unsigned long long g_asx_counts[16];
 #define ASX_MARK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_asx_marks[i] = clock64(); } while (0)
+#define ASX_COUNT(i) do { if (threadIdx.x == 0) atomicAdd(&g_asx_counts[i], 1ull); } while (0)
 #else
 #define ASX_MARK(i) do {} while (0)
+#define ASX_COUNT(i) do {} while (0)
 #endif
 
 struct DiagOut {

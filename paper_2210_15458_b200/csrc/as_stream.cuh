@@ -35,7 +35,7 @@ namespace asx {
 constexpr int SK_NT = 256;                 // consumer threads
 constexpr int SK_NW = SK_NT / 32;          // consumer warps
 constexpr int SK_THREADS = SK_NT + 32;     // + producer warp
-constexpr int SK_CAPV = 1024;              // hit-vector capacity per lane
+constexpr int SK_CAPV = 2048;              // hit-vector capacity per lane
 constexpr int SK_CAP = 512;                // candidate (element) capacity per lane
 constexpr int SK_STAGE_VEC = 1024;         // 16-byte vectors per stage (16 KB)
 constexpr int SK_STAGE_BYTES = SK_STAGE_VEC * 16;
@@ -351,7 +351,8 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, const StepArgs& a, c
     SyncC::sync();
     const int bin = sm.b_i[0];
     const int old_count = sm.b_i[2];
-    if (bin < 0 || sm.b_i[1] + old_count > SK_CAP - 8) return false;
+    if (bin < 0) { ASX_COUNT(1); return false; }
+    if (sm.b_i[1] + old_count > SK_CAP - 8) { ASX_COUNT(2); return false; }
     const float t1f = lmaxf + (y0 - (float)(bin + 1) / DP_BINS_PER_UNIT - 2e-3f) / scale2;
     uint32_t depth_key = P::key_of_f(t1f);
     if (Tr::value_f(depth_key) < t1f) depth_key += 1;     // smallest key whose value is >= t1
@@ -377,9 +378,11 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, const StepArgs& a, c
 #pragma unroll
     for (int w = 0; w < SK_NW; ++w) tsum += sm.red_d[w];
     const int C = sm.cand_count;
-    if (C <= 0 || C > SK_CAP || !(tsum == tsum) || !(tsum < 1e300)) return false;
-    return epilogue_ranked<DT, NT, SyncC>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, depth_key, c,
-                                          (double)lmaxf, a.inv_tau, a.top_k, a.top_p, tsum, r);
+    if (C <= 0 || C > SK_CAP || !(tsum == tsum) || !(tsum < 1e300)) { ASX_COUNT(3); return false; }
+    const bool ok2 = epilogue_ranked<DT, NT, SyncC>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, depth_key, c,
+                                                    (double)lmaxf, a.inv_tau, a.top_k, a.top_p, tsum, r);
+    if (!ok2) ASX_COUNT(4);
+    return ok2;
 }
 
 template <int DT>
@@ -805,10 +808,14 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
         }
         if (!decided && want_tail && list_ok && !*(volatile int*)&sm.poisoned) {
             // the nucleus reaches below the exact depth of the list: lower the threshold once
+            ASX_COUNT(0);
             if (tid == 0) sm.b_i[2] = C;
             decided = deepen_nucleus<DT>(sm, a, row, gmax, t0f, tailsum, c, r);
         }
         if (!decided) {
+            ASX_COUNT(5);
+            if (nvh > SK_CAPV) ASX_COUNT(6);
+            if (sm.cand_count > SK_CAP) ASX_COUNT(7);
             if (!general_row) general_row = row;          // the row again, from global memory (L2)
             SyncC::sync();
             GenericLane<DT, NT, SyncC> gl(sm.u.gen, general_row, V, general_vec_ok);
