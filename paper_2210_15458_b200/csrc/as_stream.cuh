@@ -278,17 +278,16 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
 constexpr int DP_NB = 1024;
 constexpr float DP_BINS_PER_UNIT = 64.f;
 template <int DT>
-__device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, const StepArgs& a, const char* row, uint32_t gmax,
-                                            float t0f, double tailsum, double c, LaneResult& r) {
+__device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2, double inv_tau, double top_p,
+                                            const char* row, uint32_t gmax, float t0f, double tailsum, double c,
+                                            LaneResult& r) {
     using Tr = Traits<DT>;
     using P = Pass<DT>;
     constexpr int E = Tr::E;
     constexpr int NT = SK_NT;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int V = a.V;
     const int nvec_full = (V * Tr::BYTES) >> 4;           // whole 16-byte vectors
     const float lmaxf = Tr::value_f(gmax);
-    const float scale2 = a.scale2;
     const float y0 = (t0f - lmaxf) * scale2;
     float* hmass = reinterpret_cast<float*>(sm.u.ep.v.cvec);
     int* hcnt = reinterpret_cast<int*>(hmass + DP_NB);
@@ -323,7 +322,7 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, const StepArgs& a, c
     SyncC::sync();
     // ---- 2. lowest bin needed
     if (warp == 0) {
-        const double target = a.top_p * (list_mass + tailsum);
+        const double target = top_p * (list_mass + tailsum);
         const double need = (target - list_mass) * 1.002 + 1e-7 * target;
         constexpr int PER = DP_NB / 32;
         double m = 0.0;
@@ -380,7 +379,7 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, const StepArgs& a, c
     const int C = sm.cand_count;
     if (C <= 0 || C > SK_CAP || !(tsum == tsum) || !(tsum < 1e300)) { ASX_COUNT(3); return false; }
     const bool ok2 = epilogue_ranked<DT, NT, SyncC>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, depth_key, c,
-                                                    (double)lmaxf, a.inv_tau, a.top_k, a.top_p, tsum, r);
+                                                    (double)lmaxf, inv_tau, 0, top_p, tsum, r);
     if (!ok2) ASX_COUNT(4);
     return ok2;
 }
@@ -810,7 +809,7 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
             // the nucleus reaches below the exact depth of the list: lower the threshold once
             ASX_COUNT(0);
             if (tid == 0) sm.b_i[2] = C;
-            decided = deepen_nucleus<DT>(sm, a, row, gmax, t0f, tailsum, c, r);
+            decided = deepen_nucleus<DT>(sm, V, scale2, a.inv_tau, a.top_p, row, gmax, t0f, tailsum, c, r);
         }
         if (!decided) {
             ASX_COUNT(5);
