@@ -69,7 +69,6 @@ struct StreamSmem {
     double red_d[SK_NW];
     unsigned wmax[2][SK_NW];
     unsigned wsel[2][SK_NW];
-    unsigned wlive[SK_NW];   // each warp's latest bound for the current row (read without a barrier)
     double list_mass;    // epilogue: total mass of the ranked list (nucleus lanes)
     int vec_count;
     int cand_count;
@@ -469,33 +468,19 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
 
     // block step: max so far and (optionally) threshold from the subset maxima held in `acc`;
     // one barrier: the exchange slots are double-buffered between consecutive calls
-    // `pub` is one value per warp; the caller gets the max logit key and the min / max of `pub`.
-    auto exchange = [&](const typename P::Acc& acc, uint32_t pub, uint32_t& gmax, uint32_t& pmin, uint32_t& pmax) {
+    auto threshold = [&](const typename P::Acc& acc, uint32_t& gmax, uint32_t& t0key, bool want_sel) {
         uint32_t k0, k1;
         P::keys(acc, k0, k1);
         const uint32_t wm = warp_max_u(max(k0, k1));
+        const uint32_t ws = want_sel ? warp_select16(P::key16(k0), P::key16(k1), m_sel) : 0u;
         const int buf = thr_calls & 1;
         ++thr_calls;
-        if (lane == 0) { sm.wmax[buf][warp] = wm; sm.wsel[buf][warp] = pub; }
+        if (lane == 0) { sm.wmax[buf][warp] = wm; sm.wsel[buf][warp] = ws; }
         SyncC::sync();
-        gmax = 0; pmin = 0xFFFFFFFFu; pmax = 0;
+        gmax = 0;
+        uint32_t t16 = 0xFFFFFFFFu;
 #pragma unroll
-        for (int w = 0; w < SK_NW; ++w) {
-            gmax = max(gmax, sm.wmax[buf][w]);
-            pmin = min(pmin, sm.wsel[buf][w]);
-            pmax = max(pmax, sm.wsel[buf][w]);
-        }
-    };
-    auto my_select = [&](const typename P::Acc& acc) -> uint32_t {
-        uint32_t k0, k1;
-        P::keys(acc, k0, k1);
-        return warp_select16(P::key16(k0), P::key16(k1), m_sel);
-    };
-    auto threshold = [&](const typename P::Acc& acc, uint32_t& gmax, uint32_t& t0key, bool want_sel) {
-        const uint32_t ws = want_sel ? my_select(acc) : 0u;
-        if (lane == 0) sm.wlive[warp] = ws;
-        uint32_t t16, unused;
-        exchange(acc, ws, gmax, t16, unused);
+        for (int w = 0; w < SK_NW; ++w) { gmax = max(gmax, sm.wmax[buf][w]); t16 = min(t16, sm.wsel[buf][w]); }
         t0key = max(P::key_from16(t16), Tr::KEY_NINF);
     };
     // SK_VPT vectors of one thread against the threshold.  Per vector: one packed max (shared with
@@ -703,7 +688,7 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
             }
         } else {
             // ---- streamed: slice -> registers -> stage released; T0 at slices 0, 1, 2, 4, 8, ...
-            int refresh_at = 1, read_at = -1;
+            int refresh_at = 1;
 #ifdef ASX_PROFILE
             long long pw = 0, pl = 0, pt = 0, pc = 0, tt0;
 #define ASX_ACC(var) do { const long long tt1 = clock64(); var += tt1 - tt0; tt0 = tt1; } while (0)
@@ -724,26 +709,13 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
 #pragma unroll
                     for (int j = 0; j < SK_VPT; ++j) P::merge(acc, P::reduce(q[j]));
                 }
-                if (s == 0) {
-                    uint32_t gm;
-                    threshold(acc, gm, t0key, true);
+                if (s == 0 || s == refresh_at) {
+                    uint32_t gm, t0new;
+                    threshold(acc, gm, t0new, true);
+                    t0key = max(t0key, t0new);
                     t0f = Tr::value_f(t0key);
-                    ref = Tr::value_f(min(max(gm, Tr::KEY_NINF + 1), Tr::KEY_PINF - 1));
-                } else if (s == refresh_at) {
-                    // no barrier: publish this warp's bound now ...
-                    const uint32_t ws = my_select(acc);
-                    if (lane == 0) *(volatile unsigned*)&sm.wlive[warp] = ws;
-                    refresh_at <<= 1;
-                    read_at = s + 1;
-                } else if (s == read_at) {
-                    // ... and one slice later take the smallest of the latest published bounds: by
-                    // then the other warps have published too; an older entry is lower, hence
-                    // still a bound
-                    uint32_t t16 = 0xFFFFFFFFu;
-#pragma unroll
-                    for (int w = 0; w < SK_NW; ++w) t16 = min(t16, *(volatile unsigned*)&sm.wlive[w]);
-                    t0key = max(t0key, max(P::key_from16(t16), Tr::KEY_NINF));
-                    t0f = Tr::value_f(t0key);
+                    if (s == 0) ref = Tr::value_f(min(max(gm, Tr::KEY_NINF + 1), Tr::KEY_PINF - 1));
+                    if (s == refresh_at) refresh_at <<= 1;
                 }
                 ASX_ACC(pt);
                 slice_pass(q, s * SK_STAGE_VEC + tid, valid, s > 0, acc, t0f, ref, tail);
@@ -753,10 +725,8 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
             if (blockIdx.x == 0 && tid == 0) { g_asx_marks[24] = pw; g_asx_marks[25] = pl; g_asx_marks[26] = pt; g_asx_marks[27] = pc; }
 #endif
             if (tid == 0) P::merge(acc, P::reduce(qt));
-            // final max; warps may hold different thresholds: the list is complete from the largest up
-            uint32_t unused;
-            exchange(acc, t0key, gmax, unused, t0key);
-            t0f = Tr::value_f(t0key);
+            uint32_t t0unused;
+            threshold(acc, gmax, t0unused, false);   // final max (t0key keeps the value the hits were taken with)
             const bool bad = code_bad || gmax >= Tr::KEY_PINF || gmax <= Tr::KEY_NINF;
             if (bad) {
                 r = failed_lane(c_in, ST_NUMERIC);
@@ -772,8 +742,6 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
         if (list_ok) {
             for (int i = tid; i < nvh; i += NT) {
                 const uint4 q = sm.u.ep.v.cvec[i];
-                // most listed vectors came in under an earlier, lower threshold
-                if (!want_tail && !(P::part_max(P::reduce(q)) >= t0f)) continue;
                 const int base = sm.u.ep.cidx[i] * E;
                 float x[E];
                 P::floats(q, x);
