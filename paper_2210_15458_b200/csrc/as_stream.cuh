@@ -83,27 +83,20 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 
 // m-th largest (1-based) of the 64 16-bit keys held two per lane, by a search on the value, two
 // bits per step: the largest v with count(keys >= v) >= m (0 if fewer than m keys are positive).
-__device__ __forceinline__ uint32_t warp_select16(uint32_t a16, uint32_t b16, int m) {
-    if (m <= 6) {
-        // few steps: take the maximum m times, removing one occurrence each time
-        const int lane = threadIdx.x & 31;
-        uint32_t cur = 0;
-#pragma unroll 1
-        for (int it = 0; it < m; ++it) {
-            cur = warp_max_u(max(a16, b16));
-            const unsigned ba = __ballot_sync(FULL, a16 == cur);
-            if (ba) {
-                if (lane == __ffs(ba) - 1) a16 = 0;
-            } else {
-                const unsigned bb = __ballot_sync(FULL, b16 == cur);
-                if (lane == __ffs(bb) - 1) b16 = 0;
-            }
-        }
-        return cur;
+__device__ __forceinline__ uint32_t warp_select16(uint32_t a16, uint32_t b16, int m, uint32_t lo16 = 0) {
+    // Only an answer above lo16 (the threshold already in force) is of use, and it cannot exceed the
+    // warp's maximum: search the bits below their common prefix.  0 = no bound above lo16.
+    const uint32_t hi16 = warp_max_u(max(a16, b16));
+    if (hi16 <= lo16) return 0;
+    int nb = 32 - __clz(lo16 ^ hi16);            // differing low bits
+    nb = (nb + 1) & ~1;                          // two bits per step
+    uint32_t res = nb >= 16 ? 0u : (hi16 >> nb) << nb;
+    if (res) {
+        const int n0 = __popc(__ballot_sync(FULL, a16 >= res)) + __popc(__ballot_sync(FULL, b16 >= res));
+        if (n0 < m) return 0;                    // the m-th largest lies below the common prefix
     }
-    uint32_t res = 0;
 #pragma unroll 1
-    for (int bit = 14; bit >= 0; bit -= 2) {
+    for (int bit = nb - 2; bit >= 0; bit -= 2) {
         const uint32_t c1 = res | (1u << bit), c2 = res | (2u << bit), c3 = res | (3u << bit);
         const int n1 = __popc(__ballot_sync(FULL, a16 >= c1)) + __popc(__ballot_sync(FULL, b16 >= c1));
         const int n2 = __popc(__ballot_sync(FULL, a16 >= c2)) + __popc(__ballot_sync(FULL, b16 >= c2));
@@ -468,11 +461,11 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
 
     // block step: max so far and (optionally) threshold from the subset maxima held in `acc`;
     // one barrier: the exchange slots are double-buffered between consecutive calls
-    auto threshold = [&](const typename P::Acc& acc, uint32_t& gmax, uint32_t& t0key, bool want_sel) {
+    auto threshold = [&](const typename P::Acc& acc, uint32_t& gmax, uint32_t& t0key, bool want_sel, uint32_t lo_key) {
         uint32_t k0, k1;
         P::keys(acc, k0, k1);
         const uint32_t wm = warp_max_u(max(k0, k1));
-        const uint32_t ws = want_sel ? warp_select16(P::key16(k0), P::key16(k1), m_sel) : 0u;
+        const uint32_t ws = want_sel ? warp_select16(P::key16(k0), P::key16(k1), m_sel, P::key16(lo_key)) : 0u;
         const int buf = thr_calls & 1;
         ++thr_calls;
         if (lane == 0) { sm.wmax[buf][warp] = wm; sm.wsel[buf][warp] = ws; }
@@ -506,23 +499,27 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
             }
         }
         if (__any_sync(FULL, hm != 0)) {
+            // one slot reservation per warp and slice: ballots per vector position, then a single atomic
+            unsigned bal[SK_VPT];
+            int total = 0;
 #pragma unroll
             for (int j = 0; j < SK_VPT; ++j) {
-                const bool hit = (hm >> j) & 1u;
-                const unsigned bal = __ballot_sync(FULL, hit);
-                if (bal) {
-                    const int leader = __ffs(bal) - 1;
-                    int base = 0;
-                    if (lane == leader) base = atomicAdd(&sm.vec_count, __popc(bal));
-                    base = __shfl_sync(FULL, base, leader);
-                    if (hit) {
-                        const int slot = base + __popc(bal & ((1u << lane) - 1u));
-                        if (slot < SK_CAPV) {
-                            sm.u.ep.v.cvec[slot] = q[j];
-                            sm.u.ep.cidx[slot] = vec0 + j * NT;
-                        }
+                bal[j] = __ballot_sync(FULL, (hm >> j) & 1u);
+                total += __popc(bal[j]);
+            }
+            int base = 0;
+            if (lane == 0) base = atomicAdd(&sm.vec_count, total);
+            base = __shfl_sync(FULL, base, 0);
+#pragma unroll
+            for (int j = 0; j < SK_VPT; ++j) {
+                if ((hm >> j) & 1u) {
+                    const int slot = base + __popc(bal[j] & ((1u << lane) - 1u));
+                    if (slot < SK_CAPV) {
+                        sm.u.ep.v.cvec[slot] = q[j];
+                        sm.u.ep.cidx[slot] = vec0 + j * NT;
                     }
                 }
+                base += __popc(bal[j]);
             }
         }
     };
@@ -626,7 +623,7 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
             }
             if (tid == 0) P::merge(acc, P::reduce(qt));
             ASX_MARK(2);
-            threshold(acc, gmax, t0key, cut);
+            threshold(acc, gmax, t0key, cut, 0u);
             ASX_MARK(3);
             const bool bad = code_bad || gmax >= Tr::KEY_PINF || gmax <= Tr::KEY_NINF;
             if (bad) {
@@ -711,7 +708,7 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
                 }
                 if (s == 0 || s == refresh_at) {
                     uint32_t gm, t0new;
-                    threshold(acc, gm, t0new, true);
+                    threshold(acc, gm, t0new, true, t0key);
                     t0key = max(t0key, t0new);
                     t0f = Tr::value_f(t0key);
                     if (s == 0) ref = Tr::value_f(min(max(gm, Tr::KEY_NINF + 1), Tr::KEY_PINF - 1));
@@ -726,7 +723,7 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
 #endif
             if (tid == 0) P::merge(acc, P::reduce(qt));
             uint32_t t0unused;
-            threshold(acc, gmax, t0unused, false);   // final max (t0key keeps the value the hits were taken with)
+            threshold(acc, gmax, t0unused, false, 0u);   // final max (t0key keeps the value the hits were taken with)
             const bool bad = code_bad || gmax >= Tr::KEY_PINF || gmax <= Tr::KEY_NINF;
             if (bad) {
                 r = failed_lane(c_in, ST_NUMERIC);
@@ -742,6 +739,8 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
         if (list_ok) {
             for (int i = tid; i < nvh; i += NT) {
                 const uint4 q = sm.u.ep.v.cvec[i];
+                // most listed vectors came in under an earlier, lower threshold
+                if (!want_tail && !(P::part_max(P::reduce(q)) >= t0f)) continue;
                 const int base = sm.u.ep.cidx[i] * E;
                 float x[E];
                 P::floats(q, x);
