@@ -465,11 +465,20 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
         uint32_t k0, k1;
         P::keys(acc, k0, k1);
         const uint32_t wm = warp_max_u(max(k0, k1));
+#ifdef ASX_PROFILE
+        const long long tq0 = clock64();
+#endif
         const uint32_t ws = want_sel ? warp_select16(P::key16(k0), P::key16(k1), m_sel, P::key16(lo_key)) : 0u;
+#ifdef ASX_PROFILE
+        const long long tq1 = clock64();
+#endif
         const int buf = thr_calls & 1;
         ++thr_calls;
         if (lane == 0) { sm.wmax[buf][warp] = wm; sm.wsel[buf][warp] = ws; }
         SyncC::sync();
+#ifdef ASX_PROFILE
+        if (blockIdx.x == 0 && tid == 0) { g_asx_marks[28] += tq1 - tq0; g_asx_marks[29] += clock64() - tq1; g_asx_marks[30] += 1; }
+#endif
         gmax = 0;
         uint32_t t16 = 0xFFFFFFFFu;
 #pragma unroll

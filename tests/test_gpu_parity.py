@@ -422,3 +422,30 @@ def test_step_flat_and_adversarial_rows_fall_back(B, orc):
     check(B, orc, wide, F32, rng.random(6), 1.0, 0, 0.97, what="wide nucleus")
     check(B, orc, wide, F32, rng.random(6), 1.0, 5000, 1.0, what="large top-k")
     check(B, orc, wide, F32, rng.random(6), 1.0, 5000, 0.3, what="large top-k + nucleus")
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_step_nucleus_deeper_than_the_list(B, orc, dtype):
+    # nucleus-only lanes whose nucleus holds a few hundred tokens: more than the exact depth of the
+    # candidate list, so the threshold has to be lowered once from the mass histogram; plus lanes
+    # whose nucleus is far too large for any list (general routine)
+    rng = np.random.default_rng(800)
+    for V in (50000, 140000):
+        lanes = 24
+        x = rng.normal(-12.0, 1.0, (lanes, V)).astype(np.float32)
+        for i in range(lanes):
+            n_hi = 120 + 20 * i                                   # 120 .. 580 comparable heavy tokens
+            idx = rng.choice(V, n_hi, replace=False)
+            x[i, idx] = rng.normal(2.0, 0.6, n_hi).astype(np.float32)
+        arr = _store(x, dtype)
+        codes = rng.random(lanes)
+        d = {}
+        ref = orc.step(arr, dtype, codes, 1.0, 0, 0.9, threads=8)
+        tok, c2 = B.as_step(to_dev(arr, dtype), torch.from_numpy(codes).cuda(), 1.0, 0, 0.9, diag=d)
+        torch.cuda.synchronize()
+        r = compare_step(ref, tok.cpu().numpy(), c2.cpu().numpy(), d["p_tok"].cpu().numpy(),
+                         d["n_kept"].cpu().numpy(), d["lane_status"].cpu().numpy(), what="deep nucleus V=%d" % V)
+        assert r["compared"] >= lanes - 4
+        path = d["path"].cpu().numpy()
+        assert ref.n_kept.max() > 300
+        assert (path[ref.n_kept < 400] == B.PATH_COMPACT).sum() >= 8    # served without the general routine
