@@ -187,12 +187,16 @@ int as_decode_bigram_codes(const void *d_table, int dtype, int V, long long ld,
  *   AS_TUNE_CTAS_PER_SM   resident CTAs per SM the grid is sized for
  *   AS_TUNE_STAGES        16 KB ring stages of the streaming kernel for rows that do not
  *                         fit the ring (2..12)
+ *   AS_TUNE_MIN_CTAS      streaming kernel build for bf16 rows that do not fit the ring:
+ *                         3 = three CTAs per SM (1024-entry hit list, <= 72 registers; default),
+ *                         2 = two CTAs per SM (2048-entry hit list)
  * Returns AS_ERR_INVALID_ARG for an unknown key or value.
  */
 #define AS_TUNE_STEP_PATH 1
 #define AS_TUNE_CLUSTER 2
 #define AS_TUNE_CTAS_PER_SM 3
 #define AS_TUNE_STAGES 4
+#define AS_TUNE_MIN_CTAS 5
 int as_tune(int key, int value);
 
 /* Text of the calling thread's most recent error ("" if none). Never NULL. */

@@ -32,6 +32,7 @@ TUNE_STEP_PATH = 1
 TUNE_CLUSTER = 2
 TUNE_CTAS_PER_SM = 3
 TUNE_STAGES = 4
+TUNE_MIN_CTAS = 5
 
 EXPORTS = ["as_lattice_codes", "as_step", "as_step_host", "as_step_host_work_bytes", "as_decode_bigram",
            "as_decode_bigram_codes", "as_tune", "as_last_error", "as_version"]

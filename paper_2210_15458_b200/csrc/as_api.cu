@@ -13,7 +13,7 @@ namespace asx {
 // host-side state
 // ---------------------------------------------------------------------------
 static thread_local char g_err[512] = "";
-static int g_tune_path = 0, g_tune_cluster = 0, g_tune_ctas = 0, g_tune_stages = 0;
+static int g_tune_path = 0, g_tune_cluster = 0, g_tune_ctas = 0, g_tune_stages = 0, g_tune_minb = 0;
 
 static int set_err(int code, const char* fmt, ...) {
     va_list ap;
@@ -104,22 +104,21 @@ static int launch_staged(const StepArgs& a, size_t smem, int sms, int want_per_s
     return AS_OK;
 }
 
-static size_t stream_fixed_bytes() { return (sizeof(StreamSmem) + 127) & ~(size_t)127; }
-
-template <int DT>
+template <int DT, int CAPV, int MINB>
 static int launch_stream(const StepArgs& a, int stages, int sms, int want_per_sm, cudaStream_t st) {
     static bool attr_set[64] = {false};
     static int per_sm_cache[64][SK_MAXSTAGES + 1] = {{0}};
     int dev = 0;
     cudaGetDevice(&dev);
-    auto kern = step_stream_kernel<DT>;
+    auto kern = step_stream_kernel<DT, CAPV, MINB>;
     cudaError_t e;
     if (!attr_set[dev]) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_OPTIN_MAX - 1024));
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(max dynamic shared memory)");
         attr_set[dev] = true;
     }
-    const size_t smem = stream_fixed_bytes() + (size_t)stages * SK_STAGE_BYTES;
+    const size_t fixed = (sizeof(StreamSmemT<CAPV>) + 127) & ~(size_t)127;
+    const size_t smem = fixed + (size_t)stages * SK_STAGE_BYTES;
     if (per_sm_cache[dev][stages] == 0) {
         int n = 0;
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, SK_THREADS, smem);
@@ -291,6 +290,10 @@ int as_tune(int key, int value) {
             if (value < 0 || value > 32) return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_CTAS_PER_SM takes 0..32");
             g_tune_ctas = value;
             return AS_OK;
+        case AS_TUNE_MIN_CTAS:
+            if (value != 0 && value != 2 && value != 3) return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_MIN_CTAS takes 0, 2 or 3");
+            g_tune_minb = value;
+            return AS_OK;
         case AS_TUNE_STAGES:
             if (value < 0 || value == 1 || value > SK_MAXSTAGES) return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_STAGES takes 0 or 2..12");
             g_tune_stages = value;
@@ -345,8 +348,11 @@ int as_step(const void* d_logits, int dtype, int lanes, int V, long long ld, con
         if (resident || a.fast) {
             int stages = resident ? (nsl < 1 ? 1 : nsl) : (g_tune_stages > 0 ? g_tune_stages : 3);
             if (!resident && stages >= nsl) stages = nsl - 1;
-            return dtype == AS_F32 ? launch_stream<DT_F32>(a, stages, di->sms, g_tune_ctas, st)
-                                   : launch_stream<DT_BF16>(a, stages, di->sms, g_tune_ctas, st);
+            if (dtype == AS_F32) return launch_stream<DT_F32, 2048, 2>(a, stages, di->sms, g_tune_ctas, st);
+            // bf16 rows that stream: a 1024-entry hit list and <= 72 registers let three CTAs share an SM
+            if (!resident && g_tune_minb != 2)
+                return launch_stream<DT_BF16, 1024, 3>(a, stages < 3 ? stages : 3, di->sms, g_tune_ctas, st);
+            return launch_stream<DT_BF16, 2048, 2>(a, stages, di->sms, g_tune_ctas, st);
         }
     }
     if (g_tune_path == 2) {

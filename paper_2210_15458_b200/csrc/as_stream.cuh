@@ -35,7 +35,6 @@ namespace asx {
 constexpr int SK_NT = 256;                 // consumer threads
 constexpr int SK_NW = SK_NT / 32;          // consumer warps
 constexpr int SK_THREADS = SK_NT + 32;     // + producer warp
-constexpr int SK_CAPV = 2048;              // hit-vector capacity per lane
 constexpr int SK_CAP = 512;                // candidate (element) capacity per lane
 constexpr int SK_STAGE_VEC = 1024;         // 16-byte vectors per stage (16 KB)
 constexpr int SK_STAGE_BYTES = SK_STAGE_VEC * 16;
@@ -48,19 +47,21 @@ constexpr int SK_KP = 96;                  // K0 for nucleus-only lanes
 
 using SyncC = SyncNamed<SK_NT>;
 
-struct StreamSmem {
+// CAPV: hit-vector capacity per lane (1024 lets three CTAs share an SM; fp32 rows need 2048)
+template <int CAPV>
+struct StreamSmemT {
     unsigned long long full_bar[SK_MAXSTAGES];
     unsigned long long empty_bar[SK_MAXSTAGES];
     union {
         struct {
             union {
-                uint4 cvec[SK_CAPV];                       // hit vectors (dead once extracted)
+                uint4 cvec[CAPV];                       // hit vectors (dead once extracted)
                 struct {
                     unsigned long long srt[SK_CAP + 4];    // candidates by rank
                     double e[SK_CAP];                      // mass by rank
                 } rk;
             } v;
-            int cidx[SK_CAPV];                             // vector index of each hit vector
+            int cidx[CAPV];                             // vector index of each hit vector
             unsigned long long cand[SK_CAP + 4];           // (key << 32) | ~index, any order
         } ep;
         GenericSmem<SK_NT> gen;
@@ -109,7 +110,7 @@ __device__ __forceinline__ uint32_t warp_select16(uint32_t a16, uint32_t b16, in
 // Exact decode on a candidate list src[0..C) (composites, any order); dst is scratch of C + 4
 // entries.  depth_key: every element of the row with key >= depth_key is in the list, so ranks
 // are exact down to that key.  Returns false if the list cannot decide the lane.
-template <int DT, int NT, class Sync>
+template <int DT, int NT, class Sync, class StreamSmem>
 __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long* src, unsigned long long* dst,
                                              double* e, int C, uint32_t depth_key, double c, double lmax,
                                              double inv_tau, int top_k, double top_p, double tail,
@@ -270,7 +271,7 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
 //      runs again.  Returns false if the window or the list capacity does not suffice.
 constexpr int DP_NB = 1024;
 constexpr float DP_BINS_PER_UNIT = 64.f;
-template <int DT>
+template <int DT, class StreamSmem>
 __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2, double inv_tau, double top_p,
                                             const char* row, uint32_t gmax, float t0f, double tailsum, double c,
                                             LaneResult& r) {
@@ -371,14 +372,16 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2,
     for (int w = 0; w < SK_NW; ++w) tsum += sm.red_d[w];
     const int C = sm.cand_count;
     if (C <= 0 || C > SK_CAP || !(tsum == tsum) || !(tsum < 1e300)) { ASX_COUNT(3); return false; }
-    const bool ok2 = epilogue_ranked<DT, NT, SyncC>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, depth_key, c,
+    const bool ok2 = epilogue_ranked<DT, NT, SyncC, StreamSmem>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, depth_key, c,
                                                     (double)lmaxf, inv_tau, 0, top_p, tsum, r);
     if (!ok2) ASX_COUNT(4);
     return ok2;
 }
 
-template <int DT>
-__global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepArgs a, const int stages) {
+template <int DT, int CAPV, int MINB>
+__global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const StepArgs a, const int stages) {
+    using StreamSmem = StreamSmemT<CAPV>;
+    constexpr int SK_CAPV = CAPV;
     using Tr = Traits<DT>;
     using P = Pass<DT>;
     constexpr int NT = SK_NT;
@@ -810,14 +813,14 @@ __global__ void __launch_bounds__(SK_THREADS, 2) step_stream_kernel(const StepAr
             r = failed_lane(c_in, ST_TIMEOUT);
             decided = true;
         } else if (list_ok && (!want_tail || (tailsum == tailsum && tailsum < 1e300))) {
-            decided = epilogue_ranked<DT, NT, SyncC>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, t0key, c,
+            decided = epilogue_ranked<DT, NT, SyncC, StreamSmem>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, t0key, c,
                                                      lmax, a.inv_tau, a.top_k, a.top_p, tailsum, r);
         }
         if (!decided && want_tail && list_ok && !*(volatile int*)&sm.poisoned) {
             // the nucleus reaches below the exact depth of the list: lower the threshold once
             ASX_COUNT(0);
             if (tid == 0) sm.b_i[2] = C;
-            decided = deepen_nucleus<DT>(sm, V, scale2, a.inv_tau, a.top_p, row, gmax, t0f, tailsum, c, r);
+            decided = deepen_nucleus<DT, StreamSmem>(sm, V, scale2, a.inv_tau, a.top_p, row, gmax, t0f, tailsum, c, r);
         }
         if (!decided) {
             ASX_COUNT(5);
