@@ -348,7 +348,11 @@ int as_step(const void* d_logits, int dtype, int lanes, int V, long long ld, con
         if (resident || a.fast) {
             int stages = resident ? (nsl < 1 ? 1 : nsl) : (g_tune_stages > 0 ? g_tune_stages : 3);
             if (!resident && stages >= nsl) stages = nsl - 1;
-            if (dtype == AS_F32) return launch_stream<DT_F32, 2048, 2>(a, stages, di->sms, g_tune_ctas, st);
+            if (dtype == AS_F32) {
+                if (!resident && g_tune_minb != 2)
+                    return launch_stream<DT_F32, 1536, 3>(a, stages < 2 ? stages : 2, di->sms, g_tune_ctas, st);
+                return launch_stream<DT_F32, 2048, 2>(a, stages, di->sms, g_tune_ctas, st);
+            }
             // bf16 rows that stream: a 1024-entry hit list and <= 72 registers let three CTAs share an SM
             if (!resident && g_tune_minb != 2)
                 return launch_stream<DT_BF16, 1024, 3>(a, stages < 3 ? stages : 3, di->sms, g_tune_ctas, st);
