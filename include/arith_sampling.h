@@ -139,6 +139,36 @@ int as_step_host(const void *h_logits, int dtype, int lanes, int V, long long ld
 size_t as_step_host_work_bytes(int dtype, int lanes, long long ld);
 
 /*
+ * as_step_host without any allocation, for callers that cannot provide device memory.
+ * (The paper has no counterpart to this call: it is a packaging of as_step_host.)
+ *
+ * Who needs it: code that is handed a stream but owns no device memory and may not ask for any --
+ * a plug-in running inside a serving runtime that keeps the whole GPU in its own fixed pool, or a
+ * call site where cudaMalloc's implicit device-wide synchronisation would stall other streams.
+ * as_step_host needs a device work buffer (d_work) for the copied logits, codes and results; this
+ * variant uses a buffer built into the library instead: AS_STATIC_WORK_BYTES of device memory that
+ * every GPU which loads the library holds until the process exits.
+ *
+ * Arguments and results are those of as_step_host, minus d_work / work_bytes.  It calls no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *   - A request whose as_step_host_work_bytes(dtype, lanes, ld) exceeds AS_STATIC_WORK_BYTES is
+ *     refused with AS_ERR_UNSUPPORTED (as_last_error() names both sizes); nothing is enqueued.
+ *   - The first call on each device looks up the buffer's device address (one-time set-up with
+ *     that device current); make that first call before any stream capture.
+ *   - All calls on a device share the one buffer.  Nothing in it has to start at zero: every byte
+ *     the step reads is written by this call's own copies first, and every result the host
+ *     receives is written by this call's kernel.  Two calls that overlap on the GPU (different
+ *     streams, or two host threads) race on the buffer: serialise them.  The call returns after
+ *     its results have reached the host buffers (it synchronises `stream`), so back-to-back calls
+ *     from one thread are safe.
+ */
+#define AS_STATIC_WORK_BYTES (24u << 20)
+int as_step_host_static(const void *h_logits, int dtype, int lanes, int V, long long ld,
+                        const double *h_codes, double temp, int top_k, double top_p,
+                        int32_t *h_tokens, double *h_codes_out, int32_t *h_lane_status,
+                        void *stream);
+
+/*
  * Full decode loop of Algorithm 1 (REPEAT ... UNTIL X = EOS) over a bigram
  * model: row table[prev] holds the next-token logits given the previous token.
  * The code set is the shifted lattice of as_lattice_codes, one copy per start

@@ -34,7 +34,8 @@ TUNE_CTAS_PER_SM = 3
 TUNE_STAGES = 4
 TUNE_MIN_CTAS = 5
 
-EXPORTS = ["as_lattice_codes", "as_step", "as_step_host", "as_step_host_work_bytes", "as_decode_bigram",
+EXPORTS = ["as_lattice_codes", "as_step", "as_step_host", "as_step_host_work_bytes", "as_step_host_static",
+           "as_decode_bigram",
            "as_decode_bigram_codes", "as_tune", "as_last_error", "as_version"]
 
 
@@ -70,6 +71,8 @@ def lib():
         L.as_lattice_codes.argtypes = [I, D, P, P]
         L.as_step.argtypes = [P, I, I, I, LL, P, D, I, D, P, P, ctypes.POINTER(as_step_diag), P]
         L.as_step_host.argtypes = [P, I, I, I, LL, P, D, I, D, P, P, P, P, ctypes.c_size_t, P]
+        L.as_step_host_static.argtypes = [P, I, I, I, LL, P, D, I, D, P, P, P, P]
+        L.as_step_host_static.restype = I
         L.as_step_host_work_bytes.argtypes = [I, I, LL]
         L.as_step_host_work_bytes.restype = ctypes.c_size_t
         L.as_decode_bigram.argtypes = [P, I, I, LL, P, I, I, D, I, I, D, I, D, P, P, P, P, P]
@@ -170,6 +173,24 @@ def as_step_host(h_logits: torch.Tensor, h_codes: torch.Tensor, temp: float, top
     _check(lib().as_step_host(_ptr(h_logits), _logits_dtype(h_logits), lanes, V, ld, _ptr(h_codes), temp,
                               top_k, top_p, _ptr(h_tokens), _ptr(h_codes_out), _ptr(h_lane_status),
                               _ptr(d_work), d_work.numel() * d_work.element_size(), _stream(stream)))
+
+
+STATIC_WORK_BYTES = 24 << 20
+
+
+def as_step_host_static(h_logits: torch.Tensor, h_codes: torch.Tensor, temp: float, top_k: int, top_p: float,
+                        h_tokens: torch.Tensor, h_codes_out: torch.Tensor, h_lane_status: Optional[torch.Tensor],
+                        V: Optional[int] = None, stream=None) -> None:
+    """as_step_host for callers that own no device memory: the device work space is a buffer
+    built into the library (STATIC_WORK_BYTES).  Every tensor here is a CPU tensor; nothing is
+    allocated on the device, neither by the library nor by this wrapper.  Steps that need more
+    work space than the buffer holds raise AsError(ERR_UNSUPPORTED).  Calls share the buffer, so
+    do not let two of them overlap on the GPU."""
+    lanes, width, ld = _logits_layout(h_logits)
+    V = width if V is None else V
+    _check(lib().as_step_host_static(_ptr(h_logits), _logits_dtype(h_logits), lanes, V, ld, _ptr(h_codes), temp,
+                                     top_k, top_p, _ptr(h_tokens), _ptr(h_codes_out), _ptr(h_lane_status),
+                                     _stream(stream)))
 
 
 def as_decode_bigram(table: torch.Tensor, start_tokens: torch.Tensor, N: int, u: float, T: int, eos: int,

@@ -425,6 +425,51 @@ int as_step_host(const void* h_logits, int dtype, int lanes, int V, long long ld
     return AS_OK;
 }
 
+// ---------------------------------------------------------------------------
+// as_step_host_static: the work buffer lives in the library
+// ---------------------------------------------------------------------------
+// Device memory reserved at load time on every GPU that loads this library.  In host code the
+// name below is only a handle for the runtime, not a device address: the address a kernel or a
+// copy can use comes from cudaGetSymbolAddress, looked up once per device.
+static __device__ __align__(256) unsigned char g_static_work[AS_STATIC_WORK_BYTES];
+static void* g_static_work_addr[64] = {nullptr};
+
+static int static_work_address(void** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= 64) return set_err(AS_ERR_CUDA, "device ordinal %d out of range", dev);
+    if (!g_static_work_addr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_work);      // this device is current
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(static work buffer)");
+        if (!p) return set_err(AS_ERR_CUDA, "static work buffer has no device address");
+        g_static_work_addr[dev] = p;
+    }
+    *out = g_static_work_addr[dev];
+    return AS_OK;
+}
+
+int as_step_host_static(const void* h_logits, int dtype, int lanes, int V, long long ld, const double* h_codes,
+                        double temp, int top_k, double top_p, int32_t* h_tokens, double* h_codes_out,
+                        int32_t* h_lane_status, void* stream) {
+    if (lanes < 0) return set_err(AS_ERR_INVALID_ARG, "lanes = %d must be >= 0", lanes);
+    int rc = check_scalars(dtype, V, ld, temp, top_p);
+    if (rc != AS_OK) return rc;
+    if (lanes == 0) return AS_OK;
+    const size_t need = as_step_host_work_bytes(dtype, lanes, ld);
+    if (need == 0 || need > (size_t)AS_STATIC_WORK_BYTES)
+        return set_err(AS_ERR_UNSUPPORTED,
+                       "this step needs %zu bytes of device work space, the built-in buffer holds %zu "
+                       "(AS_STATIC_WORK_BYTES): use as_step_host with your own buffer, or fewer lanes per call",
+                       need, (size_t)AS_STATIC_WORK_BYTES);
+    void* work = nullptr;
+    rc = static_work_address(&work);
+    if (rc != AS_OK) return rc;
+    return as_step_host(h_logits, dtype, lanes, V, ld, h_codes, temp, top_k, top_p, h_tokens, h_codes_out,
+                        h_lane_status, work, (size_t)AS_STATIC_WORK_BYTES, stream);
+}
+
 static int decode_common(const void* d_table, int dtype, int V, long long ld, const int32_t* d_tok,
                          const double* d_codes_in, int lanes, int N, double u, int T, int eos,
                          double temp, int top_k, double top_p, int32_t* d_seq, int32_t* d_len,
