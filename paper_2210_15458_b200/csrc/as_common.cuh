@@ -194,6 +194,126 @@ __device__ __forceinline__ int warp_suffix_i(int v, int lane) {
     return v;
 }
 
+// ---------------------------------------------------------------------------
+// 2^(t/64) for t <= 0 in fp64, t given in units of 1/64 (t = (x - max)/temp * 64 log2 e):
+// t = 64 n + j + f, |f| <= 1/2;  2^(t/64) = 2^n * 2^(j/64) * exp(f ln2/64), the last factor by a
+// degree-5 polynomial (truncation ~3e-17).  One fused multiply-add upstream forms t, so the
+// whole evaluation is 10 fp64 operations.  Arguments below -64000 (2^-1000) return 0.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ double exp2_64th(double t, const double* __restrict__ tbl) {
+    if (!(t >= -64000.0)) return 0.0;
+    const double MAGIC = 6755399441055744.0;
+    double r = t + MAGIC;
+    const int k = __double2loint(r);
+    r -= MAGIC;
+    const double f = t - r;
+    const double L = 0x1.62e42fefa39efp-7;               // ln2 / 64
+    double p = fma(f, L * L * L * L * L / 120.0, L * L * L * L / 24.0);
+    p = fma(p, f, L * L * L / 6.0);
+    p = fma(p, f, L * L / 2.0);
+    p = fma(p, f, L);
+    p = fma(p, f, 1.0);
+    const double v = tbl[k & 63] * p;
+    const int n = k >> 6;
+    return __hiloint2double(__double2hiint(v) + (n << 20), __double2loint(v));
+}
+
+// ---------------------------------------------------------------------------
+// Packed NaN-propagating maxima and float views of one 16-byte vector.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t max_nan_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ float max_nan_f32(float a, float b) {
+    float d;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+__device__ __forceinline__ float ex2_approx(float y) {
+    float d;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(d) : "f"(y));
+    return d;
+}
+
+template <int DT> struct Pass;
+template <> struct Pass<DT_BF16> {
+    // running NaN-propagating max, two bf16 lanes packed in one register
+    struct Acc { uint32_t m; };
+    __device__ static Acc init() { return Acc{0xFF80FF80u}; }            // (-inf, -inf)
+    __device__ static void fold(Acc& a, const uint4& q) {
+        a.m = max_nan_bf16x2(a.m, max_nan_bf16x2(max_nan_bf16x2(q.x, q.y), max_nan_bf16x2(q.z, q.w)));
+    }
+    // NaN-propagating max of one vector, kept packed; merged into the running max and
+    // reused for the "any element >= threshold" test
+    __device__ static Acc reduce(const uint4& q) {
+        return Acc{max_nan_bf16x2(max_nan_bf16x2(q.x, q.y), max_nan_bf16x2(q.z, q.w))};
+    }
+    __device__ static void merge(Acc& a, const Acc& b) { a.m = max_nan_bf16x2(a.m, b.m); }
+    __device__ static void fold_scalar(Acc& a, const void* row, long long j) {
+        const uint32_t b = reinterpret_cast<const uint16_t*>(row)[j];
+        a.m = max_nan_bf16x2(a.m, b | (b << 16));
+    }
+    __device__ static float load_f(const void* row, long long j) {
+        return __uint_as_float((uint32_t)reinterpret_cast<const uint16_t*>(row)[j] << 16);
+    }
+    __device__ static float part_max(const Acc& b) {
+        return fmaxf(__uint_as_float(b.m << 16), __uint_as_float(b.m & 0xFFFF0000u));
+    }
+    __device__ static void keys(const Acc& a, uint32_t& k0, uint32_t& k1) {
+        k0 = Traits<DT_BF16>::key_of(a.m & 0xFFFFu);
+        k1 = Traits<DT_BF16>::key_of(a.m >> 16);
+    }
+    __device__ static uint32_t key16(uint32_t key) { return key; }
+    __device__ static uint32_t key_from16(uint32_t k16) { return k16; }
+    __device__ static void floats(const uint4& q, float (&x)[8]) {
+        x[0] = __uint_as_float(q.x << 16); x[1] = __uint_as_float(q.x & 0xFFFF0000u);
+        x[2] = __uint_as_float(q.y << 16); x[3] = __uint_as_float(q.y & 0xFFFF0000u);
+        x[4] = __uint_as_float(q.z << 16); x[5] = __uint_as_float(q.z & 0xFFFF0000u);
+        x[6] = __uint_as_float(q.w << 16); x[7] = __uint_as_float(q.w & 0xFFFF0000u);
+    }
+    // max of the 8 elements (no NaN present any more)
+    __device__ static float vmax(const uint4& q) {
+        const uint32_t m = max_nan_bf16x2(max_nan_bf16x2(q.x, q.y), max_nan_bf16x2(q.z, q.w));
+        return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+    }
+    __device__ static uint32_t key_of_f(float x) { return Traits<DT_BF16>::key_of(__float_as_uint(x) >> 16); }
+};
+template <> struct Pass<DT_F32> {
+    struct Acc { float a, b; };
+    __device__ static Acc init() { return Acc{__uint_as_float(0xFF800000u), __uint_as_float(0xFF800000u)}; }
+    __device__ static void fold(Acc& s, const uint4& q) {
+        s.a = max_nan_f32(s.a, max_nan_f32(__uint_as_float(q.x), __uint_as_float(q.z)));
+        s.b = max_nan_f32(s.b, max_nan_f32(__uint_as_float(q.y), __uint_as_float(q.w)));
+    }
+    __device__ static Acc reduce(const uint4& q) {
+        return Acc{max_nan_f32(__uint_as_float(q.x), __uint_as_float(q.z)),
+                   max_nan_f32(__uint_as_float(q.y), __uint_as_float(q.w))};
+    }
+    __device__ static void merge(Acc& s, const Acc& b) { s.a = max_nan_f32(s.a, b.a); s.b = max_nan_f32(s.b, b.b); }
+    __device__ static void fold_scalar(Acc& s, const void* row, long long j) {
+        s.a = max_nan_f32(s.a, reinterpret_cast<const float*>(row)[j]);
+    }
+    __device__ static float load_f(const void* row, long long j) { return reinterpret_cast<const float*>(row)[j]; }
+    __device__ static float part_max(const Acc& b) { return fmaxf(b.a, b.b); }
+    __device__ static void keys(const Acc& s, uint32_t& k0, uint32_t& k1) {
+        k0 = Traits<DT_F32>::key_of(__float_as_uint(s.a));
+        k1 = Traits<DT_F32>::key_of(__float_as_uint(s.b));
+    }
+    __device__ static uint32_t key16(uint32_t key) { return key >> 16; }
+    __device__ static uint32_t key_from16(uint32_t k16) { return k16 << 16; }   // rounds the bound down
+    __device__ static void floats(const uint4& q, float (&x)[4]) {
+        x[0] = __uint_as_float(q.x); x[1] = __uint_as_float(q.y);
+        x[2] = __uint_as_float(q.z); x[3] = __uint_as_float(q.w);
+    }
+    __device__ static float vmax(const uint4& q) {
+        return fmaxf(fmaxf(__uint_as_float(q.x), __uint_as_float(q.y)),
+                     fmaxf(__uint_as_float(q.z), __uint_as_float(q.w)));
+    }
+    __device__ static uint32_t key_of_f(float x) { return Traits<DT_F32>::key_of(__float_as_uint(x)); }
+};
+
 // Result of one decode step for one lane, identical in every thread of the CTA.
 struct LaneResult {
     int token;

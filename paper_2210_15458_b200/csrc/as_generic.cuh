@@ -293,7 +293,158 @@ struct GenericLane {
         return r;
     }
 
+    // ------------------------------------------------------------------ no cut: every finite token kept
+    // Lean version of the same steps for lanes without top-k / nucleus on 16-byte aligned rows:
+    // a packed NaN-propagating max pass, then masses straight from the float values.
+    __device__ __forceinline__ void chunk_floats(int ci, int r, float (&x)[E], int& base) const {
+        using P = Pass<DT>;
+        const int vi = (ci * R + r) * 32 + lane;
+        base = vi * E;
+        if (vi < nvec && base + E <= V) {
+            const uint4 q = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row) + (size_t)base * Tr::BYTES);
+            P::floats(q, x);
+        } else {
+#pragma unroll
+            for (int e = 0; e < E; ++e)
+                x[e] = (vi < nvec && base + e < V) ? P::load_f(row, base + e) : __uint_as_float(0xFF800000u);
+        }
+    }
+
+    __device__ __noinline__ LaneResult run_nocut(double c_in, double inv_tau_) {
+        using P = Pass<DT>;
+        inv_tau = inv_tau_;
+        fill_exp_table(sm.exp_tbl, tid);
+        double c = c_in;
+        const bool code_bad = !(c >= 0.0 && c <= 1.0);
+        if (c == 1.0) c = ASX_ONE_BELOW;
+        // ---- 1. maximum (NaN and +inf propagate into it)
+        typename P::Acc acc = P::init();
+        const int nvf = (V * Tr::BYTES) >> 4;
+        for (int vi = tid; vi < nvf; vi += NT)
+            P::merge(acc, P::reduce(*reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row) + (size_t)vi * 16)));
+        for (int j = nvf * E + tid; j < V; j += NT) P::fold_scalar(acc, row, j);
+        uint32_t k0, k1;
+        P::keys(acc, k0, k1);
+        uint32_t kmax = warp_max_u(max(k0, k1));
+        if (lane == 0) sm.red_u[warp] = kmax;
+        if (tid == 0) sm.b_i[2] = 0;
+        Sync::sync();
+        kmax = 0;
+        for (int w = 0; w < NW; ++w) kmax = max(kmax, sm.red_u[w]);
+        if (code_bad || kmax >= Tr::KEY_PINF || kmax <= Tr::KEY_NINF) {
+            Sync::sync();
+            return fail(c_in, ST_NUMERIC);
+        }
+        lmax = (double)Tr::value_f(kmax);
+        const double s64 = inv_tau * 0x1.71547652b82fep+6;          // 64 log2(e) / temp
+        const double c64 = -lmax * s64;
+        // ---- 2. per-chunk masses in index order
+        int nfin = 0;
+        for (int ci = warp; ci < nchunks; ci += NW) {
+            double local = 0.0;
+            for (int r = 0; r < R; ++r) {
+                float x[E];
+                int base;
+                chunk_floats(ci, r, x, base);
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    local += exp2_64th(fma((double)x[e], s64, c64), sm.exp_tbl);
+                    nfin += (x[e] > __uint_as_float(0xFF800000u));
+                }
+            }
+            local = warp_sum_d(local);
+            if (lane == 0) sm.chunk_sum[ci] = local;
+        }
+        nfin = warp_sum_i(nfin);
+        if (lane == 0) atomicAdd(&sm.b_i[2], nfin);
+        Sync::sync();
+        scan_exclusive(sm.chunk_sum, nchunks);
+        // ---- 3. the chunk, then the element, whose interval holds c * Z
+        const double Z = sm.chunk_sum[nchunks];
+        const double t = c * Z;
+        const int n_kept = sm.b_i[2];
+        if (tid == 0) { sm.b_i[0] = INT_MAX; sm.b_i[1] = -1; }
+        Sync::sync();
+        for (int ci = tid; ci < nchunks; ci += NT) {
+            const double excl = sm.chunk_sum[ci], incl = sm.chunk_sum[ci + 1];
+            if (incl > excl) {
+                atomicMax(&sm.b_i[1], ci);
+                if (t < incl) atomicMin(&sm.b_i[0], ci);
+            }
+        }
+        Sync::sync();
+        const bool force_last = (sm.b_i[0] == INT_MAX);
+        const int cstar = force_last ? sm.b_i[1] : sm.b_i[0];
+        if (warp == 0) {
+            double run = sm.chunk_sum[cstar];
+            int last_idx = -1;
+            double last_S = 0.0, last_e = 1.0;
+            int tok = -1;
+            double tok_S = 0.0, tok_e = 1.0;
+            for (int r = 0; r < R && tok < 0; ++r) {
+                float x[E];
+                int base;
+                chunk_floats(cstar, r, x, base);
+                double ev[E];
+                double local = 0.0;
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    ev[e] = exp2_64th(fma((double)x[e], s64, c64), sm.exp_tbl);
+                    local += ev[e];
+                }
+                const double incl = warp_incl_scan_d(local, lane);
+                double excl = __shfl_up_sync(FULL, incl, 1);
+                if (lane == 0) excl = 0.0;
+                int pick = -1;
+                double pick_S = 0.0, pick_e = 1.0;
+                double S = run + excl;
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    if (ev[e] > 0.0) {
+                        if (pick < 0 && t < S + ev[e]) { pick = base + e; pick_S = S; pick_e = ev[e]; }
+                        last_idx = base + e; last_S = S; last_e = ev[e];
+                        S += ev[e];
+                    }
+                }
+                const bool cross = !force_last && local > 0.0 && (t < run + incl);
+                const unsigned bal = __ballot_sync(FULL, cross);
+                if (bal) {
+                    const int L = __ffs(bal) - 1;
+                    if (pick < 0) { pick = last_idx; pick_S = last_S; pick_e = last_e; }
+                    tok = __shfl_sync(FULL, pick, L);
+                    tok_S = __shfl_sync(FULL, pick_S, L);
+                    tok_e = __shfl_sync(FULL, pick_e, L);
+                }
+                run += __shfl_sync(FULL, incl, 31);
+            }
+            if (tok < 0) {   // rounding at the top end: the last token with mass in the chunk
+                const unsigned best = warp_max_u((unsigned)(last_idx + 1));
+                const unsigned bal = __ballot_sync(FULL, (unsigned)(last_idx + 1) == best);
+                const int L = __ffs(bal) - 1;
+                tok = __shfl_sync(FULL, last_idx, L);
+                tok_S = __shfl_sync(FULL, last_S, L);
+                tok_e = __shfl_sync(FULL, last_e, L);
+            }
+            if (lane == 0) {
+                double cn = (t - tok_S) / tok_e;
+                if (!(cn >= 0.0)) cn = 0.0;
+                if (cn > ASX_ONE_BELOW) cn = ASX_ONE_BELOW;
+                LaneResult r;
+                r.token = tok; r.status = tok < 0 ? ST_NUMERIC : ST_OK; r.n_kept = n_kept;
+                r.code_out = tok < 0 ? c_in : cn;
+                r.p_tok = tok_e / Z;
+                r.cdf_lo = tok_S / Z;
+                sm.res = r;
+            }
+        }
+        Sync::sync();
+        const LaneResult out = sm.res;
+        Sync::sync();
+        return out;
+    }
+
     __device__ __noinline__ LaneResult run(double c_in, double inv_tau_, int top_k, double top_p) {
+        if (top_k <= 0 && !(top_p > 0.0 && top_p < 1.0) && vec_ok) return run_nocut(c_in, inv_tau_);
         inv_tau = inv_tau_;
         fill_exp_table(sm.exp_tbl, tid);
         double c = c_in;

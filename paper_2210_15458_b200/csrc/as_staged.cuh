@@ -111,22 +111,6 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
         if (clock64() - t0 > ST_WAIT_CYCLES) return false;
     }
 }
-__device__ __forceinline__ uint32_t max_nan_bf16x2(uint32_t a, uint32_t b) {
-    uint32_t d;
-    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-    return d;
-}
-__device__ __forceinline__ float max_nan_f32(float a, float b) {
-    float d;
-    asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
-    return d;
-}
-__device__ __forceinline__ float ex2_approx(float y) {
-    float d;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(d) : "f"(y));
-    return d;
-}
-
 // ---------------------------------------------------------------------------
 // shared memory
 // ---------------------------------------------------------------------------
@@ -157,72 +141,6 @@ struct StagedSmem {
     int cand_count;
     int b_i[4];
     LaneResult res;
-};
-
-template <int DT> struct Pass;
-template <> struct Pass<DT_BF16> {
-    // running NaN-propagating max, two bf16 lanes packed in one register
-    struct Acc { uint32_t m; };
-    __device__ static Acc init() { return Acc{0xFF80FF80u}; }            // (-inf, -inf)
-    __device__ static void fold(Acc& a, const uint4& q) {
-        a.m = max_nan_bf16x2(a.m, max_nan_bf16x2(max_nan_bf16x2(q.x, q.y), max_nan_bf16x2(q.z, q.w)));
-    }
-    // NaN-propagating max of one vector, kept packed; merged into the running max and
-    // reused for the "any element >= threshold" test
-    __device__ static Acc reduce(const uint4& q) {
-        return Acc{max_nan_bf16x2(max_nan_bf16x2(q.x, q.y), max_nan_bf16x2(q.z, q.w))};
-    }
-    __device__ static void merge(Acc& a, const Acc& b) { a.m = max_nan_bf16x2(a.m, b.m); }
-    __device__ static float part_max(const Acc& b) {
-        return fmaxf(__uint_as_float(b.m << 16), __uint_as_float(b.m & 0xFFFF0000u));
-    }
-    __device__ static void keys(const Acc& a, uint32_t& k0, uint32_t& k1) {
-        k0 = Traits<DT_BF16>::key_of(a.m & 0xFFFFu);
-        k1 = Traits<DT_BF16>::key_of(a.m >> 16);
-    }
-    __device__ static uint32_t key16(uint32_t key) { return key; }
-    __device__ static uint32_t key_from16(uint32_t k16) { return k16; }
-    __device__ static void floats(const uint4& q, float (&x)[8]) {
-        x[0] = __uint_as_float(q.x << 16); x[1] = __uint_as_float(q.x & 0xFFFF0000u);
-        x[2] = __uint_as_float(q.y << 16); x[3] = __uint_as_float(q.y & 0xFFFF0000u);
-        x[4] = __uint_as_float(q.z << 16); x[5] = __uint_as_float(q.z & 0xFFFF0000u);
-        x[6] = __uint_as_float(q.w << 16); x[7] = __uint_as_float(q.w & 0xFFFF0000u);
-    }
-    // max of the 8 elements (no NaN present any more)
-    __device__ static float vmax(const uint4& q) {
-        const uint32_t m = max_nan_bf16x2(max_nan_bf16x2(q.x, q.y), max_nan_bf16x2(q.z, q.w));
-        return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
-    }
-    __device__ static uint32_t key_of_f(float x) { return Traits<DT_BF16>::key_of(__float_as_uint(x) >> 16); }
-};
-template <> struct Pass<DT_F32> {
-    struct Acc { float a, b; };
-    __device__ static Acc init() { return Acc{__uint_as_float(0xFF800000u), __uint_as_float(0xFF800000u)}; }
-    __device__ static void fold(Acc& s, const uint4& q) {
-        s.a = max_nan_f32(s.a, max_nan_f32(__uint_as_float(q.x), __uint_as_float(q.z)));
-        s.b = max_nan_f32(s.b, max_nan_f32(__uint_as_float(q.y), __uint_as_float(q.w)));
-    }
-    __device__ static Acc reduce(const uint4& q) {
-        return Acc{max_nan_f32(__uint_as_float(q.x), __uint_as_float(q.z)),
-                   max_nan_f32(__uint_as_float(q.y), __uint_as_float(q.w))};
-    }
-    __device__ static void merge(Acc& s, const Acc& b) { s.a = max_nan_f32(s.a, b.a); s.b = max_nan_f32(s.b, b.b); }
-    __device__ static float part_max(const Acc& b) { return fmaxf(b.a, b.b); }
-    __device__ static void keys(const Acc& s, uint32_t& k0, uint32_t& k1) {
-        k0 = Traits<DT_F32>::key_of(__float_as_uint(s.a));
-        k1 = Traits<DT_F32>::key_of(__float_as_uint(s.b));
-    }
-    __device__ static uint32_t key16(uint32_t key) { return key >> 16; }
-    __device__ static uint32_t key_from16(uint32_t k16) { return k16 << 16; }   // rounds the bound down
-    __device__ static void floats(const uint4& q, float (&x)[4]) {
-        x[0] = __uint_as_float(q.x); x[1] = __uint_as_float(q.y);
-        x[2] = __uint_as_float(q.z); x[3] = __uint_as_float(q.w);
-    }
-    __device__ static float vmax(const uint4& q) {
-        return fmaxf(fmaxf(__uint_as_float(q.x), __uint_as_float(q.y)),
-                     fmaxf(__uint_as_float(q.z), __uint_as_float(q.w)));
-    }
-    __device__ static uint32_t key_of_f(float x) { return Traits<DT_F32>::key_of(__float_as_uint(x)); }
 };
 
 __device__ __forceinline__ void write_result(const StepArgs& a, int ln, const LaneResult& r, int path) {
