@@ -745,8 +745,10 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
 
         // ---- hit vectors -> candidates >= the final threshold; the rest of them joins the tail
         ASX_MARK(4);
-        SyncC::sync();
-        const int nvh = sm.vec_count;
+        // (rows that fit the ring with a top-k push their candidates directly: nothing is listed)
+        const bool listed = !(resident && cut && !want_tail);
+        if (listed) SyncC::sync();
+        const int nvh = listed ? sm.vec_count : 0;
         bool list_ok = !decided && !general_row && nvh <= SK_CAPV;
         if (list_ok) {
             for (int i = tid; i < nvh; i += NT) {
