@@ -32,6 +32,9 @@ if ROOT not in sys.path:
 from paper_2210_15458_b200 import synth  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the step kernel on the default
+# workload, from the ncu capture summarised in profiles/as_step_stream_c2.md
+NCU_TRAFFIC_BYTES = {"c2": 16475392}
 RING_BYTES = 3 * L2_BYTES          # rotating input buffers: each launch reads from HBM
 
 
@@ -364,7 +367,8 @@ def run_ours(args):
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "as_step", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": peak_kind, "frac_of_8TBs_nominal": achieved / 8000.0,
-                     "us_per_launch": kms * 1e3, "bytes_per_launch": step_bytes(w), "traffic": None},
+                     "us_per_launch": kms * 1e3, "bytes_per_launch": step_bytes(w),
+                     "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
     }
     if world == 1:
         e_ms, h2d, d2h = e2e_step(w, args.steps, args.warmup)
