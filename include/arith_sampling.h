@@ -215,8 +215,9 @@ int as_decode_bigram_codes(const void *d_table, int dtype, int V, long long ld,
  *                         2 = cluster kernel (row split over the CTAs of a cluster)
  *   AS_TUNE_CLUSTER       CTAs per lane for the cluster kernel (1, 2, 4, 8)
  *   AS_TUNE_CTAS_PER_SM   resident CTAs per SM the grid is sized for
- *   AS_TUNE_STAGES        16 KB ring stages of the streaming kernel for rows that do not
- *                         fit the ring (2..12)
+ *   AS_TUNE_STAGES        16 KB ring stages of the streaming kernel (2..12); rows longer than
+ *                         the ring stream through it, so a small value also makes rows stream
+ *                         that would otherwise stay resident
  *   AS_TUNE_MIN_CTAS      streaming kernel build for bf16 rows that do not fit the ring:
  *                         3 = three CTAs per SM (1024-entry hit list, <= 72 registers; default),
  *                         2 = two CTAs per SM (2048-entry hit list)

@@ -343,7 +343,8 @@ int as_step(const void* d_logits, int dtype, int lanes, int V, long long ld, con
     if (g_tune_path == 0) {
         // streaming kernel: one CTA per lane; rows of up to 6 stages (96 KB) stay resident in the ring
         const int nsl = (int)((row_bytes + SK_STAGE_BYTES - 1) / SK_STAGE_BYTES);
-        const bool resident = nsl <= SK_RES_STAGES;
+        // rows of up to SK_RES_STAGES stages stay resident unless a smaller ring is asked for
+        const bool resident = nsl <= SK_RES_STAGES && !(g_tune_stages > 0 && g_tune_stages < nsl);
         a.fast = (top_k > 0 && top_k <= (resident ? SK_K0_RESIDENT : SK_K0_STREAMED)) || (top_k == 0 && top_p < 1.0);
         if (resident || a.fast) {
             int stages = resident ? (nsl < 1 ? 1 : nsl) : (g_tune_stages > 0 ? g_tune_stages : 3);
