@@ -62,7 +62,7 @@ extern "C" {
 #define AS_ERR_TIMEOUT (-4)      /* a bounded on-device wait ran out (reported per lane) */
 #define AS_ERR_NUMERIC (-5)      /* per-lane: non-finite logits / empty row / bad code */
 
-/* Largest vocabulary size accepted by as_step / as_decode_bigram*. */
+/* Largest vocabulary size accepted by as_step / as_decode_bigram* / as_encode_bigram. */
 #define AS_MAX_V (1 << 20)
 
 /*
@@ -207,6 +207,32 @@ int as_decode_bigram_codes(const void *d_table, int dtype, int V, long long ld,
                            int T, int eos, double temp, int top_k, double top_p,
                            int32_t *d_seq, int32_t *d_len, double *d_codes_final,
                            int32_t *d_lane_status, void *stream);
+
+/*
+ * Sequence -> interval, the codebook of Sec. 4.1 read in the other direction:
+ * in dictionary order every sequence owns the interval [lo, lo + P(sequence)),
+ * and a code decodes to that sequence exactly when it falls inside.  For lane i
+ * with tokens d_seq[i, 0..len-1] continued from d_prev[i] under the bigram
+ * table of as_decode_bigram:
+ *   lo    = sum_t ( prod_{s<t} p_s ) * F_t   (F_t: mass below token t in
+ *           vocabulary-index order under that step's modified distribution)
+ *   width = prod_t p_t
+ * with the same temperature / top-k / nucleus treatment as as_step.
+ *   d_prev  [lanes] i32 device   previous token of each lane, in [0, V)
+ *   d_seq   [lanes, T] i32 device, read only;  d_len [lanes] i32 device: tokens
+ *           to take from each row (values above T are read as T; padding is ignored)
+ *   d_lo, d_width  [lanes] f64 device, written
+ *   d_lane_status  NULL or [lanes] i32 device: AS_OK; AS_ERR_NUMERIC if a token
+ *           has probability zero under its step's distribution (cut by top-k /
+ *           nucleus, or masked) or the row is not usable; AS_ERR_INVALID_ARG if a
+ *           token id lies outside [0, V).  lo and width then hold the interval of
+ *           the prefix before the failing token.
+ * Errors: AS_ERR_INVALID_ARG, AS_ERR_UNSUPPORTED, AS_ERR_CUDA as for as_step.
+ */
+int as_encode_bigram(const void *d_table, int dtype, int V, long long ld,
+                     const int32_t *d_prev, const int32_t *d_seq, const int32_t *d_len,
+                     int lanes, int T, double temp, int top_k, double top_p,
+                     double *d_lo, double *d_width, int32_t *d_lane_status, void *stream);
 
 /*
  * Launch-shape overrides for measurement sweeps (process-wide, not thread-safe;

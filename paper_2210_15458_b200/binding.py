@@ -36,7 +36,7 @@ TUNE_MIN_CTAS = 5
 
 EXPORTS = ["as_lattice_codes", "as_step", "as_step_host", "as_step_host_work_bytes", "as_step_host_static",
            "as_decode_bigram",
-           "as_decode_bigram_codes", "as_tune", "as_last_error", "as_version"]
+           "as_decode_bigram_codes", "as_encode_bigram", "as_tune", "as_last_error", "as_version"]
 
 
 class AsError(RuntimeError):
@@ -77,10 +77,11 @@ def lib():
         L.as_step_host_work_bytes.restype = ctypes.c_size_t
         L.as_decode_bigram.argtypes = [P, I, I, LL, P, I, I, D, I, I, D, I, D, P, P, P, P, P]
         L.as_decode_bigram_codes.argtypes = [P, I, I, LL, P, P, I, I, I, D, I, D, P, P, P, P, P]
+        L.as_encode_bigram.argtypes = [P, I, I, LL, P, P, P, I, I, D, I, D, P, P, P, P]
         L.as_tune.argtypes = [I, I]
         L.as_last_error.restype = ctypes.c_char_p
         for n in ("as_lattice_codes", "as_step", "as_step_host", "as_decode_bigram",
-                  "as_decode_bigram_codes", "as_tune", "as_version"):
+                  "as_decode_bigram_codes", "as_encode_bigram", "as_tune", "as_version"):
             getattr(L, n).restype = I
         _lib = L
     return _lib
@@ -233,3 +234,25 @@ def as_decode_bigram_codes(table: torch.Tensor, prev: torch.Tensor, codes_in: to
                                         lanes, T, eos, temp, top_k, top_p, _ptr(seq), _ptr(length),
                                         _ptr(codes_final), _ptr(lane_status), _stream(stream)))
     return seq, length
+
+
+def as_encode_bigram(table: torch.Tensor, prev: torch.Tensor, seq: torch.Tensor, length: torch.Tensor,
+                     temp: float = 1.0, top_k: int = 0, top_p: float = 1.0, V: Optional[int] = None,
+                     lane_status: Optional[torch.Tensor] = None, stream=None):
+    """Interval [lo, lo + width) of each lane's sequence in dictionary order (Sec. 4.1)."""
+    rows, width_, ld = _logits_layout(table)
+    V = width_ if V is None else V
+    if rows < V:
+        raise ValueError("bigram table needs at least V rows")
+    if seq.dim() != 2 or not seq.is_contiguous() or seq.dtype != torch.int32:
+        raise ValueError("seq must be a contiguous [lanes, T] int32 tensor")
+    lanes, T = seq.shape
+    if prev.numel() != lanes or length.numel() != lanes:
+        raise ValueError("prev and length need one entry per lane")
+    dev = table.device
+    lo = torch.empty(lanes, dtype=torch.float64, device=dev)
+    width = torch.empty(lanes, dtype=torch.float64, device=dev)
+    _check(lib().as_encode_bigram(_ptr(table), _logits_dtype(table), V, ld, _ptr(prev), _ptr(seq), _ptr(length),
+                                  lanes, T, temp, top_k, top_p, _ptr(lo), _ptr(width), _ptr(lane_status),
+                                  _stream(stream)))
+    return lo, width

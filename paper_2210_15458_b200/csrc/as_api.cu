@@ -230,6 +230,44 @@ decode_generic_kernel(const void* __restrict__ table, int V, long long ld,
     }
 }
 
+// Sequence -> interval (the codebook of Sec. 4.1 in the other direction): one CTA per lane walks
+// the lane's tokens; lo gathers width * F_{i-1}, width multiplies by p_i.
+template <int DT>
+__global__ void __launch_bounds__(GEN_NT)
+encode_generic_kernel(const void* __restrict__ table, int V, long long ld, const int* __restrict__ prev0,
+                      const int* __restrict__ seq, const int* __restrict__ len, int lanes, int T,
+                      double inv_tau, int top_k, double top_p, double* __restrict__ lo_out,
+                      double* __restrict__ width_out, int* __restrict__ lane_status) {
+    __shared__ GenericSmem<GEN_NT> sm;
+    for (int ln = blockIdx.x; ln < lanes; ln += gridDim.x) {
+        int prev = prev0[ln];
+        const int n = min(len[ln], T);
+        double lo = 0.0, comp = 0.0, width = 1.0;
+        int status = ST_OK;
+        for (int t = 0; t < n; ++t) {
+            const int tok = seq[(size_t)ln * T + t];
+            if (prev < 0 || prev >= V || tok < 0 || tok >= V) { status = -1; break; }   // AS_ERR_INVALID_ARG
+            const char* row = reinterpret_cast<const char*>(table) + (size_t)prev * (size_t)ld * Traits<DT>::BYTES;
+            const bool vec_ok = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
+            GenericLane<DT, GEN_NT> g(sm, row, V, vec_ok);
+            const LaneResult r = g.interval_of(tok, inv_tau, top_k, top_p);
+            if (r.status != ST_OK) { status = r.status; break; }
+            // compensated running sum: the terms shrink geometrically with t
+            const double term = width * r.cdf_lo;
+            const double s = lo + term;
+            comp += (fabs(lo) >= fabs(term)) ? (lo - s) + term : (term - s) + lo;
+            lo = s;
+            width *= r.p_tok;
+            prev = tok;
+        }
+        if (threadIdx.x == 0) {
+            lo_out[ln] = lo + comp;
+            width_out[ln] = width;
+            if (lane_status) lane_status[ln] = status;
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------
 // argument checks
 // ---------------------------------------------------------------------------
@@ -519,6 +557,35 @@ int as_decode_bigram_codes(const void* d_table, int dtype, int V, long long ld, 
     if (!d_codes_in) return set_err(AS_ERR_INVALID_ARG, "d_codes_in is NULL");
     return decode_common(d_table, dtype, V, ld, d_prev, d_codes_in, lanes, 1, 0.0, T, eos, temp, top_k, top_p,
                          d_seq, d_len, d_codes_final, d_lane_status, stream);
+}
+
+int as_encode_bigram(const void* d_table, int dtype, int V, long long ld, const int32_t* d_prev,
+                     const int32_t* d_seq, const int32_t* d_len, int lanes, int T, double temp,
+                     int top_k, double top_p, double* d_lo, double* d_width, int32_t* d_lane_status,
+                     void* stream) {
+    if (lanes < 0) return set_err(AS_ERR_INVALID_ARG, "lanes = %d must be >= 0", lanes);
+    if (T < 0) return set_err(AS_ERR_INVALID_ARG, "T = %d must be >= 0", T);
+    int rc = check_scalars(dtype, V, ld, temp, top_p);
+    if (rc != AS_OK) return rc;
+    if (lanes == 0) return AS_OK;
+    if ((rc = check_data(d_table, dtype)) != AS_OK) return rc;
+    if (!d_prev || !d_len || !d_lo || !d_width) return set_err(AS_ERR_INVALID_ARG, "d_prev, d_len, d_lo or d_width is NULL");
+    if (T > 0 && !d_seq) return set_err(AS_ERR_INVALID_ARG, "d_seq is NULL");
+    const DeviceInfo* di;
+    rc = device_info(&di);
+    if (rc != AS_OK) return rc;
+    if (top_k < 0 || top_k >= V) top_k = 0;
+    if (!(top_p > 0.0 && top_p < 1.0)) top_p = 1.0;
+    const double inv_tau = 1.0 / temp;
+    const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dtype == AS_F32)
+        encode_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_table, V, ld, d_prev, d_seq, d_len, lanes, T, inv_tau, top_k, top_p, d_lo, d_width, d_lane_status);
+    else
+        encode_generic_kernel<DT_BF16><<<grid, GEN_NT, 0, st>>>(d_table, V, ld, d_prev, d_seq, d_len, lanes, T, inv_tau, top_k, top_p, d_lo, d_width, d_lane_status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "encode kernel launch");
+    return AS_OK;
 }
 
 }  // extern "C"

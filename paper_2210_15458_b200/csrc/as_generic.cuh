@@ -443,14 +443,10 @@ struct GenericLane {
         return out;
     }
 
-    __device__ __noinline__ LaneResult run(double c_in, double inv_tau_, int top_k, double top_p) {
-        if (top_k <= 0 && !(top_p > 0.0 && top_p < 1.0) && vec_ok) return run_nocut(c_in, inv_tau_);
-        inv_tau = inv_tau_;
-        fill_exp_table(sm.exp_tbl, tid);
-        double c = c_in;
-        const bool code_bad = !(c >= 0.0 && c <= 1.0);
-        if (c == 1.0) c = ASX_ONE_BELOW;
-
+    // Steps 1-4 of the general routine: the kept set as a predicate `p`, its size, and in
+    // chunk_sum the exclusive scan of the kept masses per chunk (chunk_sum[nchunks] = Z).
+    // Needs inv_tau set and the exp table filled; returns ST_OK or ST_NUMERIC.
+    __device__ __forceinline__ int prepare(int top_k, double top_p, Pred& p, int& n_kept) {
         // ---- 1. extremes and finite count
         unsigned kmax = 0, kmin = 0xFFFFFFFFu;
         int nfin = 0;
@@ -476,13 +472,11 @@ struct GenericLane {
             nfin += sm.red_i[w];
         }
         Sync::sync();
-        if (code_bad || kmin < Tr::KEY_NINF || kmax >= Tr::KEY_PINF || kmax == Tr::KEY_NINF)
-            return fail(c_in, ST_NUMERIC);
+        if (kmin < Tr::KEY_NINF || kmax >= Tr::KEY_PINF || kmax == Tr::KEY_NINF) return ST_NUMERIC;
         lmax = (double)Tr::value_f(kmax);
 
-        Pred p;
         p.T = Tr::KEY_NINF; p.need = 0; p.eq_mode = 0;     // every finite logit
-        int n_kept = nfin;
+        n_kept = nfin;
 
         // ---- 2. top-k
         if (top_k > 0 && top_k < nfin) {
@@ -549,6 +543,20 @@ struct GenericLane {
                 scan_exclusive(sm.chunk_sum, nchunks);
             }
         }
+
+        return ST_OK;
+    }
+
+    __device__ __noinline__ LaneResult run(double c_in, double inv_tau_, int top_k, double top_p) {
+        if (top_k <= 0 && !(top_p > 0.0 && top_p < 1.0) && vec_ok) return run_nocut(c_in, inv_tau_);
+        inv_tau = inv_tau_;
+        fill_exp_table(sm.exp_tbl, tid);
+        double c = c_in;
+        const bool code_bad = !(c >= 0.0 && c <= 1.0);
+        if (c == 1.0) c = ASX_ONE_BELOW;
+        Pred p;
+        int n_kept;
+        if (prepare(top_k, top_p, p, n_kept) != ST_OK || code_bad) return fail(c_in, ST_NUMERIC);
 
         // ---- 5/6. locate the chunk, then the element
         const double Z = sm.chunk_sum[nchunks];
@@ -630,6 +638,57 @@ struct GenericLane {
                 r.code_out = tok < 0 ? c_in : cn;
                 r.p_tok = tok_e / Z;
                 r.cdf_lo = tok_S / Z;
+                sm.res = r;
+            }
+        }
+        Sync::sync();
+        const LaneResult out = sm.res;
+        Sync::sync();
+        return out;
+    }
+
+    // The other direction of one step (the codebook of Sec. 4.1 read from token to interval):
+    // for a given token, cdf_lo = F_{tok-1} and p_tok under the same modified distribution.
+    // A token outside the kept set (probability zero) gives ST_NUMERIC.
+    __device__ __noinline__ LaneResult interval_of(int tok, double inv_tau_, int top_k, double top_p) {
+        inv_tau = inv_tau_;
+        fill_exp_table(sm.exp_tbl, tid);
+        Pred p;
+        int n_kept;
+        if (prepare(top_k, top_p, p, n_kept) != ST_OK) return fail(0.0, ST_NUMERIC);
+        const double Z = sm.chunk_sum[nchunks];
+        const int vi_tok = tok / E;
+        const int cstar = (vi_tok >> 5) / R;
+        if (warp == 0) {
+            double below = 0.0, e_tok = 0.0;
+            int has = 0;
+            int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[cstar] : 0;
+            for (int r = 0; r < R; ++r) {
+                if ((cstar * R + r) * 32 * E > tok) break;      // warp-uniform: rows past the token
+                uint32_t k[E];
+                int base;
+                chunk_keys(cstar, r, k, base);
+                const int rank0 = lane_rank0(k, p, tie_run);
+                const unsigned bits = kept_bits(k, p, rank0);
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    if (bits & (1u << e)) {
+                        const double m = mass(k[e]);
+                        if (base + e < tok) below += m;
+                        if (base + e == tok) { e_tok = m; has = 1; }
+                    }
+                }
+            }
+            below = warp_sum_d(below);
+            e_tok = warp_sum_d(e_tok);      // one lane holds it, the others add zero
+            has = warp_sum_i(has);
+            if (lane == 0) {
+                LaneResult r;
+                const bool kept = has > 0;
+                r.token = kept ? tok : -1; r.status = kept ? ST_OK : ST_NUMERIC; r.n_kept = n_kept;
+                r.code_out = 0.0;
+                r.p_tok = e_tok / Z;
+                r.cdf_lo = (sm.chunk_sum[cstar] + below) / Z;
                 sm.res = r;
             }
         }

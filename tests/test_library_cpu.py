@@ -59,6 +59,17 @@ def test_invalid_arguments_are_rejected_on_the_host(L):
     assert L.as_decode_bigram(p, 0, 2, 2, p, 1, 4, 1.5, 4, 0, 1.0, 0, 1.0, p, p, None, None, None) == B.ERR_INVALID_ARG
     assert L.as_decode_bigram(p, 0, 2, 2, p, 1, 4, 0.5, -1, 0, 1.0, 0, 1.0, p, p, None, None, None) == B.ERR_INVALID_ARG
     assert L.as_decode_bigram_codes(p, 0, 2, 2, p, None, 1, 4, 0, 1.0, 0, 1.0, p, p, None, None, None) == B.ERR_INVALID_ARG
+    enc = lambda **k: L.as_encode_bigram(k.get("table", p), 0, 2, 2, k.get("prev", p), k.get("seq", p), p,
+                                         k.get("lanes", 1), k.get("T", 4), k.get("temp", 1.0), 0, 1.0,
+                                         k.get("lo", p), p, None, None)
+    assert enc(lanes=-1) == B.ERR_INVALID_ARG
+    assert enc(T=-1) == B.ERR_INVALID_ARG
+    assert enc(temp=-1.0) == B.ERR_INVALID_ARG
+    assert enc(table=None) == B.ERR_INVALID_ARG
+    assert enc(prev=None) == B.ERR_INVALID_ARG
+    assert enc(seq=None) == B.ERR_INVALID_ARG
+    assert enc(lo=None) == B.ERR_INVALID_ARG
+    assert enc(lanes=0) == B.OK
     assert L.as_tune(99, 0) == B.ERR_INVALID_ARG and L.as_tune(B.TUNE_CLUSTER, 3) == B.ERR_INVALID_ARG
     assert L.as_step_host_work_bytes(0, 4, 10) >= 4 * 10 * 4 + 4 * 24
 
