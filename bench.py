@@ -306,6 +306,21 @@ def bench_bigram(steps: int, warmup: int):
                      "mean_len": tokens / w.lanes,
                      "row_gbs_upper": tokens * w.V * w.elem_bytes / ms / 1e6,
                      "duplicate_prefix_rate": dup_rates(seq)}
+    # the other direction on the sequences just decoded: sequence -> interval, same tokens
+    run_iid()
+    fn = lambda: B.as_encode_bigram(table, prev, seq, ln, w.temp, w.top_k, w.top_p)
+    for _ in range(max(1, warmup)):
+        fn()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for _ in range(steps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / steps
+    tokens = int(ln.sum().item())
+    out["encode"] = {"ms_per_encode": ms, "tokens": tokens, "tokens_per_s": tokens / ms * 1e3}
     out["workload"] = "c4: bf16 bigram table 32128x32128, 64 starts x 32 codes, T<=128, temp 0.8, EOS 1"
     return out
 
