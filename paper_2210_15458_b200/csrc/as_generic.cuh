@@ -647,10 +647,93 @@ struct GenericLane {
         return out;
     }
 
+    // interval_of for lanes without top-k / nucleus on 16-byte aligned rows: a packed max pass,
+    // then one pass that sums every mass and, separately, the masses below the token.
+    __device__ __noinline__ LaneResult interval_nocut(int tok, double inv_tau_) {
+        using P = Pass<DT>;
+        inv_tau = inv_tau_;
+        fill_exp_table(sm.exp_tbl, tid);
+        typename P::Acc acc = P::init();
+        const int nvf = (V * Tr::BYTES) >> 4;
+        for (int vi = tid; vi < nvf; vi += NT)
+            P::merge(acc, P::reduce(*reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row) + (size_t)vi * 16)));
+        for (int j = nvf * E + tid; j < V; j += NT) P::fold_scalar(acc, row, j);
+        uint32_t k0, k1;
+        P::keys(acc, k0, k1);
+        uint32_t kmax = warp_max_u(max(k0, k1));
+        if (lane == 0) sm.red_u[warp] = kmax;
+        Sync::sync();
+        kmax = 0;
+        for (int w = 0; w < NW; ++w) kmax = max(kmax, sm.red_u[w]);
+        if (kmax >= Tr::KEY_PINF || kmax <= Tr::KEY_NINF) {
+            Sync::sync();
+            return fail(0.0, ST_NUMERIC);
+        }
+        lmax = (double)Tr::value_f(kmax);
+        const double s64 = inv_tau * 0x1.71547652b82fep+6;          // 64 log2(e) / temp
+        const double c64 = -lmax * s64;
+        double all = 0.0, below = 0.0, e_tok = 0.0;
+        int has = 0, nfin = 0;
+        for (int vi = tid; vi < nvec; vi += NT) {
+            float x[E];
+            const int base = vi * E;
+            if (base + E <= V) {
+                const uint4 q = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row) + (size_t)base * Tr::BYTES);
+                P::floats(q, x);
+            } else {
+#pragma unroll
+                for (int e = 0; e < E; ++e)
+                    x[e] = (base + e < V) ? P::load_f(row, base + e) : __uint_as_float(0xFF800000u);
+            }
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const double m = exp2_64th(fma((double)x[e], s64, c64), sm.exp_tbl);
+                const bool fin = x[e] > __uint_as_float(0xFF800000u);
+                all += m;
+                nfin += fin;
+                if (base + e < tok) below += m;
+                if (base + e == tok && fin) { e_tok = m; has = 1; }
+            }
+        }
+        all = warp_sum_d(all);
+        below = warp_sum_d(below);
+        e_tok = warp_sum_d(e_tok);
+        has = warp_sum_i(has);
+        nfin = warp_sum_i(nfin);
+        if (lane == 0) {
+            sm.hist_mass[warp] = all;
+            sm.hist_mass[NW + warp] = below;
+            sm.hist_mass[2 * NW + warp] = e_tok;
+            sm.hist_cnt[warp] = has;
+            sm.hist_cnt[NW + warp] = nfin;
+        }
+        Sync::sync();
+        LaneResult r;
+        {
+            double Z = 0.0, S = 0.0, et = 0.0;
+            int h = 0, n = 0;
+            for (int w = 0; w < NW; ++w) {
+                Z += sm.hist_mass[w];
+                S += sm.hist_mass[NW + w];
+                et += sm.hist_mass[2 * NW + w];
+                h += sm.hist_cnt[w];
+                n += sm.hist_cnt[NW + w];
+            }
+            const bool kept = h > 0;
+            r.token = kept ? tok : -1; r.status = kept ? ST_OK : ST_NUMERIC; r.n_kept = n;
+            r.code_out = 0.0;
+            r.p_tok = et / Z;
+            r.cdf_lo = S / Z;
+        }
+        Sync::sync();
+        return r;
+    }
+
     // The other direction of one step (the codebook of Sec. 4.1 read from token to interval):
     // for a given token, cdf_lo = F_{tok-1} and p_tok under the same modified distribution.
     // A token outside the kept set (probability zero) gives ST_NUMERIC.
     __device__ __noinline__ LaneResult interval_of(int tok, double inv_tau_, int top_k, double top_p) {
+        if (top_k <= 0 && !(top_p > 0.0 && top_p < 1.0) && vec_ok) return interval_nocut(tok, inv_tau_);
         inv_tau = inv_tau_;
         fill_exp_table(sm.exp_tbl, tid);
         Pred p;
