@@ -262,12 +262,12 @@ def cpu_baseline_step(w, budget_s: float = 12.0):
 
 
 # ----------------------------------------------------------------------------- bigram workload (c4)
-def bench_bigram(steps: int, warmup: int):
+def bench_bigram(steps: int, warmup: int, S: int = 64):
     """tokens/s of the full decode loop over the 32128 x 32128 bf16 bigram table, lattice
     codes versus iid codes (ordinary ancestral sampling through the same kernel)."""
     import torch
     from paper_2210_15458_b200 import binding as B
-    w = synth.c4()
+    w = synth.c4(S=S)
     table = to_dev(w.table(), w.dtype)
     starts = torch.from_numpy(w.starts()).cuda()
     out = {}
@@ -321,7 +321,7 @@ def bench_bigram(steps: int, warmup: int):
     ms = a.elapsed_time(b) / steps
     tokens = int(ln.sum().item())
     out["encode"] = {"ms_per_encode": ms, "tokens": tokens, "tokens_per_s": tokens / ms * 1e3}
-    out["workload"] = "c4: bf16 bigram table 32128x32128, 64 starts x 32 codes, T<=128, temp 0.8, EOS 1"
+    out["workload"] = "c4: bf16 bigram table 32128x32128, %d starts x 32 codes, T<=128, temp 0.8, EOS 1" % S
     return out
 
 
@@ -457,12 +457,18 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c5"])
-    ap.add_argument("--lanes", type=int, default=None, help="lanes for c3 / c5 (default: the configured size)")
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c5", "c4"],
+                    help="c4 prints the bigram decode / encode loop's own line (a side measurement)")
+    ap.add_argument("--lanes", type=int, default=None,
+                    help="lanes for c3 / c5 / c4 (default: the configured size; c4: a multiple of 32)")
     ap.add_argument("--no-extras", action="store_true", help="skip the other workloads' short measurements")
     args = ap.parse_args()
     args.warmup = max(3, args.warmup)
-    if args.impl == "reference":
+    if args.workload == "c4":
+        if args.impl == "reference" or dist_env()[2] > 1:
+            raise SystemExit("--workload c4 is a single-GPU side measurement of the CUDA path")
+        print(json.dumps(bench_bigram(min(args.steps, 20), min(args.warmup, 3), S=(args.lanes or 2048) // 32)))
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
