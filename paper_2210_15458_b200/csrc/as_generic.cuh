@@ -201,6 +201,11 @@ struct GenericLane {
             sm.hist_mass[i] = 0.0;
         }
         Sync::sync();
+        // Each thread gathers runs of equal digits in registers and touches shared memory only
+        // when the digit changes: the leading digits of a row fall into two or three bins, and
+        // a shared-memory fp64 add is a compare-and-swap loop that such crowding serialises.
+        int cur_d = -1, cur_n = 0;
+        double cur_m = 0.0;
         for (int ci = warp; ci < nchunks; ci += NW) {
             int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[ci] : 0;
             for (int r = 0; r < R; ++r) {
@@ -213,11 +218,22 @@ struct GenericLane {
                 for (int e = 0; e < E; ++e) {
                     if ((bits & (1u << e)) && (k[e] & mask) == prefix) {
                         const int d = (k[e] >> shift) & 255;
-                        atomicAdd(&sm.hist_cnt[d], 1);
-                        if (MASS) atomicAdd(&sm.hist_mass[d], mass(k[e]));
+                        if (d != cur_d) {
+                            if (cur_n) {
+                                atomicAdd(&sm.hist_cnt[cur_d], cur_n);
+                                if (MASS) atomicAdd(&sm.hist_mass[cur_d], cur_m);
+                            }
+                            cur_d = d; cur_n = 0; cur_m = 0.0;
+                        }
+                        ++cur_n;
+                        if (MASS) cur_m += mass(k[e]);
                     }
                 }
             }
+        }
+        if (cur_n) {
+            atomicAdd(&sm.hist_cnt[cur_d], cur_n);
+            if (MASS) atomicAdd(&sm.hist_mass[cur_d], cur_m);
         }
         Sync::sync();
     }

@@ -378,6 +378,43 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2,
     return ok2;
 }
 
+// A lane whose hit vectors outgrew the list: the threshold is still exact (it comes from the
+// subset maxima, not from the list), so one more pass over the row (just streamed, mostly in
+// L2) takes the candidates >= t0key directly and sums the rest against `ref` in fp32.
+// Returns this thread's share of that sum; the caller's barrier completes the list.
+template <int DT, class StreamSmem>
+__device__ __noinline__ float recollect_row(StreamSmem& sm, int V, const char* row, float t0f, uint32_t t0key,
+                                            float ref, float scale2) {
+    using Tr = Traits<DT>;
+    using P = Pass<DT>;
+    constexpr int E = Tr::E;
+    const int tid = threadIdx.x;
+    const int nvec_full = (V * Tr::BYTES) >> 4;
+    float tail = 0.f;
+    auto take = [&](float x, int j) {
+        bool hit = false;
+        if (x >= t0f) {
+            const uint32_t key = P::key_of_f(x);
+            if (key >= t0key && key > Tr::KEY_NINF) {
+                hit = true;
+                const int slot = atomicAdd(&sm.cand_count, 1);
+                if (slot < SK_CAP) sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)j;
+            }
+        }
+        if (!hit) tail += ex2_approx((x - ref) * scale2);
+    };
+#pragma unroll 2
+    for (int v = tid; v < nvec_full; v += SK_NT) {
+        const uint4 q = __ldg(reinterpret_cast<const uint4*>(row) + v);
+        float x[E];
+        P::floats(q, x);
+#pragma unroll
+        for (int e = 0; e < E; ++e) take(x[e], v * E + e);
+    }
+    for (int j = nvec_full * E + tid; j < V; j += SK_NT) take(Tr::value_f(Tr::load_key(row, j)), j);
+    return tail;
+}
+
 template <int DT, int CAPV, int MINB>
 __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const StepArgs a, const int stages) {
     using StreamSmem = StreamSmemT<CAPV>;
@@ -791,6 +828,17 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                     if (want_tail && !hit) tail += ex2_approx((x[e] - ref) * scale2);
                 }
             }
+        }
+        if (!list_ok && !decided && !general_row && nvh > SK_CAPV && !*(volatile int*)&sm.poisoned) {
+            // more hit vectors than the list holds: take the candidates in one more pass, against
+            // the threshold that the whole row's subset maxima give now
+            ASX_COUNT(8);
+            uint32_t gm2, t0new;
+            threshold(acc, gm2, t0new, true, t0key);
+            t0key = max(t0key, t0new);
+            t0f = Tr::value_f(t0key);
+            tail = recollect_row<DT, StreamSmem>(sm, V, row, t0f, t0key, ref, scale2);
+            list_ok = true;
         }
         double tailsum = 0.0;
         if (want_tail) {
