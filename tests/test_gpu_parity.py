@@ -453,15 +453,16 @@ def test_step_nucleus_deeper_than_the_list(B, orc, dtype):
 
 @pytest.mark.parametrize("dtype", [F32, BF16])
 def test_step_hit_list_overflow_takes_one_more_pass(B, orc, dtype):
-    # rows that rise towards their end: between two refreshes of the threshold every vector beats
-    # the stale value, so the hit list overflows; the final threshold is exact all the same and
-    # the candidates are taken in a second pass over the row, without the general routine
+    # rows whose level rises from one 16 KB slice to the next: between two refreshes of the
+    # threshold a large share of the vectors beats the stale value, so the hit list overflows;
+    # the final threshold is exact all the same and the candidates are taken in a second pass
+    # over the row, without the general routine
     rng = np.random.default_rng(900)
-    V = 140000 if dtype == F32 else 200000
+    per_slice = 4096 if dtype == F32 else 8192
+    V = 36 * per_slice + 1232                                  # row pitch stays a multiple of 16 bytes
     lanes = 12
-    x = np.sort(rng.normal(0, 3, (lanes, V)).astype(np.float32), axis=1)
-    x[:, -1] += np.arange(lanes, dtype=np.float32) * 0.25         # different shapes at the very top
-    x[6:] += rng.normal(0, 0.3, (lanes - 6, V)).astype(np.float32)  # half of them only roughly sorted
+    x = rng.normal(0, 3, (lanes, V)).astype(np.float32)
+    x += (np.arange(V) // per_slice).astype(np.float32) * 0.45
     arr = _store(x, dtype)
     codes = rng.random(lanes)
     for temp, k, p in [(1.0, 40, 1.0), (0.8, 0, 0.9), (1.0, 64, 0.95)]:
@@ -472,4 +473,4 @@ def test_step_hit_list_overflow_takes_one_more_pass(B, orc, dtype):
         compare_step(ref, tok.cpu().numpy(), c2.cpu().numpy(), d["p_tok"].cpu().numpy(),
                      d["n_kept"].cpu().numpy(), d["lane_status"].cpu().numpy(),
                      what="overflow %s" % ((temp, k, p),))
-        assert (d["path"].cpu().numpy() == B.PATH_COMPACT).sum() >= lanes // 2
+        assert (d["path"].cpu().numpy() == B.PATH_COMPACT).sum() >= lanes - 2
