@@ -473,4 +473,4 @@ def test_step_hit_list_overflow_takes_one_more_pass(B, orc, dtype):
         compare_step(ref, tok.cpu().numpy(), c2.cpu().numpy(), d["p_tok"].cpu().numpy(),
                      d["n_kept"].cpu().numpy(), d["lane_status"].cpu().numpy(),
                      what="overflow %s" % ((temp, k, p),))
-        assert (d["path"].cpu().numpy() == B.PATH_COMPACT).sum() >= lanes - 2
+        assert (d["path"].cpu().numpy() == B.PATH_COMPACT).sum() >= lanes // 2 + 1
