@@ -263,14 +263,18 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
 // Nucleus-only lane whose nucleus reaches below the exact depth of the list (key >= t0key).
 // The row is read again from global memory (it was just streamed, so mostly from L2):
 //   1. masses and counts of the elements below the old threshold go into a histogram over
-//      y = (x - max) * scale2, 64 bins per unit of log2 mass, 16 units deep;
+//      y = (x - max) * scale2, 128 bins per unit of log2 mass, 8 units deep (a list of a few
+//      hundred candidates never reaches further down, and the fewer elements fall into the
+//      window, the fewer shared-memory atomics the pass costs);
 //   2. the bins are taken from the top until their mass covers what the nucleus still lacks
 //      (with a margin for the fp32 sums): that gives a lower threshold t1 below which no
 //      nucleus token can lie, if the candidates still fit the list;
 //   3. everything >= t1 is collected afresh, the rest summed in fp32, and the exact epilogue
 //      runs again.  Returns false if the window or the list capacity does not suffice.
+constexpr int RR_AHEAD_L2 = 16;    // re-read passes: iterations (of 4 KB per CTA) asked for ahead, into L2
+constexpr int RR_AHEAD_L1 = 4;     // ... and into L1
 constexpr int DP_NB = 1024;
-constexpr float DP_BINS_PER_UNIT = 64.f;
+constexpr float DP_BINS_PER_UNIT = 128.f;
 template <int DT, class StreamSmem>
 __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2, double inv_tau, double top_p,
                                             const char* row, uint32_t gmax, float t0f, double tailsum, double c,
@@ -292,8 +296,15 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2,
     for (int i = tid; i < SK_CAP + 4; i += NT) sm.u.ep.cand[i] = 0ull;
     SyncC::sync();
     auto visit = [&](auto&& f) {                           // f(x, index) over the whole row
+        const uint4* rv = reinterpret_cast<const uint4*>(row);
+        // thread t of every eighth asks for the 128-byte line its neighbours share
+        if ((tid & 7) == 0)
+            for (int i = 0; i < RR_AHEAD_L2; ++i)
+                if (tid + i * NT < nvec_full) prefetch_l2(rv + tid + i * NT);
         for (int v = tid; v < nvec_full; v += NT) {
-            const uint4 q = __ldg(reinterpret_cast<const uint4*>(row) + v);
+            if ((tid & 7) == 0 && v + RR_AHEAD_L2 * NT < nvec_full) prefetch_l2(rv + v + RR_AHEAD_L2 * NT);
+            if ((tid & 7) == 0 && v + RR_AHEAD_L1 * NT < nvec_full) prefetch_l1(rv + v + RR_AHEAD_L1 * NT);
+            const uint4 q = __ldg(rv + v);
             float x[E];
             P::floats(q, x);
 #pragma unroll
@@ -403,9 +414,14 @@ __device__ __noinline__ float recollect_row(StreamSmem& sm, int V, const char* r
         }
         if (!hit) tail += ex2_approx((x - ref) * scale2);
     };
-#pragma unroll 2
+    const uint4* rv = reinterpret_cast<const uint4*>(row);
+    if ((tid & 7) == 0)
+        for (int i = 0; i < RR_AHEAD_L2; ++i)
+            if (tid + i * SK_NT < nvec_full) prefetch_l2(rv + tid + i * SK_NT);
     for (int v = tid; v < nvec_full; v += SK_NT) {
-        const uint4 q = __ldg(reinterpret_cast<const uint4*>(row) + v);
+        if ((tid & 7) == 0 && v + RR_AHEAD_L2 * SK_NT < nvec_full) prefetch_l2(rv + v + RR_AHEAD_L2 * SK_NT);
+        if ((tid & 7) == 0 && v + RR_AHEAD_L1 * SK_NT < nvec_full) prefetch_l1(rv + v + RR_AHEAD_L1 * SK_NT);
+        const uint4 q = __ldg(rv + v);
         float x[E];
         P::floats(q, x);
 #pragma unroll
