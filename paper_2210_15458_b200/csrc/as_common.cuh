@@ -218,11 +218,6 @@ __device__ __forceinline__ double exp2_64th(double t, const double* __restrict__
     return __hiloint2double(__double2hiint(v) + (n << 20), __double2loint(v));
 }
 
-// Cache hints for passes that re-read a row with one load per thread in flight: the line a later
-// iteration needs is asked for now, at no cost in registers.
-__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
-__device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
-
 // ---------------------------------------------------------------------------
 // Packed NaN-propagating maxima and float views of one 16-byte vector.
 // ---------------------------------------------------------------------------

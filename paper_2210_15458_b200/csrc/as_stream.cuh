@@ -260,6 +260,35 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
     return sm.b_i[1] != 0;
 }
 
+// One more pass over a 16-byte aligned row in global memory, f(vector, vector index), thread t
+// taking vectors t, t + 256, ...  Each thread keeps D asynchronous 16-byte copies in flight into
+// slots of its own in `staging` (D * 256 vectors of shared memory that are dead meanwhile): with a
+// single load per thread in flight a lone CTA is latency-bound, and holding more loads in
+// registers would cost the whole kernel registers.
+template <int D, class F>
+__device__ __forceinline__ void reread_row(uint4* staging, const char* row, int nvec_full, F&& f) {
+    const int tid = threadIdx.x;
+    const uint4* rv = reinterpret_cast<const uint4*>(row);
+    uint4* mine = staging + tid;
+    const uint32_t mine_s = smem_u32(mine);
+    auto copy = [&](int slot, int v) {
+        if (v < nvec_full)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(mine_s + slot * (SK_NT * 16)), "l"(rv + v) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");     // one group per step, empty or not
+    };
+#pragma unroll
+    for (int d = 0; d < D; ++d) copy(d, tid + d * SK_NT);
+    int slot = 0;
+    for (int v = tid; v < nvec_full; v += SK_NT) {
+        asm volatile("cp.async.wait_group %0;" ::"n"(D - 1) : "memory");
+        const uint4 q = mine[slot * SK_NT];
+        f(q, v);
+        copy(slot, v + D * SK_NT);                 // after f: the slot's value has been consumed
+        slot = slot + 1 == D ? 0 : slot + 1;
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
 // Nucleus-only lane whose nucleus reaches below the exact depth of the list (key >= t0key).
 // The row is read again from global memory (it was just streamed, so mostly from L2):
 //   1. masses and counts of the elements below the old threshold go into a histogram over
@@ -271,8 +300,6 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
 //      nucleus token can lie, if the candidates still fit the list;
 //   3. everything >= t1 is collected afresh, the rest summed in fp32, and the exact epilogue
 //      runs again.  Returns false if the window or the list capacity does not suffice.
-constexpr int RR_AHEAD_L2 = 16;    // re-read passes: iterations (of 4 KB per CTA) asked for ahead, into L2
-constexpr int RR_AHEAD_L1 = 4;     // ... and into L1
 constexpr int DP_NB = 1024;
 constexpr float DP_BINS_PER_UNIT = 128.f;
 template <int DT, class StreamSmem>
@@ -296,20 +323,15 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2,
     for (int i = tid; i < SK_CAP + 4; i += NT) sm.u.ep.cand[i] = 0ull;
     SyncC::sync();
     auto visit = [&](auto&& f) {                           // f(x, index) over the whole row
-        const uint4* rv = reinterpret_cast<const uint4*>(row);
-        // thread t of every eighth asks for the 128-byte line its neighbours share
-        if ((tid & 7) == 0)
-            for (int i = 0; i < RR_AHEAD_L2; ++i)
-                if (tid + i * NT < nvec_full) prefetch_l2(rv + tid + i * NT);
-        for (int v = tid; v < nvec_full; v += NT) {
-            if ((tid & 7) == 0 && v + RR_AHEAD_L2 * NT < nvec_full) prefetch_l2(rv + v + RR_AHEAD_L2 * NT);
-            if ((tid & 7) == 0 && v + RR_AHEAD_L1 * NT < nvec_full) prefetch_l1(rv + v + RR_AHEAD_L1 * NT);
-            const uint4 q = __ldg(rv + v);
+        // staging: the hit-vector list past the histogram
+        constexpr int D = (int)((sizeof(sm.u.ep.v.cvec) - DP_NB * 8) / (NT * 16));
+        static_assert(D >= 2, "the list is too small to stage a re-read");
+        reread_row<D>(sm.u.ep.v.cvec + DP_NB / 2, row, nvec_full, [&](const uint4& q, int v) {
             float x[E];
             P::floats(q, x);
 #pragma unroll
             for (int e = 0; e < E; ++e) f(x[e], v * E + e);
-        }
+        });
         for (int j = nvec_full * E + tid; j < V; j += NT) f(Tr::value_f(Tr::load_key(row, j)), j);
     };
     // ---- 1. histogram below the old threshold
@@ -414,19 +436,13 @@ __device__ __noinline__ float recollect_row(StreamSmem& sm, int V, const char* r
         }
         if (!hit) tail += ex2_approx((x - ref) * scale2);
     };
-    const uint4* rv = reinterpret_cast<const uint4*>(row);
-    if ((tid & 7) == 0)
-        for (int i = 0; i < RR_AHEAD_L2; ++i)
-            if (tid + i * SK_NT < nvec_full) prefetch_l2(rv + tid + i * SK_NT);
-    for (int v = tid; v < nvec_full; v += SK_NT) {
-        if ((tid & 7) == 0 && v + RR_AHEAD_L2 * SK_NT < nvec_full) prefetch_l2(rv + v + RR_AHEAD_L2 * SK_NT);
-        if ((tid & 7) == 0 && v + RR_AHEAD_L1 * SK_NT < nvec_full) prefetch_l1(rv + v + RR_AHEAD_L1 * SK_NT);
-        const uint4 q = __ldg(rv + v);
+    constexpr int D = (int)(sizeof(sm.u.ep.v.cvec) / (SK_NT * 16)) < 8 ? (int)(sizeof(sm.u.ep.v.cvec) / (SK_NT * 16)) : 8;
+    reread_row<D>(sm.u.ep.v.cvec, row, nvec_full, [&](const uint4& q, int v) {   // the list is dead: staging
         float x[E];
         P::floats(q, x);
 #pragma unroll
         for (int e = 0; e < E; ++e) take(x[e], v * E + e);
-    }
+    });
     for (int j = nvec_full * E + tid; j < V; j += SK_NT) take(Tr::value_f(Tr::load_key(row, j)), j);
     return tail;
 }
