@@ -26,6 +26,12 @@
  *   orc_encode_bigram     the other direction of the codebook (Sec. 4.1): the
  *                         interval [w, w + P(sequence)) of a sequence in
  *                         dictionary order.
+ *   orc_ngram_diversity   the n-gram diversity score of Sec. 5.1 ("Diverse beam
+ *                         generation"): d = sum_{n=1..4} d_n, d_n = unique
+ *                         n-grams / all n-grams in the N sequences of a group.
+ *   orc_reward_mean       the sample-mean estimator (1/N) sum_i s(x_i) of Sec. 4.2
+ *                         (Proposition on its unbiasedness) for an additive
+ *                         reward s(x) = sum_t r[x_t].
  *
  * Readings taken where the paper is silent (all also stated in the design
  * notes): intervals are half-open [F_{i-1}, F_i); order of modifiers is
@@ -409,6 +415,92 @@ int orc_encode_bigram(const void *table, int dtype, long V, long ld,
         if (status) status[i] = st;
     }
     ws_free(&w);
+    return ORC_OK;
+}
+
+/*
+ * n-gram diversity (Sec. 5.1, "Diverse beam generation"): for every group g
+ * of N consecutive lanes and n = 1..4,
+ *   total[g][n-1]  = number of n-grams in the group's sequences
+ *                  = sum_i max(len_i - n + 1, 0)
+ *   unique[g][n-1] = number of distinct ones among them (an n-gram is the
+ *                    tuple of n consecutive emitted tokens; padding is not
+ *                    part of any n-gram)
+ *   d[g] = sum_n unique/total, a term with total = 0 contributing 0
+ * (reading: the paper does not say what an empty denominator gives).
+ * By the definition: write out all n-grams, sort them, count the distinct.
+ */
+static long g_ng_n;
+static int cmp_ngram(const void *pa, const void *pb)
+{
+    const int32_t *a = (const int32_t *)pa, *b = (const int32_t *)pb;
+    long k;
+    for (k = 0; k < g_ng_n; ++k) {
+        if (a[k] < b[k]) return -1;
+        if (a[k] > b[k]) return 1;
+    }
+    return 0;
+}
+
+int orc_ngram_diversity(const int32_t *seq, const int32_t *len, long S, long N, long T,
+                        int64_t *unique, int64_t *total, double *d)
+{
+    long g, n, i, t, k;
+    if (!seq || !len || !unique || !total || !d || S < 0 || N < 1 || T < 0) return ORC_ERR_INVALID_ARG;
+    int32_t *buf = (int32_t *)malloc(sizeof(int32_t) * 4 * (size_t)(N * T + 1));
+    if (!buf) return ORC_ERR_INVALID_ARG;
+    for (g = 0; g < S; ++g) {
+        double dsum = 0.0;
+        for (n = 1; n <= 4; ++n) {
+            long m = 0;
+            for (i = 0; i < N; ++i) {
+                long lane = g * N + i;
+                long L = len[lane] < T ? len[lane] : T;
+                for (t = 0; t + n <= L; ++t, ++m)
+                    for (k = 0; k < n; ++k) buf[m * n + k] = seq[lane * T + t + k];
+            }
+            g_ng_n = n;
+            qsort(buf, (size_t)m, sizeof(int32_t) * (size_t)n, cmp_ngram);
+            long u = 0;
+            for (i = 0; i < m; ++i)
+                if (i == 0 || cmp_ngram(buf + (i - 1) * n, buf + i * n) != 0) ++u;
+            unique[g * 4 + n - 1] = u;
+            total[g * 4 + n - 1] = m;
+            if (m > 0) dsum += (double)u / (double)m;
+        }
+        d[g] = dsum;
+    }
+    free(buf);
+    return ORC_OK;
+}
+
+/*
+ * Sample-mean estimator (Sec. 4.2, Proposition "estimator unbiased and
+ * consistent"; used in Sec. 5.2): with the additive reward
+ * s(x) = sum_{t < len} r[x_t], per lane s, per group of N consecutive lanes
+ * mean[g] = (1/N) sum_i s(x_i).
+ */
+int orc_reward_mean(const int32_t *seq, const int32_t *len, long S, long N, long T,
+                    const double *r, long V, double *lane_reward, double *mean)
+{
+    long g, i, t;
+    if (!seq || !len || !r || !mean || S < 0 || N < 1 || T < 0 || V < 1) return ORC_ERR_INVALID_ARG;
+    for (g = 0; g < S; ++g) {
+        nsum acc = {0.0, 0.0};
+        for (i = 0; i < N; ++i) {
+            long lane = g * N + i;
+            long L = len[lane] < T ? len[lane] : T;
+            nsum s = {0.0, 0.0};
+            for (t = 0; t < L; ++t) {
+                long tok = seq[lane * T + t];
+                if (tok < 0 || tok >= V) return ORC_ERR_INVALID_ARG;
+                nsum_add(&s, r[tok]);
+            }
+            if (lane_reward) lane_reward[lane] = nsum_val(&s);
+            nsum_add(&acc, nsum_val(&s));
+        }
+        mean[g] = nsum_val(&acc) / (double)N;
+    }
     return ORC_OK;
 }
 

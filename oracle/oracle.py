@@ -53,8 +53,11 @@ def lib():
                                                  + [P] * 8 + [L, L])
         _lib.orc_decode_bigram.argtypes = [P, ctypes.c_int, L, L, P, L, L, D, L, L, D, L, D, P, P, P, P]
         _lib.orc_encode_bigram.argtypes = [P, ctypes.c_int, L, L, P, P, P, L, L, D, L, D, P, P, P]
+        _lib.orc_ngram_diversity.argtypes = [P, P, L, L, L, P, P, P]
+        _lib.orc_reward_mean.argtypes = [P, P, L, L, L, P, L, P, P]
         for f in (_lib.orc_lattice_codes, _lib.orc_step, _lib.orc_decode_bigram_codes,
-                  _lib.orc_decode_bigram, _lib.orc_encode_bigram, _lib.orc_version):
+                  _lib.orc_decode_bigram, _lib.orc_encode_bigram, _lib.orc_ngram_diversity,
+                  _lib.orc_reward_mean, _lib.orc_version):
             f.restype = ctypes.c_int
     return _lib
 
@@ -218,3 +221,37 @@ def encode_bigram(table: np.ndarray, dtype: int, prev: np.ndarray, seq: np.ndarr
     if rc != OK:
         raise ValueError("orc_encode_bigram returned %d" % rc)
     return lo, width, status
+
+
+def ngram_diversity(seq: np.ndarray, length: np.ndarray, N: int):
+    """(unique[S,4], total[S,4], d[S]) of Sec. 5.1's n-gram diversity per group of N lanes."""
+    seq = np.ascontiguousarray(seq, dtype=np.int32)
+    length = np.ascontiguousarray(length, dtype=np.int32)
+    lanes, T = seq.shape
+    if lanes % N:
+        raise ValueError("lanes must be a multiple of N")
+    S = lanes // N
+    unique = np.empty((S, 4), np.int64)
+    total = np.empty((S, 4), np.int64)
+    d = np.empty(S, np.float64)
+    rc = lib().orc_ngram_diversity(_ptr(seq), _ptr(length), S, N, T, _ptr(unique), _ptr(total), _ptr(d))
+    if rc != OK:
+        raise ValueError("orc_ngram_diversity returned %d" % rc)
+    return unique, total, d
+
+
+def reward_mean(seq: np.ndarray, length: np.ndarray, N: int, r: np.ndarray):
+    """(lane_reward[lanes], mean[S]): additive reward per lane and its mean per group of N lanes."""
+    seq = np.ascontiguousarray(seq, dtype=np.int32)
+    length = np.ascontiguousarray(length, dtype=np.int32)
+    r = np.ascontiguousarray(r, dtype=np.float64)
+    lanes, T = seq.shape
+    if lanes % N:
+        raise ValueError("lanes must be a multiple of N")
+    S = lanes // N
+    lane_reward = np.empty(lanes, np.float64)
+    mean = np.empty(S, np.float64)
+    rc = lib().orc_reward_mean(_ptr(seq), _ptr(length), S, N, T, _ptr(r), len(r), _ptr(lane_reward), _ptr(mean))
+    if rc != OK:
+        raise ValueError("orc_reward_mean returned %d" % rc)
+    return lane_reward, mean

@@ -424,3 +424,136 @@ def test_threads_do_not_change_results(orc):
     a = orc.step(logits, F32, codes, temp=0.9, top_k=7, top_p=0.9)
     b = orc.step(logits, F32, codes, temp=0.9, top_k=7, top_p=0.9, threads=5)
     assert (a.tokens == b.tokens).all() and (a.codes == b.codes).all()
+
+
+# --------------------------------------------------------------------------- n-gram diversity (Sec. 5.1)
+def _diversity_by_sets(seq, length, N):
+    """The definition with Python sets: distinct n-grams over all n-grams, per group."""
+    lanes, T = seq.shape
+    out_u, out_t, out_d = [], [], []
+    for g in range(lanes // N):
+        us, ts, d = [], [], Fraction(0)
+        for n in (1, 2, 3, 4):
+            grams = [tuple(int(v) for v in seq[i, t:t + n]) for i in range(g * N, (g + 1) * N)
+                     for t in range(0, min(int(length[i]), T) - n + 1)]
+            us.append(len(set(grams)))
+            ts.append(len(grams))
+            if grams:
+                d += Fraction(len(set(grams)), len(grams))
+        out_u.append(us)
+        out_t.append(ts)
+        out_d.append(float(d))
+    return np.array(out_u), np.array(out_t), np.array(out_d)
+
+
+def test_diversity_hand_example(orc):
+    # two sequences (1 2 3) and (1 2 4 5): unigrams 1 2 3 1 2 4 5 -> 5 distinct of 7; bigrams
+    # (1 2)(2 3)(1 2)(2 4)(4 5) -> 4 of 5; trigrams (1 2 3)(1 2 4)(2 4 5) -> 3 of 3; one 4-gram
+    seq = np.array([[1, 2, 3, -1], [1, 2, 4, 5]], np.int32)
+    u, t, d = orc.ngram_diversity(seq, np.array([3, 4], np.int32), 2)
+    assert u.tolist() == [[5, 4, 3, 1]] and t.tolist() == [[7, 5, 3, 1]]
+    assert d[0] == pytest.approx(5 / 7 + 4 / 5 + 1 + 1, abs=1e-15)
+
+
+def test_diversity_closed_forms(orc):
+    T, N = 9, 6
+    # N copies of one sequence of distinct tokens: every n-gram occurs N times -> d_n = 1/N
+    same = np.tile(np.arange(10, 10 + T, dtype=np.int32), (N, 1))
+    u, t, d = orc.ngram_diversity(same, np.full(N, T, np.int32), N)
+    assert u.tolist() == [[T, T - 1, T - 2, T - 3]] and t.tolist() == [[N * T, N * (T - 1), N * (T - 2), N * (T - 3)]]
+    assert d[0] == pytest.approx(4.0 / N, abs=1e-15)
+    # all tokens distinct across the group: nothing repeats -> d = 4
+    distinct = np.arange(N * T, dtype=np.int32).reshape(N, T)
+    u, t, d = orc.ngram_diversity(distinct, np.full(N, T, np.int32), N)
+    assert (u == t).all() and d[0] == 4.0
+    # one repeated token: a single unigram, bigram, ... whatever the length
+    ones = np.full((N, T), 7, np.int32)
+    u, t, d = orc.ngram_diversity(ones, np.full(N, T, np.int32), N)
+    assert u.tolist() == [[1, 1, 1, 1]]
+    # lengths below n give no n-grams; an empty group scores 0 (reading: empty ratio = 0)
+    short = np.array([[3, 4, -1, -1], [3, -1, -1, -1], [-1, -1, -1, -1]], np.int32)
+    u, t, d = orc.ngram_diversity(short, np.array([2, 1, 0], np.int32), 3)
+    assert t.tolist() == [[3, 1, 0, 0]] and u.tolist() == [[2, 1, 0, 0]]
+    assert d[0] == pytest.approx(2 / 3 + 1.0, abs=1e-15)
+    u, t, d = orc.ngram_diversity(short, np.zeros(3, np.int32), 3)
+    assert t.sum() == 0 and d[0] == 0.0
+    # padding is never part of an n-gram, whatever value it holds
+    a = np.array([[5, 6, 7, 8, 9], [5, 6, 1, 1, 1]], np.int32)
+    b = a.copy()
+    b[1, 2:] = -1
+    ua, ta, da = orc.ngram_diversity(a, np.array([5, 2], np.int32), 2)
+    ub, tb, db = orc.ngram_diversity(b, np.array([5, 2], np.int32), 2)
+    assert (ua == ub).all() and (ta == tb).all() and da[0] == db[0]
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_diversity_against_set_counting(orc, seed):
+    rng = np.random.default_rng(seed)
+    S, N, T = 5, 7, 11
+    seq = rng.integers(0, 4 + 3 * seed, (S * N, T)).astype(np.int32)      # small alphabets: many repeats
+    length = rng.integers(0, T + 1, S * N).astype(np.int32)
+    for i in range(S * N):
+        seq[i, length[i]:] = -1
+    u, t, d = orc.ngram_diversity(seq, length, N)
+    wu, wt, wd = _diversity_by_sets(seq, length, N)
+    assert (u == wu).all() and (t == wt).all()
+    np.testing.assert_allclose(d, wd, rtol=0, atol=1e-14)
+
+
+def test_diversity_of_decoded_groups_lattice_vs_iid(orc):
+    # Sec. 5.1's observation in miniature: at equal temperature a group decoded from lattice
+    # codes is at least as diverse on average as one decoded from iid codes
+    table = _tiny_model(12, seed=77, sigma=1.5)
+    N, T, S = 8, 6, 40
+    starts = np.arange(S, dtype=np.int32) % 12
+    rng = np.random.default_rng(5)
+    lat = orc.decode_bigram(table, F32, starts, N, 0.37, T, -1)
+    iid = orc.decode_bigram_codes(table, F32, np.repeat(starts, N).astype(np.int32), rng.random(S * N), T, -1)
+    d_lat = orc.ngram_diversity(lat.seq, lat.len, N)[2].mean()
+    d_iid = orc.ngram_diversity(iid.seq, iid.len, N)[2].mean()
+    assert d_lat > d_iid
+
+
+# --------------------------------------------------------------------------- sample-mean estimator (Sec. 4.2)
+def test_reward_mean_is_exact_when_widths_are_multiples_of_1_over_N(orc):
+    # one step over 4 symbols with probabilities 1/8, 3/8, 2/8, 2/8 (as exactly as fp32 logits
+    # allow): N = 8 lattice codes hit the symbols 1, 3, 2, 2 times for every shift that keeps
+    # 1e-6 away from the lattice, so the estimator equals the expectation with zero variance
+    p = np.array([1, 3, 2, 2]) / 8.0
+    table = _rows([np.log(p)] * 4)
+    r = np.array([0.25, -1.5, 4.0, 10.0])
+    want = float((p * r).sum())
+    for u in [0.013, 0.3, 0.5, 0.77, 0.999]:
+        o = orc.decode_bigram(table, F32, np.array([0], np.int32), 8, u, 1, -1)
+        lane, mean = orc.reward_mean(o.seq, o.len, 8, r)
+        assert np.bincount(o.seq[:, 0], minlength=4).tolist() == [1, 3, 2, 2]
+        assert mean[0] == pytest.approx(want, abs=1e-14)
+        assert lane.tolist() == [r[t] for t in o.seq[:, 0]]
+
+
+def test_reward_mean_is_unbiased_over_shifts(orc):
+    # Sec. 4.2's proposition against the exact expectation from the enumerated codebook
+    table = _tiny_model(4, seed=91)
+    T, start, N, eos = 4, 2, 3, 0
+    book = _book(table, start, T, eos)
+    r = np.array([0.5, -2.0, 3.0, 1.25])
+    want = float(ex.expectation(book, lambda seq: sum(r[t] for t in seq)))
+    K = 3000
+    tot = 0.0
+    for k in range(K):
+        o = orc.decode_bigram(table, F32, np.array([start], np.int32), N, (k + 0.5) / K, T, eos)
+        lane, mean = orc.reward_mean(o.seq, o.len, N, r)
+        for i in range(N):                                   # per lane: padding adds nothing
+            assert lane[i] == pytest.approx(sum(r[t] for t in o.seq[i, :o.len[i]]), abs=1e-14)
+        tot += mean[0]
+    assert tot / K == pytest.approx(want, abs=5e-3)
+
+
+def test_reward_mean_groups_and_bad_tokens(orc):
+    seq = np.array([[0, 1, -1], [2, 2, 2], [1, -1, -1], [0, 0, 1]], np.int32)
+    ln = np.array([2, 3, 1, 3], np.int32)
+    r = np.array([1.0, 10.0, 100.0])
+    lane, mean = orc.reward_mean(seq, ln, 2, r)
+    assert lane.tolist() == [11.0, 300.0, 10.0, 12.0] and mean.tolist() == [155.5, 11.0]
+    with pytest.raises(ValueError):
+        orc.reward_mean(np.array([[5]], np.int32), np.array([1], np.int32), 1, r)
