@@ -235,6 +235,43 @@ int as_encode_bigram(const void *d_table, int dtype, int V, long long ld,
                      double *d_lo, double *d_width, int32_t *d_lane_status, void *stream);
 
 /*
+ * n-gram diversity score of a set of sequences (Sec. 5.1, "Diverse beam
+ * generation"): d = sum_{n=1..4} d_n with
+ *   d_n = (number of distinct n-grams) / (number of n-grams) in the N sequences
+ * of a group.  Lanes g*N .. g*N+N-1 of d_seq form group g (the layout that
+ * as_decode_bigram writes for start token g).  An n-gram is n consecutive
+ * emitted tokens of one sequence; padding belongs to none.  A d_n whose
+ * denominator is zero contributes 0.
+ *   d_seq  [S*N, T] i32 device, read only;  d_len [S*N] i32 device (clamped to [0, T])
+ *   d_unique, d_total  [S, 4] i64 device, written: the counts for n = 1..4
+ *   d_div  [S] f64 device, written: d
+ * One group must fit shared memory: N * T <= AS_NGRAM_MAX_ITEMS, else
+ * AS_ERR_UNSUPPORTED.  Other errors: AS_ERR_INVALID_ARG (NULL pointer, S < 0,
+ * N < 1, T < 0), AS_ERR_CUDA.
+ */
+#define AS_NGRAM_MAX_ITEMS 16384
+int as_ngram_diversity(const int32_t *d_seq, const int32_t *d_len, int S, int N, int T,
+                       int64_t *d_unique, int64_t *d_total, double *d_div, void *stream);
+
+/*
+ * Sample-mean estimator of Sec. 4.2 (the proposition that (1/N) sum_i s(x_i)
+ * over the sequences of one shifted lattice is unbiased and consistent; used
+ * for the variance comparison of Sec. 5.2) for an additive reward
+ *   s(x) = sum_{t < len} d_r[x_t]:
+ *   d_lane_reward[lane] = s(x_lane)            (NULL to skip)
+ *   d_mean[g] = (1/N) sum of s over lanes g*N .. g*N+N-1
+ *   d_r  [V] f64 device;  d_seq, d_len as for as_ngram_diversity
+ *   d_group_status  NULL or [S] i32 device: AS_OK, or AS_ERR_INVALID_ARG if a
+ *                   token of the group lies outside [0, V) (it then adds nothing)
+ * Errors: AS_ERR_INVALID_ARG (NULL pointer, S < 0, N outside [1, AS_REWARD_MAX_N],
+ * T < 0, V < 1), AS_ERR_CUDA.
+ */
+#define AS_REWARD_MAX_N 4096
+int as_reward_mean(const int32_t *d_seq, const int32_t *d_len, int S, int N, int T,
+                   const double *d_r, int V, double *d_lane_reward, double *d_mean,
+                   int32_t *d_group_status, void *stream);
+
+/*
  * Launch-shape overrides for measurement sweeps (process-wide, not thread-safe;
  * 0 restores the built-in choice).  Keys:
  *   AS_TUNE_STEP_PATH     0 = streaming kernel (one CTA per lane), 1 = general kernel only,

@@ -36,7 +36,8 @@ TUNE_MIN_CTAS = 5
 
 EXPORTS = ["as_lattice_codes", "as_step", "as_step_host", "as_step_host_work_bytes", "as_step_host_static",
            "as_decode_bigram",
-           "as_decode_bigram_codes", "as_encode_bigram", "as_tune", "as_last_error", "as_version"]
+           "as_decode_bigram_codes", "as_encode_bigram", "as_ngram_diversity", "as_reward_mean", "as_tune",
+           "as_last_error", "as_version"]
 
 
 class AsError(RuntimeError):
@@ -78,10 +79,13 @@ def lib():
         L.as_decode_bigram.argtypes = [P, I, I, LL, P, I, I, D, I, I, D, I, D, P, P, P, P, P]
         L.as_decode_bigram_codes.argtypes = [P, I, I, LL, P, P, I, I, I, D, I, D, P, P, P, P, P]
         L.as_encode_bigram.argtypes = [P, I, I, LL, P, P, P, I, I, D, I, D, P, P, P, P]
+        L.as_ngram_diversity.argtypes = [P, P, I, I, I, P, P, P, P]
+        L.as_reward_mean.argtypes = [P, P, I, I, I, P, I, P, P, P, P]
         L.as_tune.argtypes = [I, I]
         L.as_last_error.restype = ctypes.c_char_p
         for n in ("as_lattice_codes", "as_step", "as_step_host", "as_decode_bigram",
-                  "as_decode_bigram_codes", "as_encode_bigram", "as_tune", "as_version"):
+                  "as_decode_bigram_codes", "as_encode_bigram", "as_ngram_diversity", "as_reward_mean", "as_tune",
+                  "as_version"):
             getattr(L, n).restype = I
         _lib = L
     return _lib
@@ -256,3 +260,38 @@ def as_encode_bigram(table: torch.Tensor, prev: torch.Tensor, seq: torch.Tensor,
                                   lanes, T, temp, top_k, top_p, _ptr(lo), _ptr(width), _ptr(lane_status),
                                   _stream(stream)))
     return lo, width
+
+
+def _groups(seq: torch.Tensor, length: torch.Tensor, N: int):
+    if seq.dim() != 2 or not seq.is_contiguous() or seq.dtype != torch.int32:
+        raise ValueError("seq must be a contiguous [lanes, T] int32 tensor")
+    lanes, T = seq.shape
+    if N < 1 or lanes % N or length.numel() != lanes:
+        raise ValueError("lanes must be a multiple of N, with one length per lane")
+    return lanes // N, T
+
+
+def as_ngram_diversity(seq: torch.Tensor, length: torch.Tensor, N: int, stream=None):
+    """(unique[S,4], total[S,4], d[S]): n-gram diversity of each group of N lanes (Sec. 5.1)."""
+    S, T = _groups(seq, length, N)
+    dev = seq.device
+    unique = torch.empty((S, 4), dtype=torch.int64, device=dev)
+    total = torch.empty((S, 4), dtype=torch.int64, device=dev)
+    d = torch.empty(S, dtype=torch.float64, device=dev)
+    _check(lib().as_ngram_diversity(_ptr(seq), _ptr(length), S, N, T, _ptr(unique), _ptr(total), _ptr(d),
+                                    _stream(stream)))
+    return unique, total, d
+
+
+def as_reward_mean(seq: torch.Tensor, length: torch.Tensor, N: int, r: torch.Tensor,
+                   group_status: Optional[torch.Tensor] = None, stream=None):
+    """(lane_reward[lanes], mean[S]) for the additive reward r[token] (Sec. 4.2 estimator)."""
+    S, T = _groups(seq, length, N)
+    if r.dtype != torch.float64 or not r.is_contiguous():
+        raise ValueError("r must be a contiguous float64 tensor")
+    dev = seq.device
+    lane_reward = torch.empty(S * N, dtype=torch.float64, device=dev)
+    mean = torch.empty(S, dtype=torch.float64, device=dev)
+    _check(lib().as_reward_mean(_ptr(seq), _ptr(length), S, N, T, _ptr(r), r.numel(), _ptr(lane_reward),
+                                _ptr(mean), _ptr(group_status), _stream(stream)))
+    return lane_reward, mean

@@ -1,6 +1,7 @@
 // C-ABI entry points (see include/arith_sampling.h) and the kernels behind them.
 #include "../../include/arith_sampling.h"
 #include "as_stream.cuh"
+#include "as_metrics.cuh"
 
 #include <cmath>
 #include <cstdarg>
@@ -585,6 +586,62 @@ int as_encode_bigram(const void* d_table, int dtype, int V, long long ld, const 
         encode_generic_kernel<DT_BF16><<<grid, GEN_NT, 0, st>>>(d_table, V, ld, d_prev, d_seq, d_len, lanes, T, inv_tau, top_k, top_p, d_lo, d_width, d_lane_status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "encode kernel launch");
+    return AS_OK;
+}
+
+int as_ngram_diversity(const int32_t* d_seq, const int32_t* d_len, int S, int N, int T,
+                       int64_t* d_unique, int64_t* d_total, double* d_div, void* stream) {
+    if (S < 0) return set_err(AS_ERR_INVALID_ARG, "S = %d must be >= 0", S);
+    if (N < 1) return set_err(AS_ERR_INVALID_ARG, "N = %d must be >= 1", N);
+    if (T < 0) return set_err(AS_ERR_INVALID_ARG, "T = %d must be >= 0", T);
+    if ((long long)N * T > AS_NGRAM_MAX_ITEMS)
+        return set_err(AS_ERR_UNSUPPORTED, "N * T = %lld exceeds AS_NGRAM_MAX_ITEMS = %d", (long long)N * T, AS_NGRAM_MAX_ITEMS);
+    if (S == 0) return AS_OK;
+    if (!d_len || !d_unique || !d_total || !d_div || (!d_seq && T > 0))
+        return set_err(AS_ERR_INVALID_ARG, "d_seq, d_len, d_unique, d_total or d_div is NULL");
+    const DeviceInfo* di;
+    int rc = device_info(&di);
+    if (rc != AS_OK) return rc;
+    const int items = N * T;
+    int cap = 64;
+    while (cap < 2 * items) cap <<= 1;
+    const size_t smem = sizeof(int) * ((size_t)items + N + cap);
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaError_t e;
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(ngram_diversity_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_OPTIN_MAX - 1024));
+        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(max dynamic shared memory)");
+        attr_set[dev] = true;
+    }
+    if (smem > SMEM_OPTIN_MAX - 1024) return set_err(AS_ERR_UNSUPPORTED, "group of %d x %d tokens does not fit shared memory", N, T);
+    const int grid = S < di->sms * 2 ? S : di->sms * 2;
+    ngram_diversity_kernel<<<grid, NG_NT, smem, (cudaStream_t)stream>>>(d_seq, d_len, S, N, T, cap,
+                                                                        reinterpret_cast<long long*>(d_unique),
+                                                                        reinterpret_cast<long long*>(d_total), d_div);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "n-gram diversity kernel launch");
+    return AS_OK;
+}
+
+int as_reward_mean(const int32_t* d_seq, const int32_t* d_len, int S, int N, int T, const double* d_r, int V,
+                   double* d_lane_reward, double* d_mean, int32_t* d_group_status, void* stream) {
+    if (S < 0) return set_err(AS_ERR_INVALID_ARG, "S = %d must be >= 0", S);
+    if (N < 1 || N > AS_REWARD_MAX_N) return set_err(AS_ERR_INVALID_ARG, "N = %d must lie in [1, %d]", N, AS_REWARD_MAX_N);
+    if (T < 0) return set_err(AS_ERR_INVALID_ARG, "T = %d must be >= 0", T);
+    if (V < 1) return set_err(AS_ERR_INVALID_ARG, "V = %d must be >= 1", V);
+    if (S == 0) return AS_OK;
+    if (!d_len || !d_r || !d_mean || (!d_seq && T > 0))
+        return set_err(AS_ERR_INVALID_ARG, "d_seq, d_len, d_r or d_mean is NULL");
+    const DeviceInfo* di;
+    int rc = device_info(&di);
+    if (rc != AS_OK) return rc;
+    const int grid = S < di->sms * 8 ? S : di->sms * 8;
+    reward_mean_kernel<<<grid, RM_NT, sizeof(double) * (size_t)N, (cudaStream_t)stream>>>(
+        d_seq, d_len, S, N, T, d_r, V, d_lane_reward, d_mean, d_group_status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "reward mean kernel launch");
     return AS_OK;
 }
 

@@ -70,6 +70,16 @@ def test_invalid_arguments_are_rejected_on_the_host(L):
     assert enc(seq=None) == B.ERR_INVALID_ARG
     assert enc(lo=None) == B.ERR_INVALID_ARG
     assert enc(lanes=0) == B.OK
+    div = lambda **k: L.as_ngram_diversity(k.get("seq", p), p, k.get("S", 1), k.get("N", 2), k.get("T", 4), p, p,
+                                           k.get("d", p), None)
+    assert div(S=-1) == B.ERR_INVALID_ARG and div(N=0) == B.ERR_INVALID_ARG and div(T=-1) == B.ERR_INVALID_ARG
+    assert div(seq=None) == B.ERR_INVALID_ARG and div(d=None) == B.ERR_INVALID_ARG
+    assert div(N=32, T=1024) == B.ERR_UNSUPPORTED and div(S=0) == B.OK
+    rm = lambda **k: L.as_reward_mean(k.get("seq", p), p, k.get("S", 1), k.get("N", 2), k.get("T", 4), k.get("r", p),
+                                      k.get("V", 3), None, k.get("mean", p), None, None)
+    assert rm(S=-1) == B.ERR_INVALID_ARG and rm(N=0) == B.ERR_INVALID_ARG and rm(N=5000) == B.ERR_INVALID_ARG
+    assert rm(V=0) == B.ERR_INVALID_ARG and rm(r=None) == B.ERR_INVALID_ARG and rm(mean=None) == B.ERR_INVALID_ARG
+    assert rm(S=0) == B.OK
     assert L.as_tune(99, 0) == B.ERR_INVALID_ARG and L.as_tune(B.TUNE_CLUSTER, 3) == B.ERR_INVALID_ARG
     assert L.as_step_host_work_bytes(0, 4, 10) >= 4 * 10 * 4 + 4 * 24
 
