@@ -321,6 +321,41 @@ def bench_bigram(steps: int, warmup: int, S: int = 64):
     ms = a.elapsed_time(b) / steps
     tokens = int(ln.sum().item())
     out["encode"] = {"ms_per_encode": ms, "tokens": tokens, "tokens_per_s": tokens / ms * 1e3}
+    # what is computed from the decoded groups: n-gram diversity (Sec. 5.1) and the sample-mean
+    # estimator of an additive synthetic reward (Sec. 4.2 / 5.2), lattice codes against iid codes
+    r = torch.from_numpy(synth.reward_table(w.V, 78)).cuda()
+
+    def timed_call(fn, reps=20):
+        fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    K = 16
+    shifts = np.random.default_rng(79).random(K)
+    stats = {}
+    for name in ("lattice", "iid"):
+        means, divs = [], []
+        for k in range(K):
+            if name == "lattice":
+                B.as_decode_bigram(table, starts, w.N, float(shifts[k]), w.T, w.eos, w.temp, w.top_k, w.top_p,
+                                   seq=seq, length=ln)
+            else:
+                codes = torch.from_numpy(synth.iid_codes(w.lanes, 1000 + k)).cuda()
+                B.as_decode_bigram_codes(table, prev, codes, w.T, w.eos, w.temp, w.top_k, w.top_p, seq=seq, length=ln)
+            means.append(B.as_reward_mean(seq, ln, w.N, r)[1])
+            divs.append(B.as_ngram_diversity(seq, ln, w.N)[2])
+        means, divs = torch.stack(means), torch.stack(divs)
+        stats[name] = {"estimator_sd_over_%d_runs_mean_over_groups" % K: float(means.std(dim=0).mean().item()),
+                       "ngram_diversity_mean": float(divs.mean().item())}
+    stats["ms_ngram_diversity"] = timed_call(lambda: B.as_ngram_diversity(seq, ln, w.N))
+    stats["ms_reward_mean"] = timed_call(lambda: B.as_reward_mean(seq, ln, w.N, r))
+    out["groups"] = stats
     out["workload"] = "c4: bf16 bigram table 32128x32128, %d starts x 32 codes, T<=128, temp 0.8, EOS 1" % S
     return out
 

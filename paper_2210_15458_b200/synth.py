@@ -199,3 +199,8 @@ def c4(eos_bias: Optional[float] = None, V: int = 32128, S: int = 64, T: int = 1
 def c5(lanes: int = 1024) -> StepWorkload:
     return StepWorkload("c5", lanes=lanes, V=256000, dtype=BF16, sigma=3.0, temp=0.8, top_k=64,
                         top_p=0.95, seed_logits=50, seed_perm=51, seed_shift=52, N=lanes)
+
+
+def reward_table(V: int, seed: int) -> np.ndarray:
+    """Per-token rewards r[v] ~ N(0, 1) for the additive sequence reward of the estimator runs."""
+    return np.random.default_rng(seed).normal(0.0, 1.0, V)
