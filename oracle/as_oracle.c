@@ -243,6 +243,32 @@ int orc_lattice_codes(long N, double u, double *codes)
  * One decode step for lanes [lane_begin, lane_end) of logits[lanes, ld].
  * Any output pointer may be NULL.  Outputs are indexed by absolute lane.
  */
+/*
+ * The code sets the paper itself writes down, as variants of the lattice above:
+ *   variant 1  Definition "Arithmetic sampling" (Sec. 4.2) as printed:
+ *              c_i = (i/(N+1) + b) mod 1, i = 1..N, one shared b in [0,1);
+ *   variant 2  the naive codebook of the proposition "Naive arithmetic
+ *              sampling" (Sec. 4.2): c_i = i/(N+1), i = 1..N, no shift (the
+ *              example after it: N = 1 gives the single code 0.5).
+ * codes[i-1] receives c_i.  Variant 0 is orc_lattice_codes.
+ */
+int orc_lattice_codes_variant(long N, double b, long variant, double *codes)
+{
+    long i;
+    if (variant == 0) return orc_lattice_codes(N, b, codes);
+    if (N < 1 || !codes || (variant != 1 && variant != 2)) return ORC_ERR_INVALID_ARG;
+    if (variant == 1 && !(b >= 0.0 && b < 1.0)) return ORC_ERR_INVALID_ARG;
+    for (i = 1; i <= N; ++i) {
+        double c = (double)i / (double)(N + 1);
+        if (variant == 1) {
+            c += b;
+            if (c >= 1.0) c -= 1.0;
+        }
+        codes[i - 1] = c;
+    }
+    return ORC_OK;
+}
+
 int orc_step(const void *logits, int dtype, long lanes, long V, long ld,
              const double *codes, double temp, long top_k, double top_p,
              int32_t *tokens, double *codes_out, double *p_tok, double *cdf_lo,

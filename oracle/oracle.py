@@ -53,6 +53,8 @@ def lib():
                                                  + [P] * 8 + [L, L])
         _lib.orc_decode_bigram.argtypes = [P, ctypes.c_int, L, L, P, L, L, D, L, L, D, L, D, P, P, P, P]
         _lib.orc_encode_bigram.argtypes = [P, ctypes.c_int, L, L, P, P, P, L, L, D, L, D, P, P, P]
+        _lib.orc_lattice_codes_variant.argtypes = [L, D, L, P]
+        _lib.orc_lattice_codes_variant.restype = ctypes.c_int
         _lib.orc_ngram_diversity.argtypes = [P, P, L, L, L, P, P, P]
         _lib.orc_reward_mean.argtypes = [P, P, L, L, L, P, L, P, P]
         for f in (_lib.orc_lattice_codes, _lib.orc_step, _lib.orc_decode_bigram_codes,
@@ -98,6 +100,15 @@ def lattice_codes(N: int, u: float) -> np.ndarray:
     rc = lib().orc_lattice_codes(N, u, _ptr(out))
     if rc != OK:
         raise ValueError("orc_lattice_codes: invalid argument")
+    return out
+
+
+def lattice_codes_variant(N: int, b: float, variant: int) -> np.ndarray:
+    """variant 0: (j+b)/N; 1: (i/(N+1) + b) mod 1; 2: i/(N+1) (no shift)."""
+    out = np.empty(max(N, 0), dtype=np.float64)
+    rc = lib().orc_lattice_codes_variant(N, b, variant, _ptr(out))
+    if rc != OK:
+        raise ValueError("orc_lattice_codes_variant: invalid argument")
     return out
 
 

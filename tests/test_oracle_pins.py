@@ -557,3 +557,41 @@ def test_reward_mean_groups_and_bad_tokens(orc):
     assert lane.tolist() == [11.0, 300.0, 10.0, 12.0] and mean.tolist() == [155.5, 11.0]
     with pytest.raises(ValueError):
         orc.reward_mean(np.array([[5]], np.int32), np.array([1], np.int32), 1, r)
+
+
+# --------------------------------------------------------------------------- the paper's own code sets
+def test_lattice_variants_closed_forms(orc):
+    for N in (1, 2, 5, 16, 257):
+        naive = orc.lattice_codes_variant(N, 0.0, 2)
+        assert naive.tolist() == [float(Fraction(i, N + 1)) for i in range(1, N + 1)]
+        for b in (0.0, 0.25, 0.999):
+            got = orc.lattice_codes_variant(N, b, 1)
+            want = [(Fraction(i, N + 1) + Fraction(b)) % 1 for i in range(1, N + 1)]
+            assert got == pytest.approx([float(w) for w in want], abs=2e-16)
+            assert ((got >= 0) & (got < 1)).all()
+            # on the circle: N - 1 gaps of 1/(N+1) and one of 2/(N+1) -- unlike variant 0, whose
+            # gaps are all 1/N; this is why the bounds of Sec. 4.3 are stated for variant 0
+            srt = np.sort(got)
+            gaps = np.diff(np.concatenate([srt, [srt[0] + 1.0]]))
+            assert np.sort(gaps)[:-1] == pytest.approx(1.0 / (N + 1), abs=1e-12) or N == 1
+            assert gaps.max() == pytest.approx(2.0 / (N + 1), abs=1e-12)
+        assert (orc.lattice_codes_variant(N, 0.3, 0) == orc.lattice_codes(N, 0.3)).all()
+    with pytest.raises(ValueError):
+        orc.lattice_codes_variant(4, 0.5, 3)
+    with pytest.raises(ValueError):
+        orc.lattice_codes_variant(4, 1.0, 1)
+
+
+def test_naive_codebook_example_is_biased_but_consistent(orc):
+    # the example after the proposition "Naive arithmetic sampling": symbols A (0.6) and B (0.4),
+    # N = 1 gives the code 0.5, which always decodes to A: the sample mean of 1[B] is 0, not 0.4
+    table = _rows([np.log([0.6, 0.4])] * 2)
+    c = orc.lattice_codes_variant(1, 0.0, 2)
+    assert c.tolist() == [0.5]
+    o = orc.decode_bigram_codes(table, F32, np.array([0], np.int32), c, 1, -1)
+    assert o.seq[0, 0] == 0
+    # consistency (Eq. of that proposition): the mean over N naive codes tends to E[s] as 1/N
+    for N in (10, 100, 1000):
+        codes = orc.lattice_codes_variant(N, 0.0, 2)
+        o = orc.decode_bigram_codes(table, F32, np.zeros(N, np.int32), codes, 1, -1)
+        assert abs((o.seq[:, 0] == 1).mean() - 0.4) <= 1.0 / N
