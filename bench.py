@@ -262,12 +262,12 @@ def cpu_baseline_step(w, budget_s: float = 12.0):
 
 
 # ----------------------------------------------------------------------------- bigram workload (c4)
-def bench_bigram(steps: int, warmup: int, S: int = 64):
+def bench_bigram(steps: int, warmup: int, S: int = 64, T: int = 128):
     """tokens/s of the full decode loop over the 32128 x 32128 bf16 bigram table, lattice
     codes versus iid codes (ordinary ancestral sampling through the same kernel)."""
     import torch
     from paper_2210_15458_b200 import binding as B
-    w = synth.c4(S=S)
+    w = synth.c4(S=S, T=T)
     table = to_dev(w.table(), w.dtype)
     starts = torch.from_numpy(w.starts()).cuda()
     out = {}
@@ -285,7 +285,7 @@ def bench_bigram(steps: int, warmup: int, S: int = 64):
     def dup_rates(s):
         s = s.cpu().numpy().reshape(w.S, w.N, w.T)
         res = {}
-        for L in (1, 2, 4, 8, w.T):
+        for L in (1, 2, 4, 8, 128):
             r = [1.0 - len({tuple(x[:L]) for x in grp}) / w.N for grp in s]
             res[str(L)] = float(np.mean(r))
         return res
@@ -337,6 +337,7 @@ def bench_bigram(steps: int, warmup: int, S: int = 64):
         return a.elapsed_time(b) / reps
 
     K = 16
+    fits = w.N * w.T <= B.NGRAM_MAX_ITEMS          # one group's tokens and hash table in shared memory
     shifts = np.random.default_rng(79).random(K)
     stats = {}
     for name in ("lattice", "iid"):
@@ -349,14 +350,15 @@ def bench_bigram(steps: int, warmup: int, S: int = 64):
                 codes = torch.from_numpy(synth.iid_codes(w.lanes, 1000 + k)).cuda()
                 B.as_decode_bigram_codes(table, prev, codes, w.T, w.eos, w.temp, w.top_k, w.top_p, seq=seq, length=ln)
             means.append(B.as_reward_mean(seq, ln, w.N, r)[1])
-            divs.append(B.as_ngram_diversity(seq, ln, w.N)[2])
-        means, divs = torch.stack(means), torch.stack(divs)
+            if fits:
+                divs.append(B.as_ngram_diversity(seq, ln, w.N)[2])
+        means = torch.stack(means)
         stats[name] = {"estimator_sd_over_%d_runs_mean_over_groups" % K: float(means.std(dim=0).mean().item()),
-                       "ngram_diversity_mean": float(divs.mean().item())}
-    stats["ms_ngram_diversity"] = timed_call(lambda: B.as_ngram_diversity(seq, ln, w.N))
+                       "ngram_diversity_mean": float(torch.stack(divs).mean().item()) if fits else None}
+    stats["ms_ngram_diversity"] = timed_call(lambda: B.as_ngram_diversity(seq, ln, w.N)) if fits else None
     stats["ms_reward_mean"] = timed_call(lambda: B.as_reward_mean(seq, ln, w.N, r))
     out["groups"] = stats
-    out["workload"] = "c4: bf16 bigram table 32128x32128, %d starts x 32 codes, T<=128, temp 0.8, EOS 1" % S
+    out["workload"] = "c4: bf16 bigram table 32128x32128, %d starts x 32 codes, T<=%d, temp 0.8, EOS 1" % (S, T)
     return out
 
 
@@ -496,13 +498,15 @@ def main():
                     help="c4 prints the bigram decode / encode loop's own line (a side measurement)")
     ap.add_argument("--lanes", type=int, default=None,
                     help="lanes for c3 / c5 / c4 (default: the configured size; c4: a multiple of 32)")
+    ap.add_argument("--T", type=int, default=128, help="c4 only: maximum steps per lane (512-1024: summarisation-sized outputs)")
     ap.add_argument("--no-extras", action="store_true", help="skip the other workloads' short measurements")
     args = ap.parse_args()
     args.warmup = max(3, args.warmup)
     if args.workload == "c4":
         if args.impl == "reference" or dist_env()[2] > 1:
             raise SystemExit("--workload c4 is a single-GPU side measurement of the CUDA path")
-        print(json.dumps(bench_bigram(min(args.steps, 20), min(args.warmup, 3), S=(args.lanes or 2048) // 32)))
+        print(json.dumps(bench_bigram(min(args.steps, 20), min(args.warmup, 3), S=(args.lanes or 2048) // 32,
+                                      T=args.T)))
     elif args.impl == "reference":
         run_reference(args)
     else:

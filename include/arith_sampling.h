@@ -98,6 +98,25 @@ typedef struct as_step_diag {
 int as_lattice_codes(int N, double u, double *d_codes, void *stream);
 
 /*
+ * The code sets in the forms the paper itself prints (Sec. 4.2), next to the
+ * evenly spaced one above:
+ *   AS_LATTICE_SHIFTED           (j + b)/N mod 1, j = 0..N-1: as_lattice_codes
+ *   AS_LATTICE_PAPER_DEFINITION  (i/(N+1) + b) mod 1, i = 1..N: Definition
+ *                                "Arithmetic sampling" as printed (on the circle
+ *                                its wrap gap is 2/(N+1), the others 1/(N+1))
+ *   AS_LATTICE_NAIVE             i/(N+1), i = 1..N, no shift (b ignored): the
+ *                                codebook of the proposition "Naive arithmetic
+ *                                sampling" -- consistent but biased
+ * d_codes[i-1] = c_i, [N] f64 device.  Feed the codes to as_step or
+ * as_decode_bigram_codes.  Errors: AS_ERR_INVALID_ARG for an unknown variant,
+ * N < 1, b outside [0,1) where it is used, NULL d_codes.
+ */
+#define AS_LATTICE_SHIFTED 0
+#define AS_LATTICE_PAPER_DEFINITION 1
+#define AS_LATTICE_NAIVE 2
+int as_lattice_codes_variant(int N, double b, int variant, double *d_codes, void *stream);
+
+/*
  * One decode step for every lane (the loop body of Algorithm 1, with the logit
  * modifiers named in Sec. 2 and "Top-k sampling", Sec. 5.1):
  *   x_j = logits[lane, j] / temp; optional top-k and nucleus cuts; p = softmax

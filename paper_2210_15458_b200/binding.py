@@ -34,7 +34,7 @@ TUNE_CTAS_PER_SM = 3
 TUNE_STAGES = 4
 TUNE_MIN_CTAS = 5
 
-EXPORTS = ["as_lattice_codes", "as_step", "as_step_host", "as_step_host_work_bytes", "as_step_host_static",
+EXPORTS = ["as_lattice_codes", "as_lattice_codes_variant", "as_step", "as_step_host", "as_step_host_work_bytes", "as_step_host_static",
            "as_decode_bigram",
            "as_decode_bigram_codes", "as_encode_bigram", "as_ngram_diversity", "as_reward_mean", "as_tune",
            "as_last_error", "as_version"]
@@ -79,6 +79,8 @@ def lib():
         L.as_decode_bigram.argtypes = [P, I, I, LL, P, I, I, D, I, I, D, I, D, P, P, P, P, P]
         L.as_decode_bigram_codes.argtypes = [P, I, I, LL, P, P, I, I, I, D, I, D, P, P, P, P, P]
         L.as_encode_bigram.argtypes = [P, I, I, LL, P, P, P, I, I, D, I, D, P, P, P, P]
+        L.as_lattice_codes_variant.argtypes = [I, D, I, P, P]
+        L.as_lattice_codes_variant.restype = I
         L.as_ngram_diversity.argtypes = [P, P, I, I, I, P, P, P, P]
         L.as_reward_mean.argtypes = [P, P, I, I, I, P, I, P, P, P, P]
         L.as_tune.argtypes = [I, I]
@@ -132,6 +134,18 @@ def as_lattice_codes(N: int, u: float, out: Optional[torch.Tensor] = None, strea
     if out is None:
         out = torch.empty(max(N, 0), dtype=torch.float64, device="cuda")
     _check(lib().as_lattice_codes(N, u, _ptr(out), _stream(stream)))
+    return out
+
+
+LATTICE_SHIFTED, LATTICE_PAPER_DEFINITION, LATTICE_NAIVE = 0, 1, 2
+NGRAM_MAX_ITEMS = 16384     # AS_NGRAM_MAX_ITEMS
+
+
+def as_lattice_codes_variant(N: int, b: float, variant: int, out: Optional[torch.Tensor] = None,
+                             stream=None) -> torch.Tensor:
+    if out is None:
+        out = torch.empty(max(N, 0), dtype=torch.float64, device="cuda")
+    _check(lib().as_lattice_codes_variant(N, b, variant, _ptr(out), _stream(stream)))
     return out
 
 

@@ -162,6 +162,20 @@ __global__ void lattice_kernel(int N, double u, double* __restrict__ codes) {
     }
 }
 
+// The code sets as the paper prints them (Sec. 4.2): variant 1 = (i/(N+1) + b) mod 1, the Definition
+// "Arithmetic sampling"; variant 2 = i/(N+1), the naive codebook; i = 1..N, codes[i-1] = c_i.
+__global__ void lattice_variant_kernel(int N, double b, int variant, double* __restrict__ codes) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x + 1;
+    if (i <= N) {
+        double c = (double)i / (double)(N + 1);
+        if (variant == 1) {
+            c += b;
+            if (c >= 1.0) c -= 1.0;
+        }
+        codes[i - 1] = c;
+    }
+}
+
 template <int DT>
 __global__ void __launch_bounds__(GEN_NT)
 step_generic_kernel(const void* __restrict__ logits, int lanes, int V, long long ld,
@@ -350,6 +364,23 @@ int as_lattice_codes(int N, double u, double* d_codes, void* stream) {
     int rc = device_info(&di);
     if (rc != AS_OK) return rc;
     lattice_kernel<<<(N + 255) / 256, 256, 0, (cudaStream_t)stream>>>(N, u, d_codes);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "lattice kernel launch");
+    return AS_OK;
+}
+
+int as_lattice_codes_variant(int N, double b, int variant, double* d_codes, void* stream) {
+    if (variant == AS_LATTICE_SHIFTED) return as_lattice_codes(N, b, d_codes, stream);
+    if (variant != AS_LATTICE_PAPER_DEFINITION && variant != AS_LATTICE_NAIVE)
+        return set_err(AS_ERR_INVALID_ARG, "unknown lattice variant %d", variant);
+    if (N < 1) return set_err(AS_ERR_INVALID_ARG, "N = %d must be >= 1", N);
+    if (variant == AS_LATTICE_PAPER_DEFINITION && !(b >= 0.0 && b < 1.0))
+        return set_err(AS_ERR_INVALID_ARG, "shift b must lie in [0,1)");
+    if (!d_codes) return set_err(AS_ERR_INVALID_ARG, "d_codes is NULL");
+    const DeviceInfo* di;
+    int rc = device_info(&di);
+    if (rc != AS_OK) return rc;
+    lattice_variant_kernel<<<(N + 255) / 256, 256, 0, (cudaStream_t)stream>>>(N, b, variant, d_codes);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "lattice kernel launch");
     return AS_OK;

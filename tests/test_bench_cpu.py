@@ -46,3 +46,35 @@ def test_reference_arm_other_ranks_do_nothing():
     p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1"],
                        capture_output=True, text=True, timeout=120, env=env)
     assert p.returncode == 0 and p.stdout.strip() == ""
+
+
+def _gather_worker(rank, world, port, out):
+    import torch
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    from paper_2210_15458_b200 import shard
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    n_total, T = 7, 5                                   # 7 lanes over 2 ranks: shards of 4 and 3
+    lo, hi = shard.shard_range(n_total, rank, world)
+    full = torch.arange(n_total * T, dtype=torch.int32).reshape(n_total, T)
+    lens = torch.arange(n_total, dtype=torch.int32) % (T + 1)
+    seq, length = shard.gather_sequences(full[lo:hi].clone(), lens[lo:hi].clone(), n_total)
+    out[rank] = (lo, hi, bool((seq == full).all()), bool((length == lens).all()))
+    dist.destroy_process_group()
+
+
+def test_lane_shards_and_the_final_gather_two_processes():
+    sys.path.insert(0, ROOT)
+    from paper_2210_15458_b200 import shard
+    for n in (0, 1, 7, 64, 1000):
+        for world in (1, 2, 3, 8):
+            cuts = [shard.shard_range(n, r, world) for r in range(world)]
+            assert cuts[0][0] == 0 and cuts[-1][1] == n
+            assert all(cuts[r][1] == cuts[r + 1][0] for r in range(world - 1))
+            sizes = [b - a for a, b in cuts]
+            assert max(sizes) - min(sizes) <= 1
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_gather_worker, args=(2, 29741, out), nprocs=2, join=True)
+    assert out[0] == (0, 4, True, True) and out[1] == (4, 7, True, True)

@@ -138,3 +138,20 @@ def test_estimator_has_zero_variance_on_a_lattice_matched_model(B):
         assert mean.cpu().numpy() == pytest.approx(want, abs=1e-13)
         un, tot, d = B.as_ngram_diversity(seq, ln, 8)
         assert un.cpu().tolist() == [[4, 0, 0, 0]] * 3 and tot.cpu().tolist() == [[8, 0, 0, 0]] * 3
+
+
+@pytest.mark.parametrize("N", [1, 2, 31, 256, 1000, 70001])
+def test_lattice_variants_bit_exact(B, orc, N):
+    for variant, b in [(0, 0.3), (1, 0.0), (1, 0.617), (1, 0.999999), (2, 0.0), (2, 0.4)]:
+        got = B.as_lattice_codes_variant(N, b, variant).cpu().numpy()
+        assert (got == orc.lattice_codes_variant(N, b, variant)).all()
+
+
+def test_naive_codebook_bias_example_on_the_gpu(B):
+    # the example after the proposition "Naive arithmetic sampling": N = 1 gives the code 0.5,
+    # which decodes to the symbol of probability 0.6 every time
+    table = torch.from_numpy(np.tile(np.log([0.6, 0.4, 1e-30, 1e-30]).astype(np.float32), (4, 1))).cuda()
+    codes = B.as_lattice_codes_variant(1, 0.0, B.LATTICE_NAIVE)
+    assert codes.cpu().tolist() == [0.5]
+    seq, ln = B.as_decode_bigram_codes(table, torch.zeros(1, dtype=torch.int32, device="cuda"), codes, 1, -1)
+    assert seq.cpu().tolist() == [[0]]

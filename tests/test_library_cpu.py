@@ -41,6 +41,10 @@ def test_invalid_arguments_are_rejected_on_the_host(L):
     assert L.as_lattice_codes(4, 1.0, p, None) == B.ERR_INVALID_ARG
     assert L.as_lattice_codes(4, float("nan"), p, None) == B.ERR_INVALID_ARG
     assert L.as_lattice_codes(4, 0.5, None, None) == B.ERR_INVALID_ARG
+    assert L.as_lattice_codes_variant(4, 0.5, 7, p, None) == B.ERR_INVALID_ARG
+    assert L.as_lattice_codes_variant(0, 0.5, 1, p, None) == B.ERR_INVALID_ARG
+    assert L.as_lattice_codes_variant(4, 1.0, 1, p, None) == B.ERR_INVALID_ARG
+    assert L.as_lattice_codes_variant(4, 0.5, 2, None, None) == B.ERR_INVALID_ARG
     step = lambda **k: L.as_step(k.get("logits", p), k.get("dtype", 0), k.get("lanes", 1), k.get("V", 2),
                                  k.get("ld", 2), k.get("codes", p), k.get("temp", 1.0), 0,
                                  k.get("top_p", 1.0), k.get("tokens", p), k.get("out", p), None, None)
