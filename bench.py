@@ -4,7 +4,8 @@
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c5|c4] [--impl reference]
 
 A step is one pass of the decode hot path over one batch of synthetic input: a fresh
-shifted lattice of codes (as_lattice_codes) and one decode step for every lane (as_step).
+shifted lattice of codes and one decode step for every lane, in one launch (as_step_lattice
+forms the codes in the step kernel; the two-call form is timed beside it).
 The default workload is the 256-lane x 32000-token bf16 step (temperature 0.7, top_k 40).
 Rank 0 prints ONE JSON line; see README/DESIGN for the keys.  With N > 1 (torchrun) every
 rank decodes its own batch (lanes never communicate), so scaling is weak and there is no
@@ -162,13 +163,21 @@ class StepBench:
         self.host_base = base
         self.ring_bytes = nbuf * total
         self.shifts = np.random.default_rng(1234 + rank).random(4096)
-        self.codes = torch.empty(w.N, dtype=torch.float64, device="cuda")
+        self.codes = B.as_lattice_codes(w.N, float(self.shifts[0]))      # for the calls that read stored codes
         self.tokens = torch.empty(w.lanes, dtype=torch.int32, device="cuda")
         self.codes_out = torch.empty(w.lanes, dtype=torch.float64, device="cuda")
         self.i = 0
 
     def step(self):
-        """One pass of the hot path: lattice codes for a fresh shift, then the decode step."""
+        """One pass of the hot path: the lattice codes of a fresh shift, formed in the step kernel
+        (as_step_lattice: the same values as_lattice_codes would write), and the decode step."""
+        B, w = self.B, self.w
+        B.as_step_lattice(self.ring[self.i % len(self.ring)], w.N, float(self.shifts[self.i % 4096]), 0,
+                          w.temp, w.top_k, w.top_p, tokens=self.tokens, codes_out=self.codes_out)
+        self.i += 1
+
+    def step_two_calls(self):
+        """The same pass as two launches: as_lattice_codes, then as_step on the stored codes."""
         B, w = self.B, self.w
         B.as_lattice_codes(w.N, float(self.shifts[self.i % 4096]), out=self.codes)
         B.as_step(self.ring[self.i % len(self.ring)], self.codes[: w.lanes], w.temp, w.top_k, w.top_p,
@@ -395,6 +404,7 @@ def run_ours(args):
         sb.step_kernel_only()
     kern_launches = max(args.steps, 200)
     kms = sb.timed(sb.step_kernel_only, kern_launches) / kern_launches
+    ms2 = sb.timed(sb.step_two_calls, kern_launches) / kern_launches
     clocks = sampler.stop() if rank == 0 else None
     if rank != 0:
         if world > 1:
@@ -412,10 +422,12 @@ def run_ours(args):
                                % (w.name, w.lanes, w.V, "bf16" if w.dtype else "f32", w.temp, w.top_k, w.top_p),
                    "lanes_per_gpu": w.lanes, "V": w.V, "l2": "inputs rotate through %d buffers (%.0f MB > 3x L2)"
                                                              % (len(sb.ring), sb.ring_bytes / 1e6),
+                   "step": "one as_step_lattice launch: lattice codes of a fresh shift formed in the step kernel",
                    "timing": "K steps captured in one CUDA graph, replayed once between events",
                    "parallelism": "lanes sharded, no collective"},
         "lane_steps_per_s": w.lanes * world * args.steps / (ms / 1e3),
-        "gpu_launches": 2 * args.steps,
+        "gpu_launches": args.steps,
+        "ms_per_step_two_calls": ms2,          # as_lattice_codes + as_step on the stored codes
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "as_step", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": peak_kind, "frac_of_8TBs_nominal": achieved / 8000.0,

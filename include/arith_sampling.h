@@ -141,6 +141,21 @@ int as_step(const void *d_logits, int dtype, int lanes, int V, long long ld,
             void *stream);
 
 /*
+ * The first step of a decode (Algorithm 1 entered with the codes of the
+ * Definition "Arithmetic sampling", Sec. 4.2): as_step with lane i taking the
+ * lattice code c = (j0 + i + u)/N mod 1 formed in the kernel -- bit-identical to
+ * the value as_lattice_codes writes for index j0 + i -- so that the codes need
+ * not be written out and read back.  j0 lets a caller that shards the N lanes
+ * of one lattice over several devices give each its slice.
+ *   N >= 1, u in [0,1), j0 >= 0, j0 + lanes <= N; everything else as as_step.
+ * Errors: as as_step, plus AS_ERR_INVALID_ARG for N, u, j0 out of range.
+ */
+int as_step_lattice(const void *d_logits, int dtype, int lanes, int V, long long ld,
+                    int N, double u, int j0, double temp, int top_k, double top_p,
+                    int32_t *d_tokens, double *d_codes_out,
+                    const as_step_diag *diag, void *stream);
+
+/*
  * Same step with HOST buffers: copies logits and codes to the device, runs
  * as_step, copies tokens and codes back, and returns after the results are in
  * the host buffers (it synchronises `stream`).  Pinned host memory makes the

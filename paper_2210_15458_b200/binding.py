@@ -34,7 +34,7 @@ TUNE_CTAS_PER_SM = 3
 TUNE_STAGES = 4
 TUNE_MIN_CTAS = 5
 
-EXPORTS = ["as_lattice_codes", "as_lattice_codes_variant", "as_step", "as_step_host", "as_step_host_work_bytes", "as_step_host_static",
+EXPORTS = ["as_lattice_codes", "as_lattice_codes_variant", "as_step", "as_step_lattice", "as_step_host", "as_step_host_work_bytes", "as_step_host_static",
            "as_decode_bigram",
            "as_decode_bigram_codes", "as_encode_bigram", "as_ngram_diversity", "as_reward_mean", "as_tune",
            "as_last_error", "as_version"]
@@ -79,6 +79,8 @@ def lib():
         L.as_decode_bigram.argtypes = [P, I, I, LL, P, I, I, D, I, I, D, I, D, P, P, P, P, P]
         L.as_decode_bigram_codes.argtypes = [P, I, I, LL, P, P, I, I, I, D, I, D, P, P, P, P, P]
         L.as_encode_bigram.argtypes = [P, I, I, LL, P, P, P, I, I, D, I, D, P, P, P, P]
+        L.as_step_lattice.argtypes = [P, I, I, I, LL, I, D, I, D, I, D, P, P, P, P]
+        L.as_step_lattice.restype = I
         L.as_lattice_codes_variant.argtypes = [I, D, I, P, P]
         L.as_lattice_codes_variant.restype = I
         L.as_ngram_diversity.argtypes = [P, P, I, I, I, P, P, P, P]
@@ -176,6 +178,22 @@ def as_step(logits: torch.Tensor, codes: torch.Tensor, temp: float = 1.0, top_k:
     _check(lib().as_step(_ptr(logits), _logits_dtype(logits), lanes, V, ld, _ptr(codes), temp, top_k, top_p,
                          _ptr(tokens), _ptr(codes_out), ctypes.byref(dg) if dg is not None else None,
                          _stream(stream)))
+    return tokens, codes_out
+
+
+def as_step_lattice(logits: torch.Tensor, N: int, u: float, j0: int = 0, temp: float = 1.0, top_k: int = 0,
+                    top_p: float = 1.0, tokens: Optional[torch.Tensor] = None,
+                    codes_out: Optional[torch.Tensor] = None, V: Optional[int] = None, stream=None):
+    """First decode step with the lattice codes (j0 + i + u)/N formed in the kernel."""
+    lanes, width, ld = _logits_layout(logits)
+    V = width if V is None else V
+    dev = logits.device
+    if tokens is None:
+        tokens = torch.empty(lanes, dtype=torch.int32, device=dev)
+    if codes_out is None:
+        codes_out = torch.empty(lanes, dtype=torch.float64, device=dev)
+    _check(lib().as_step_lattice(_ptr(logits), _logits_dtype(logits), lanes, V, ld, N, u, j0, temp, top_k, top_p,
+                                 _ptr(tokens), _ptr(codes_out), None, _stream(stream)))
     return tokens, codes_out
 
 

@@ -179,13 +179,19 @@ __global__ void lattice_variant_kernel(int N, double b, int variant, double* __r
 template <int DT>
 __global__ void __launch_bounds__(GEN_NT)
 step_generic_kernel(const void* __restrict__ logits, int lanes, int V, long long ld,
-                    const double* codes, double inv_tau, int top_k, double top_p,
-                    int* __restrict__ tokens, double* codes_out, DiagPtrs diag) {
+                    const double* codes, int lat_N, int lat_j0, double lat_u, double inv_tau, int top_k,
+                    double top_p, int* __restrict__ tokens, double* codes_out, DiagPtrs diag) {
     __shared__ GenericSmem<GEN_NT> sm;
     for (int ln = blockIdx.x; ln < lanes; ln += gridDim.x) {
         const char* row = reinterpret_cast<const char*>(logits) + (size_t)ln * (size_t)ld * Traits<DT>::BYTES;
         const bool vec_ok = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
-        const double c = codes[ln];
+        double c;
+        if (lat_N > 0) {            // the lattice itself (same expression as lattice_kernel)
+            c = ((double)(lat_j0 + ln) + lat_u) / (double)lat_N;
+            if (c >= 1.0) c -= 1.0;
+        } else {
+            c = codes[ln];
+        }
         GenericLane<DT, GEN_NT> g(sm, row, V, vec_ok);
         const LaneResult r = g.run(c, inv_tau, top_k, top_p);
         if (threadIdx.x == 0) {
@@ -386,15 +392,18 @@ int as_lattice_codes_variant(int N, double b, int variant, double* d_codes, void
     return AS_OK;
 }
 
-int as_step(const void* d_logits, int dtype, int lanes, int V, long long ld, const double* d_codes,
-            double temp, int top_k, double top_p, int32_t* d_tokens, double* d_codes_out,
-            const as_step_diag* diag, void* stream) {
+}  // extern "C"
+
+// as_step and as_step_lattice: lat_N = 0 reads d_codes, lat_N > 0 forms the lattice codes in the kernel
+static int step_common(const void* d_logits, int dtype, int lanes, int V, long long ld, const double* d_codes,
+                       int lat_N, int lat_j0, double lat_u, double temp, int top_k, double top_p,
+                       int32_t* d_tokens, double* d_codes_out, const as_step_diag* diag, void* stream) {
     if (lanes < 0) return set_err(AS_ERR_INVALID_ARG, "lanes = %d must be >= 0", lanes);
     int rc = check_scalars(dtype, V, ld, temp, top_p);
     if (rc != AS_OK) return rc;
     if (lanes == 0) return AS_OK;
     if ((rc = check_data(d_logits, dtype)) != AS_OK) return rc;
-    if (!d_codes || !d_tokens || !d_codes_out) return set_err(AS_ERR_INVALID_ARG, "codes / tokens / codes_out pointer is NULL");
+    if ((!d_codes && lat_N == 0) || !d_tokens || !d_codes_out) return set_err(AS_ERR_INVALID_ARG, "codes / tokens / codes_out pointer is NULL");
     const DeviceInfo* di;
     rc = device_info(&di);
     if (rc != AS_OK) return rc;
@@ -408,6 +417,7 @@ int as_step(const void* d_logits, int dtype, int lanes, int V, long long ld, con
     a.logits = d_logits; a.codes = d_codes; a.tokens = d_tokens; a.codes_out = d_codes_out; a.diag = dp;
     a.ld = ld; a.inv_tau = inv_tau; a.top_p = top_p; a.scale2 = (float)(1.4426950408889634 / temp);
     a.lanes = lanes; a.V = V; a.top_k = top_k;
+    a.lat_N = lat_N; a.lat_j0 = lat_j0; a.lat_u = lat_u;
     const int E = dtype == AS_F32 ? 4 : 8;
     const size_t row_bytes = (size_t)((V + E - 1) / E) * 16;
     if (g_tune_path == 0) {
@@ -444,12 +454,32 @@ int as_step(const void* d_logits, int dtype, int lanes, int V, long long ld, con
     }
     const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
     if (dtype == AS_F32)
-        step_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, inv_tau, top_k, top_p, d_tokens, d_codes_out, dp);
+        step_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, lat_N, lat_j0, lat_u, inv_tau, top_k, top_p, d_tokens, d_codes_out, dp);
     else
-        step_generic_kernel<DT_BF16><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, inv_tau, top_k, top_p, d_tokens, d_codes_out, dp);
+        step_generic_kernel<DT_BF16><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, lat_N, lat_j0, lat_u, inv_tau, top_k, top_p, d_tokens, d_codes_out, dp);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "step kernel launch");
     return AS_OK;
+}
+
+extern "C" {
+
+int as_step(const void* d_logits, int dtype, int lanes, int V, long long ld, const double* d_codes,
+            double temp, int top_k, double top_p, int32_t* d_tokens, double* d_codes_out,
+            const as_step_diag* diag, void* stream) {
+    return step_common(d_logits, dtype, lanes, V, ld, d_codes, 0, 0, 0.0, temp, top_k, top_p, d_tokens,
+                       d_codes_out, diag, stream);
+}
+
+int as_step_lattice(const void* d_logits, int dtype, int lanes, int V, long long ld, int N, double u, int j0,
+                    double temp, int top_k, double top_p, int32_t* d_tokens, double* d_codes_out,
+                    const as_step_diag* diag, void* stream) {
+    if (N < 1) return set_err(AS_ERR_INVALID_ARG, "N = %d must be >= 1", N);
+    if (!(u >= 0.0 && u < 1.0)) return set_err(AS_ERR_INVALID_ARG, "shift u must lie in [0,1)");
+    if (j0 < 0 || lanes < 0 || (long long)j0 + lanes > N)
+        return set_err(AS_ERR_INVALID_ARG, "lanes j0 .. j0+lanes-1 = %d .. %lld must lie in [0, N = %d)", j0, (long long)j0 + lanes - 1, N);
+    return step_common(d_logits, dtype, lanes, V, ld, nullptr, N, j0, u, temp, top_k, top_p, d_tokens,
+                       d_codes_out, diag, stream);
 }
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }

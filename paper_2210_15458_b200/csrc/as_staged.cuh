@@ -75,7 +75,21 @@ struct StepArgs {
     int V;
     int top_k;
     int fast;          // 1: try the compaction path for lanes with a cut
+    // lat_N > 0: the codes are the lattice itself, lane i taking c = (lat_j0 + i + lat_u) / lat_N
+    // mod 1 (the same fp64 expression as the lattice kernel), and `codes` is not read
+    int lat_N;
+    int lat_j0;
+    double lat_u;
 };
+
+__device__ __forceinline__ double lane_code(const StepArgs& a, int ln) {
+    if (a.lat_N > 0) {
+        double c = ((double)(a.lat_j0 + ln) + a.lat_u) / (double)a.lat_N;
+        if (c >= 1.0) c -= 1.0;
+        return c;
+    }
+    return a.codes[ln];
+}
 
 // ---------------------------------------------------------------------------
 // PTX wrappers: mbarrier + bulk async copy global -> shared
@@ -388,7 +402,7 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
         const int leader = (CS > 1) ? (it % CS) : 0;
         const bool is_leader = (crank == leader);
         const int nxt = ln + nclusters;
-        const double c_in = a.codes[ln];
+        const double c_in = lane_code(a, ln);
         double c = c_in;
         const bool code_bad = !(c >= 0.0 && c <= 1.0);
         if (c == 1.0) c = ASX_ONE_BELOW;

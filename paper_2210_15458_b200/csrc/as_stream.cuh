@@ -606,7 +606,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
     };
 
     for (int ln = blockIdx.x; ln < a.lanes; ln += gridDim.x) {
-        const double c_in = a.codes[ln];
+        const double c_in = lane_code(a, ln);
         double c = c_in;
         const bool code_bad = !(c >= 0.0 && c <= 1.0);
         if (c == 1.0) c = ASX_ONE_BELOW;

@@ -474,3 +474,27 @@ def test_step_hit_list_overflow_takes_one_more_pass(B, orc, dtype):
                      d["n_kept"].cpu().numpy(), d["lane_status"].cpu().numpy(),
                      what="overflow %s" % ((temp, k, p),))
         assert (d["path"].cpu().numpy() == B.PATH_COMPACT).sum() >= lanes // 2 + 1
+
+
+@pytest.mark.parametrize("dtype,V", [(BF16, 32000), (F32, 5000), (BF16, 140000), (F32, 33)])
+def test_step_lattice_equals_lattice_codes_then_step(B, orc, dtype, V):
+    # codes formed in the kernel are the very values as_lattice_codes writes: the fused first step
+    # must reproduce the two-call result bit for bit, on every kernel path, also for a slice j0..
+    rng = np.random.default_rng(V)
+    N, lanes, j0, u = 97, 40, 31, 0.8125
+    arr = _store(rng.normal(0, 3, (lanes, V)), dtype)
+    dev = to_dev(arr, dtype)
+    codes = B.as_lattice_codes(N, u)
+    for temp, k, p in [(0.7, 40, 1.0), (1.0, 0, 0.9), (1.0, 0, 1.0)]:
+        tok_a, c_a = B.as_step(dev, codes[j0:j0 + lanes].contiguous(), temp, k, p)
+        tok_b, c_b = B.as_step_lattice(dev, N, u, j0, temp, k, p)
+        torch.cuda.synchronize()
+        assert (tok_a == tok_b).all() and (c_a == c_b).all()
+    check(B, orc, arr, dtype, orc.lattice_codes(N, u)[j0:j0 + lanes], 0.7, 40, 1.0, what="lattice slice")
+    try:
+        B.as_tune(B.TUNE_STEP_PATH, 2)
+        tok_a, c_a = B.as_step(dev, codes[j0:j0 + lanes].contiguous(), 0.7, 40, 1.0)
+        tok_b, c_b = B.as_step_lattice(dev, N, u, j0, 0.7, 40, 1.0)
+        assert (tok_a == tok_b).all() and (c_a == c_b).all()
+    finally:
+        B.as_tune(B.TUNE_STEP_PATH, 0)

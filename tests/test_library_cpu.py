@@ -41,6 +41,10 @@ def test_invalid_arguments_are_rejected_on_the_host(L):
     assert L.as_lattice_codes(4, 1.0, p, None) == B.ERR_INVALID_ARG
     assert L.as_lattice_codes(4, float("nan"), p, None) == B.ERR_INVALID_ARG
     assert L.as_lattice_codes(4, 0.5, None, None) == B.ERR_INVALID_ARG
+    sl = lambda **k: L.as_step_lattice(p, 0, k.get("lanes", 2), 2, 2, k.get("N", 4), k.get("u", 0.5), k.get("j0", 0),
+                                       1.0, 0, 1.0, p, p, None, None)
+    assert sl(N=0) == B.ERR_INVALID_ARG and sl(u=1.0) == B.ERR_INVALID_ARG and sl(j0=-1) == B.ERR_INVALID_ARG
+    assert sl(j0=3) == B.ERR_INVALID_ARG and sl(lanes=5) == B.ERR_INVALID_ARG
     assert L.as_lattice_codes_variant(4, 0.5, 7, p, None) == B.ERR_INVALID_ARG
     assert L.as_lattice_codes_variant(0, 0.5, 1, p, None) == B.ERR_INVALID_ARG
     assert L.as_lattice_codes_variant(4, 1.0, 1, p, None) == B.ERR_INVALID_ARG
