@@ -606,10 +606,9 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
     };
 
     for (int ln = blockIdx.x; ln < a.lanes; ln += gridDim.x) {
+        // the code is first looked at just before the epilogue: its 8-byte load queues behind the
+        // row copies of the whole grid, and an earlier use would hold up the passes over the row
         const double c_in = lane_code(a, ln);
-        double c = c_in;
-        const bool code_bad = !(c >= 0.0 && c <= 1.0);
-        if (c == 1.0) c = ASX_ONE_BELOW;
         const char* row = row_of(ln);
 
         // Lanes the candidate list cannot decide end in ONE call of the general routine (kept out
@@ -706,7 +705,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             ASX_MARK(2);
             threshold(acc, gmax, t0key, cut, 0u);
             ASX_MARK(3);
-            const bool bad = code_bad || gmax >= Tr::KEY_PINF || gmax <= Tr::KEY_NINF;
+            const bool bad = gmax >= Tr::KEY_PINF || gmax <= Tr::KEY_NINF;
             if (bad) {
                 r = failed_lane(c_in, ST_NUMERIC);
                 decided = true;
@@ -805,7 +804,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             if (tid == 0) P::merge(acc, P::reduce(qt));
             uint32_t t0unused;
             threshold(acc, gmax, t0unused, false, 0u);   // final max (t0key keeps the value the hits were taken with)
-            const bool bad = code_bad || gmax >= Tr::KEY_PINF || gmax <= Tr::KEY_NINF;
+            const bool bad = gmax >= Tr::KEY_PINF || gmax <= Tr::KEY_NINF;
             if (bad) {
                 r = failed_lane(c_in, ST_NUMERIC);
                 decided = true;
@@ -891,8 +890,12 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
 #ifdef ASX_PROFILE
         if (blockIdx.x == 0 && tid == 0) { g_asx_marks[20] = nvh; g_asx_marks[21] = C; }
 #endif
+        const double c = c_in == 1.0 ? ASX_ONE_BELOW : c_in;
         if (*(volatile int*)&sm.poisoned) {
             r = failed_lane(c_in, ST_TIMEOUT);
+            decided = true;
+        } else if (!decided && !(c_in >= 0.0 && c_in <= 1.0)) {
+            r = failed_lane(c_in, ST_NUMERIC);
             decided = true;
         } else if (list_ok && (!want_tail || (tailsum == tailsum && tailsum < 1e300))) {
             decided = epilogue_ranked<DT, NT, SyncC, StreamSmem>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, t0key, c,
