@@ -164,6 +164,8 @@ int as_step_lattice(const void *d_logits, int dtype, int lanes, int V, long long
  *   [lanes] host, written;  h_lane_status NULL or [lanes] host, written.
  *   d_work   device scratch of at least as_step_host_work_bytes(...) bytes,
  *            256-byte aligned, owned by the caller; contents undefined after.
+ *            The rows are staged there at a pitch that is a multiple of 16
+ *            bytes whatever ld is, so every row takes the fast kernel path.
  * Errors: as as_step, plus AS_ERR_INVALID_ARG if work_bytes is too small.
  */
 int as_step_host(const void *h_logits, int dtype, int lanes, int V, long long ld,

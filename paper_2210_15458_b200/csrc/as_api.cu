@@ -487,7 +487,8 @@ static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 size_t as_step_host_work_bytes(int dtype, int lanes, long long ld) {
     if (lanes < 0 || ld < 0 || (dtype != AS_F32 && dtype != AS_BF16)) return 0;
     const size_t esz = dtype == AS_F32 ? 4 : 2;
-    return align256((size_t)lanes * (size_t)ld * esz) + 2 * align256((size_t)lanes * 8) +
+    // the rows are staged at a pitch rounded up to 16 bytes (see as_step_host)
+    return align256((size_t)lanes * ((((size_t)ld * esz) + 15) & ~(size_t)15)) + 2 * align256((size_t)lanes * 8) +
            2 * align256((size_t)lanes * 4) + 256;
 }
 
@@ -503,7 +504,12 @@ int as_step_host(const void* h_logits, int dtype, int lanes, int V, long long ld
     if (!d_work || (reinterpret_cast<uintptr_t>(d_work) & 255)) return set_err(AS_ERR_INVALID_ARG, "d_work must be a 256-byte aligned device pointer");
     if (work_bytes < as_step_host_work_bytes(dtype, lanes, ld)) return set_err(AS_ERR_INVALID_ARG, "work_bytes is smaller than as_step_host_work_bytes()");
     const size_t esz = dtype == AS_F32 ? 4 : 2;
-    const size_t nlog = (size_t)lanes * (size_t)ld * esz;
+    // A host pitch that is not a multiple of 16 bytes would leave every other row unaligned and
+    // send it through the general routine; the copy can place the rows at an aligned pitch for free.
+    const bool repitch = (((size_t)ld * esz) & 15) != 0;
+    const size_t dpitch = repitch ? ((((size_t)V * esz) + 15) & ~(size_t)15) : (size_t)ld * esz;
+    const long long d_ld = (long long)(dpitch / esz);
+    const size_t nlog = (size_t)lanes * ((((size_t)ld * esz) + 15) & ~(size_t)15);
     char* w = reinterpret_cast<char*>(d_work);
     void* d_logits = w;                 w += align256(nlog);
     double* d_codes = (double*)w;       w += align256((size_t)lanes * 8);
@@ -514,10 +520,15 @@ int as_step_host(const void* h_logits, int dtype, int lanes, int V, long long ld
     cudaError_t e;
     // the last row may be shorter than ld in the caller's buffer: copy lanes-1 full pitches + V
     const size_t ncopy = ((size_t)(lanes - 1) * (size_t)ld + (size_t)V) * esz;
-    if ((e = cudaMemcpyAsync(d_logits, h_logits, ncopy, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "copy logits to device");
+    if (repitch)
+        e = cudaMemcpy2DAsync(d_logits, dpitch, h_logits, (size_t)ld * esz, (size_t)V * esz, (size_t)lanes,
+                              cudaMemcpyHostToDevice, st);
+    else
+        e = cudaMemcpyAsync(d_logits, h_logits, ncopy, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e, "copy logits to device");
     if ((e = cudaMemcpyAsync(d_codes, h_codes, (size_t)lanes * 8, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "copy codes to device");
     as_step_diag dg = {nullptr, nullptr, nullptr, d_status, nullptr};
-    rc = as_step(d_logits, dtype, lanes, V, ld, d_codes, temp, top_k, top_p, d_tokens, d_codes_out, &dg, stream);
+    rc = as_step(d_logits, dtype, lanes, V, d_ld, d_codes, temp, top_k, top_p, d_tokens, d_codes_out, &dg, stream);
     if (rc != AS_OK) return rc;
     if ((e = cudaMemcpyAsync(h_tokens, d_tokens, (size_t)lanes * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "copy tokens to host");
     if ((e = cudaMemcpyAsync(h_codes_out, d_codes_out, (size_t)lanes * 8, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "copy codes to host");

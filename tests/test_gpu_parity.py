@@ -498,3 +498,23 @@ def test_step_lattice_equals_lattice_codes_then_step(B, orc, dtype, V):
         assert (tok_a == tok_b).all() and (c_a == c_b).all()
     finally:
         B.as_tune(B.TUNE_STEP_PATH, 0)
+
+
+@pytest.mark.parametrize("dtype,V,ld", [(BF16, 32001, 32001), (F32, 5003, 5003), (BF16, 32000, 32000), (BF16, 4097, 4100)])
+def test_step_host_buffers_any_pitch(B, orc, dtype, V, ld):
+    # host buffers whose pitch is not a multiple of 16 bytes are staged at an aligned pitch
+    rng = np.random.default_rng(V + ld)
+    lanes = 24
+    full = _store(rng.normal(0, 3, (lanes, ld)), dtype)
+    arr = np.ascontiguousarray(full[:, :V])
+    codes = rng.random(lanes)
+    ref = orc.step(arr, dtype, codes, 0.8, 30, 0.95, threads=8)
+    h_logits = torch.from_numpy(full.view(np.int16)).view(torch.bfloat16) if dtype == BF16 else torch.from_numpy(full)
+    h_codes = torch.from_numpy(codes)
+    tok = torch.empty(lanes, dtype=torch.int32)
+    c2 = torch.empty(lanes, dtype=torch.float64)
+    st = torch.empty(lanes, dtype=torch.int32)
+    work = torch.empty(B.as_step_host_work_bytes(dtype, lanes, ld) + 256, dtype=torch.uint8, device="cuda")
+    B.as_step_host(h_logits, h_codes, 0.8, 30, 0.95, tok, c2, st, work, V=V)
+    r = compare_step(ref, tok.numpy(), c2.numpy(), status=st.numpy(), what="host buffers V=%d ld=%d" % (V, ld))
+    assert r["compared"] >= lanes - 3
