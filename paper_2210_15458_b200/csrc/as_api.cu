@@ -105,13 +105,13 @@ static int launch_staged(const StepArgs& a, size_t smem, int sms, int want_per_s
     return AS_OK;
 }
 
-template <int DT, int CAPV, int MINB>
-static int launch_stream(const StepArgs& a, int stages, int sms, int want_per_sm, cudaStream_t st) {
+template <int DT, int CAPV, int MINB, bool UA>
+static int launch_stream_ua(const StepArgs& a, int stages, int sms, int want_per_sm, cudaStream_t st) {
     static bool attr_set[64] = {false};
     static int per_sm_cache[64][SK_MAXSTAGES + 1] = {{0}};
     int dev = 0;
     cudaGetDevice(&dev);
-    auto kern = step_stream_kernel<DT, CAPV, MINB>;
+    auto kern = step_stream_kernel<DT, CAPV, MINB, UA>;
     cudaError_t e;
     if (!attr_set[dev]) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_OPTIN_MAX - 1024));
@@ -135,6 +135,14 @@ static int launch_stream(const StepArgs& a, int stages, int sms, int want_per_sm
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "streaming step kernel launch");
     return AS_OK;
+}
+
+// rows that all start on 16-byte boundaries take the plain build; otherwise the build that
+// copies each row from the boundary below its start
+template <int DT, int CAPV, int MINB>
+static int launch_stream(const StepArgs& a, bool unaligned, int stages, int sms, int want_per_sm, cudaStream_t st) {
+    return unaligned ? launch_stream_ua<DT, CAPV, MINB, true>(a, stages, sms, want_per_sm, st)
+                     : launch_stream_ua<DT, CAPV, MINB, false>(a, stages, sms, want_per_sm, st);
 }
 
 template <int DT>
@@ -419,7 +427,10 @@ static int step_common(const void* d_logits, int dtype, int lanes, int V, long l
     a.lanes = lanes; a.V = V; a.top_k = top_k;
     a.lat_N = lat_N; a.lat_j0 = lat_j0; a.lat_u = lat_u;
     const int E = dtype == AS_F32 ? 4 : 8;
-    const size_t row_bytes = (size_t)((V + E - 1) / E) * 16;
+    const size_t esz = dtype == AS_F32 ? 4 : 2;
+    // some row starts off a 16-byte boundary: it is read from the boundary below, up to E-1 elements longer
+    const bool unaligned = (reinterpret_cast<uintptr_t>(d_logits) & 15) != 0 || (((size_t)ld * esz) & 15) != 0;
+    const size_t row_bytes = (size_t)((V + (unaligned && g_tune_path == 0 ? E - 1 : 0) + E - 1) / E) * 16;
     if (g_tune_path == 0) {
         // streaming kernel: one CTA per lane; rows of up to 6 stages (96 KB) stay resident in the ring
         const int nsl = (int)((row_bytes + SK_STAGE_BYTES - 1) / SK_STAGE_BYTES);
@@ -431,13 +442,13 @@ static int step_common(const void* d_logits, int dtype, int lanes, int V, long l
             if (!resident && stages >= nsl) stages = nsl - 1;
             if (dtype == AS_F32) {
                 if (!resident && g_tune_minb != 2)
-                    return launch_stream<DT_F32, 1536, 3>(a, stages < 2 ? stages : 2, di->sms, g_tune_ctas, st);
-                return launch_stream<DT_F32, 2048, 2>(a, stages, di->sms, g_tune_ctas, st);
+                    return launch_stream<DT_F32, 1536, 3>(a, unaligned, stages < 2 ? stages : 2, di->sms, g_tune_ctas, st);
+                return launch_stream<DT_F32, 2048, 2>(a, unaligned, stages, di->sms, g_tune_ctas, st);
             }
             // bf16 rows that stream: a 1024-entry hit list and <= 72 registers let three CTAs share an SM
             if (!resident && g_tune_minb != 2)
-                return launch_stream<DT_BF16, 1024, 3>(a, stages < 3 ? stages : 3, di->sms, g_tune_ctas, st);
-            return launch_stream<DT_BF16, 2048, 2>(a, stages, di->sms, g_tune_ctas, st);
+                return launch_stream<DT_BF16, 1024, 3>(a, unaligned, stages < 3 ? stages : 3, di->sms, g_tune_ctas, st);
+            return launch_stream<DT_BF16, 2048, 2>(a, unaligned, stages, di->sms, g_tune_ctas, st);
         }
     }
     if (g_tune_path == 2) {

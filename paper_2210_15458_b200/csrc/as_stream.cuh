@@ -447,7 +447,28 @@ __device__ __noinline__ float recollect_row(StreamSmem& sm, int V, const char* r
     return tail;
 }
 
-template <int DT, int CAPV, int MINB>
+// UA builds also serve rows that do not start on a 16-byte boundary (a pitch or base pointer that
+// is only element-aligned): such a row is copied from the boundary below its start, the `lead`
+// elements in front of it are masked to -inf in the first vector, and every token index shifts
+// by `lead`.  The bytes in front belong to the same 16-byte granule as the row's first element,
+// so the copy never leaves mapped memory; past its end nothing beyond whole granules inside the
+// row is copied.  Calls whose rows are all aligned use the build without this.
+template <int DT>
+__device__ __forceinline__ void mask_lead(uint4& q, int lead) {
+    uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (DT == DT_BF16) {
+            if (2 * i < lead) w[i] = (w[i] & 0xFFFF0000u) | 0xFF80u;
+            if (2 * i + 1 < lead) w[i] = (w[i] & 0x0000FFFFu) | 0xFF800000u;
+        } else if (i < lead) {
+            w[i] = 0xFF800000u;
+        }
+    }
+    q = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+template <int DT, int CAPV, int MINB, bool UA = false>
 __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const StepArgs a, const int stages) {
     using StreamSmem = StreamSmemT<CAPV>;
     constexpr int SK_CAPV = CAPV;
@@ -463,7 +484,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     ASX_MARK(13);
     const int V = a.V;
-    const int row_bytes = V * Tr::BYTES;
+    const int row_bytes = (V + (UA ? E - 1 : 0)) * Tr::BYTES;          // UA: the longest a row gets with its lead
     const int bulk_bytes = row_bytes & ~15;
     const int bulk_vec = bulk_bytes >> 4;
     const int tail_elems = (row_bytes - bulk_bytes) / Tr::BYTES;      // < E
@@ -474,7 +495,18 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
     auto row_of = [&](int ln) -> const char* {
         return reinterpret_cast<const char*>(a.logits) + (size_t)ln * (size_t)a.ld * Tr::BYTES;
     };
-    auto staged_ok = [&](int ln) -> bool { return (reinterpret_cast<uintptr_t>(row_of(ln)) & 15) == 0; };
+    auto staged_ok = [&](int ln) -> bool { return UA || (reinterpret_cast<uintptr_t>(row_of(ln)) & 15) == 0; };
+    auto lead_of = [&](int ln) -> int {
+        return UA ? (int)((reinterpret_cast<uintptr_t>(row_of(ln)) & 15) / Tr::BYTES) : 0;
+    };
+    // one row's own geometry (UA: it depends on the row's lead)
+    auto geom = [&](int lead, int& bb, int& bv, int& te, int& ns) {
+        const int rb = (V + lead) * Tr::BYTES;
+        bb = rb & ~15;
+        bv = bb >> 4;
+        te = (rb - bb) / Tr::BYTES;
+        ns = (bv + SK_STAGE_VEC - 1) / SK_STAGE_VEC;
+    };
 
     // The producer lane initialises the barriers of the stages in use and starts the first copies
     // before the block-wide barrier, so the first row is in flight while the rest of the CTA sets up.
@@ -485,8 +517,11 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
     auto issue_some = [&](bool first_row_only) -> bool {   // false: a bounded wait ran out
         for (; ln_issue < a.lanes; ln_issue += gridDim.x, s_issue = 0) {
             if (!staged_ok(ln_issue)) continue;
-            const char* src = row_of(ln_issue);
-            for (; s_issue < nsl; ++s_issue, ++g_issued) {
+            int bulk_bytes_i = bulk_bytes, nsl_i = nsl;
+            const int lead_i = lead_of(ln_issue);
+            if (UA) { int bv, te; geom(lead_i, bulk_bytes_i, bv, te, nsl_i); }
+            const char* src = row_of(ln_issue) - lead_i * Tr::BYTES;
+            for (; s_issue < nsl_i; ++s_issue, ++g_issued) {
                 const int st = g_issued % S;
                 if (g_issued >= (unsigned)S) {    // the stage must have been drained by every consumer warp
                     if (first_row_only) return true;
@@ -496,7 +531,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                         return false;
                     }
                 }
-                const uint32_t bytes = (uint32_t)min(SK_STAGE_BYTES, bulk_bytes - s_issue * SK_STAGE_BYTES);
+                const uint32_t bytes = (uint32_t)min(SK_STAGE_BYTES, bulk_bytes_i - s_issue * SK_STAGE_BYTES);
                 const uint32_t bar = smem_u32(&sm.full_bar[st]);
                 mbar_expect_tx(bar, bytes);
                 bulk_g2s(smem_u32(ring + (size_t)st * SK_STAGE_BYTES), src + (size_t)s_issue * SK_STAGE_BYTES, bytes, bar);
@@ -610,6 +645,10 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         // row copies of the whole grid, and an earlier use would hold up the passes over the row
         const double c_in = lane_code(a, ln);
         const char* row = row_of(ln);
+        const int lead = lead_of(ln);
+        int bulk_bytes_l = bulk_bytes, bulk_vec_l = bulk_vec, tail_elems_l = tail_elems, nsl_l = nsl;
+        if (UA) geom(lead, bulk_bytes_l, bulk_vec_l, tail_elems_l, nsl_l);
+        const char* vrow = row - lead * Tr::BYTES;     // where the copies start
 
         // Lanes the candidate list cannot decide end in ONE call of the general routine (kept out
         // of line so that the hot path stays small).
@@ -624,6 +663,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             general_row = row;
             general_vec_ok = false;
         }
+        if (UA && lead) general_vec_ok = false;       // should the general routine be needed after all
         if (tid == 0) { sm.vec_count = 0; sm.cand_count = 0; }
         // the candidate array starts zeroed: entries past the count rank below every candidate,
         // which the epilogue's 4-wide rank loop relies on
@@ -631,20 +671,20 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
 
         // ragged end of the row (< 16 bytes): one padded vector read straight from global memory
         uint4 qt = make_uint4(ninf_word, ninf_word, ninf_word, ninf_word);
-        if (tail_elems > 0 && tid == 0 && !general_row) {
+        if (tail_elems_l > 0 && tid == 0 && !general_row) {
             uint32_t w[4];
             if (DT == DT_BF16) {
-                const unsigned short* src = reinterpret_cast<const unsigned short*>(row + bulk_bytes);
+                const unsigned short* src = reinterpret_cast<const unsigned short*>(vrow + bulk_bytes_l);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const uint32_t lo = (2 * i < tail_elems) ? src[2 * i] : 0xFF80u;
-                    const uint32_t hi = (2 * i + 1 < tail_elems) ? src[2 * i + 1] : 0xFF80u;
+                    const uint32_t lo = (2 * i < tail_elems_l) ? src[2 * i] : 0xFF80u;
+                    const uint32_t hi = (2 * i + 1 < tail_elems_l) ? src[2 * i + 1] : 0xFF80u;
                     w[i] = lo | (hi << 16);
                 }
             } else {
-                const uint32_t* src = reinterpret_cast<const uint32_t*>(row + bulk_bytes);
+                const uint32_t* src = reinterpret_cast<const uint32_t*>(vrow + bulk_bytes_l);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) w[i] = (i < tail_elems) ? src[i] : 0xFF800000u;
+                for (int i = 0; i < 4; ++i) w[i] = (i < tail_elems_l) ? src[i] : 0xFF800000u;
             }
             qt = make_uint4(w[0], w[1], w[2], w[3]);
         }
@@ -685,11 +725,19 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             float pm[SK_RES_STAGES * SK_VPT];
 #pragma unroll
             for (int s = 0; s < SK_RES_STAGES; ++s) {
-                if (s < nsl) {
+                if (s < nsl_l) {
                     wait_full(g + s);
                     ASX_MARK(1);
                     uint4 q[SK_VPT];
-                    load_slice(ringv + (size_t)((g + s) % S) * SK_STAGE_VEC, min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC), q);
+                    load_slice(ringv + (size_t)((g + s) % S) * SK_STAGE_VEC, min(SK_STAGE_VEC, bulk_vec_l - s * SK_STAGE_VEC), q);
+                    if (UA && s == 0 && tid == 0 && lead) {
+                        // the elements in front of the row: masked here and in the ring (this thread
+                        // alone reads that vector again; the next bulk copy into the stage is
+                        // ordered after the store by the proxy fence)
+                        mask_lead<DT>(q[0], lead);
+                        reinterpret_cast<uint4*>(ring)[(size_t)(g % S) * SK_STAGE_VEC] = q[0];
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    }
 #pragma unroll
                     for (int j = 0; j < SK_VPT; ++j) {
                         const typename P::Acc part = P::reduce(q[j]);
@@ -709,18 +757,20 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             if (bad) {
                 r = failed_lane(c_in, ST_NUMERIC);
                 decided = true;
-                for (int s = 0; s < nsl; ++s) release(g + s);
+                for (int s = 0; s < nsl_l; ++s) release(g + s);
             } else if (!cut) {
                 // no cut: every token is kept; the general routine scans the row in shared memory
-                if (tail_elems > 0 && tid < tail_elems) {
+                if (UA && lead) {
+                    general_row = row;                 // (a row with a lead: from global memory)
+                } else if (tail_elems_l > 0 && tid < tail_elems_l) {
                     if (DT == DT_BF16)
-                        reinterpret_cast<unsigned short*>(ring + bulk_bytes)[tid] =
-                            reinterpret_cast<const unsigned short*>(row + bulk_bytes)[tid];
+                        reinterpret_cast<unsigned short*>(ring + bulk_bytes_l)[tid] =
+                            reinterpret_cast<const unsigned short*>(vrow + bulk_bytes_l)[tid];
                     else
-                        reinterpret_cast<uint32_t*>(ring + bulk_bytes)[tid] =
-                            reinterpret_cast<const uint32_t*>(row + bulk_bytes)[tid];
+                        reinterpret_cast<uint32_t*>(ring + bulk_bytes_l)[tid] =
+                            reinterpret_cast<const uint32_t*>(vrow + bulk_bytes_l)[tid];
                 }
-                general_row = ring;
+                if (!(UA && lead)) general_row = ring;
                 general_release = true;
             } else {
                 ref = Tr::value_f(gmax);
@@ -747,21 +797,21 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                                     const int slot = atomicAdd(&sm.cand_count, 1);
                                     if (slot < SK_CAP)
                                         sm.u.ep.cand[slot] = ((unsigned long long)key << 32) |
-                                                             (uint32_t)~(uint32_t)((s * SK_STAGE_VEC + v) * E + e);
+                                                             (uint32_t)~(uint32_t)((s * SK_STAGE_VEC + v) * E + e - lead);
                                 }
                             }
                         }
                     }
                 } else {
 #pragma unroll 1
-                    for (int s = 0; s < nsl; ++s) {
+                    for (int s = 0; s < nsl_l; ++s) {
                         uint4 q[SK_VPT];
                         const unsigned valid = load_slice(ringv + (size_t)((g + s) % S) * SK_STAGE_VEC,
-                                                          min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC), q);
+                                                          min(SK_STAGE_VEC, bulk_vec_l - s * SK_STAGE_VEC), q);
                         slice_pass(q, s * SK_STAGE_VEC + tid, valid, false, acc, t0f, ref, tail);
                     }
                 }
-                for (int s = 0; s < nsl; ++s) release(g + s);     // the producer may refill: next row
+                for (int s = 0; s < nsl_l; ++s) release(g + s);     // the producer may refill: next row
             }
         } else {
             // ---- streamed: slice -> registers -> stage released; T0 at slices 0, 1, 2, 4, 8, ...
@@ -774,13 +824,14 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
 #define ASX_ACC(var) do {} while (0)
 #endif
 #pragma unroll 1
-            for (int s = 0; s < nsl; ++s, ++g) {
+            for (int s = 0; s < nsl_l; ++s, ++g) {
                 wait_full(g);
                 ASX_ACC(pw);
                 uint4 q[SK_VPT];
                 const unsigned valid = load_slice(ringv + (size_t)(g % S) * SK_STAGE_VEC,
-                                                  min(SK_STAGE_VEC, bulk_vec - s * SK_STAGE_VEC), q);
+                                                  min(SK_STAGE_VEC, bulk_vec_l - s * SK_STAGE_VEC), q);
                 release(g);
+                if (UA && s == 0 && tid == 0 && lead) mask_lead<DT>(q[0], lead);
                 ASX_ACC(pl);
                 if (s == 0) {
 #pragma unroll
@@ -823,7 +874,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                 const uint4 q = sm.u.ep.v.cvec[i];
                 // most listed vectors came in under an earlier, lower threshold
                 if (!want_tail && !(P::part_max(P::reduce(q)) >= t0f)) continue;
-                const int base = sm.u.ep.cidx[i] * E;
+                const int base = sm.u.ep.cidx[i] * E - lead;
                 float x[E];
                 P::floats(q, x);
 #pragma unroll
@@ -841,7 +892,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                     if (want_tail && !hit) tail += ex2_approx((x[e] - ref) * scale2);
                 }
             }
-            if (tail_elems > 0 && tid == 0) {      // the ragged last vector lives in thread 0's registers
+            if (tail_elems_l > 0 && tid == 0) {      // the ragged last vector lives in thread 0's registers
                 float x[E];
                 P::floats(qt, x);
 #pragma unroll
@@ -853,14 +904,14 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                             hit = true;
                             const int slot = atomicAdd(&sm.cand_count, 1);
                             if (slot < SK_CAP)
-                                sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)(bulk_vec * E + e);
+                                sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)(bulk_vec_l * E + e - lead);
                         }
                     }
                     if (want_tail && !hit) tail += ex2_approx((x[e] - ref) * scale2);
                 }
             }
         }
-        if (!list_ok && !decided && !general_row && nvh > SK_CAPV && !*(volatile int*)&sm.poisoned) {
+        if (!list_ok && !decided && !general_row && nvh > SK_CAPV && !(UA && lead) && !*(volatile int*)&sm.poisoned) {
             // more hit vectors than the list holds: take the candidates in one more pass, against
             // the threshold that the whole row's subset maxima give now
             ASX_COUNT(8);
@@ -901,7 +952,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             decided = epilogue_ranked<DT, NT, SyncC, StreamSmem>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, t0key, c,
                                                      lmax, a.inv_tau, a.top_k, a.top_p, tailsum, r);
         }
-        if (!decided && want_tail && list_ok && !*(volatile int*)&sm.poisoned) {
+        if (!decided && want_tail && list_ok && !(UA && lead) && !*(volatile int*)&sm.poisoned) {
             // the nucleus reaches below the exact depth of the list: lower the threshold once
             ASX_COUNT(0);
             if (tid == 0) sm.b_i[2] = C;
@@ -917,9 +968,9 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             r = gl.run(c_in, a.inv_tau, a.top_k, a.top_p);
             path = PATH_GENERAL;
             if (general_release)
-                for (int s = 0; s < nsl; ++s) release(g + s);
+                for (int s = 0; s < nsl_l; ++s) release(g + s);
         }
-        if (resident && staged_ok(ln)) g += nsl;
+        if (resident && staged_ok(ln)) g += nsl_l;
         if (tid == 0) write_result(a, ln, r, path);
         SyncC::sync();
         ASX_MARK(12);

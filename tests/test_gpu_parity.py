@@ -518,3 +518,38 @@ def test_step_host_buffers_any_pitch(B, orc, dtype, V, ld):
     B.as_step_host(h_logits, h_codes, 0.8, 30, 0.95, tok, c2, st, work, V=V)
     r = compare_step(ref, tok.numpy(), c2.numpy(), status=st.numpy(), what="host buffers V=%d ld=%d" % (V, ld))
     assert r["compared"] >= lanes - 3
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+@pytest.mark.parametrize("V,pad", [(32001, 0), (4099, 3), (200003, 2), (140001, 0), (63, 0)])
+def test_step_rows_off_the_16_byte_grid_take_the_fast_path(B, orc, dtype, V, pad):
+    # a pitch that is only element-aligned: most rows start inside a 16-byte granule.  They are
+    # copied from the granule's start and the elements in front are masked -- which this test
+    # makes as tempting as possible: the padding between rows holds huge values, and the row's
+    # own first and last elements are its largest.
+    rng = np.random.default_rng(V + pad)
+    lanes = 19
+    ld = V + pad
+    x = rng.normal(0, 3, (lanes, ld)).astype(np.float32)
+    x[:, V:] = 80.0
+    x[:, 0] += 9.0
+    x[:, V - 1] += 9.0
+    full = _store(x, dtype)
+    off = 3                                               # the base pointer itself is off the grid too
+    flat = np.concatenate([_store(np.full(off, 90.0, np.float32), dtype), full.ravel()])
+    dev_flat = to_dev(flat, dtype)
+    dev = dev_flat[off:].view(lanes, ld)
+    arr = np.ascontiguousarray(full[:, :V])
+    codes = rng.random(lanes)
+    codes[0], codes[1] = 0.0, 1.0
+    for temp, k, p in [(0.7, 40, 1.0), (1.0, 0, 0.9), (0.9, 64, 0.95), (1.0, 1, 1.0)]:
+        d = {}
+        ref = orc.step(arr, dtype, codes, temp, k, p, threads=8)
+        tok, c2 = B.as_step(dev, torch.from_numpy(codes).cuda(), temp, k, p, diag=d, V=V)
+        torch.cuda.synchronize()
+        compare_step(ref, tok.cpu().numpy(), c2.cpu().numpy(), d["p_tok"].cpu().numpy(), d["n_kept"].cpu().numpy(),
+                     d["lane_status"].cpu().numpy(), what="off-grid rows V=%d %s" % (V, (temp, k, p)))
+        if V >= 4099:
+            assert (d["path"].cpu().numpy() == B.PATH_COMPACT).sum() >= lanes - 3
+    # no cut at all: the general routine, still correct
+    check(B, orc, arr[:4], dtype, codes[:4], 1.0, 0, 1.0, what="off-grid rows, no cut")
