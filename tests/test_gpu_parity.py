@@ -542,7 +542,7 @@ def test_step_rows_off_the_16_byte_grid_take_the_fast_path(B, orc, dtype, V, pad
     arr = np.ascontiguousarray(full[:, :V])
     codes = rng.random(lanes)
     codes[0], codes[1] = 0.0, 1.0
-    for temp, k, p in [(0.7, 40, 1.0), (1.0, 0, 0.9), (0.9, 64, 0.95), (1.0, 1, 1.0)]:
+    for temp, k, p in [(0.7, 40, 1.0), (0.5, 0, 0.9), (0.9, 64, 0.95), (1.0, 1, 1.0)]:
         d = {}
         ref = orc.step(arr, dtype, codes, temp, k, p, threads=8)
         tok, c2 = B.as_step(dev, torch.from_numpy(codes).cuda(), temp, k, p, diag=d, V=V)
