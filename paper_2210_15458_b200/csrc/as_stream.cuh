@@ -673,18 +673,20 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         uint4 qt = make_uint4(ninf_word, ninf_word, ninf_word, ninf_word);
         if (tail_elems_l > 0 && tid == 0 && !general_row) {
             uint32_t w[4];
+            // (a row shorter than a granule has its lead in this vector: those elements stay masked)
+            const int skip = (UA && bulk_vec_l == 0) ? lead : 0;
             if (DT == DT_BF16) {
                 const unsigned short* src = reinterpret_cast<const unsigned short*>(vrow + bulk_bytes_l);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const uint32_t lo = (2 * i < tail_elems_l) ? src[2 * i] : 0xFF80u;
-                    const uint32_t hi = (2 * i + 1 < tail_elems_l) ? src[2 * i + 1] : 0xFF80u;
+                    const uint32_t lo = (2 * i >= skip && 2 * i < tail_elems_l) ? src[2 * i] : 0xFF80u;
+                    const uint32_t hi = (2 * i + 1 >= skip && 2 * i + 1 < tail_elems_l) ? src[2 * i + 1] : 0xFF80u;
                     w[i] = lo | (hi << 16);
                 }
             } else {
                 const uint32_t* src = reinterpret_cast<const uint32_t*>(vrow + bulk_bytes_l);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) w[i] = (i < tail_elems_l) ? src[i] : 0xFF800000u;
+                for (int i = 0; i < 4; ++i) w[i] = (i >= skip && i < tail_elems_l) ? src[i] : 0xFF800000u;
             }
             qt = make_uint4(w[0], w[1], w[2], w[3]);
         }
