@@ -21,6 +21,7 @@
 namespace asx {
 
 constexpr int MAXCH = 512;  // chunks per row (R grows so that this suffices)
+constexpr int HIST_REP = 4; // replicas of every histogram bin
 
 // kept(key) = key > T, or key == T and: eq_mode 1 -> always; eq_mode 2 -> only the
 // first `need` such elements in index order; eq_mode 0 -> never.
@@ -34,8 +35,8 @@ template <int NT>
 struct GenericSmem {
     double chunk_sum[MAXCH + 1];
     int chunk_eq[MAXCH + 1];
-    double hist_mass[256];
-    int hist_cnt[256];
+    double hist_mass[256 * HIST_REP];     // bin d, replica r at [d * HIST_REP + r]: lanes spread over
+    int hist_cnt[256 * HIST_REP];         // the replicas, so that a crowded bin is hit by fewer threads
     double red_d[NT / 32];
     unsigned red_u[NT / 32];
     unsigned red_u2[NT / 32];
@@ -196,14 +197,17 @@ struct GenericLane {
     // `prefix` on `mask`; counts always, masses if MASS
     template <bool MASS>
     __device__ void hist_pass(const Pred& p, uint32_t prefix, uint32_t mask, int shift) {
-        for (int i = tid; i < 256; i += NT) {
+        for (int i = tid; i < 256 * HIST_REP; i += NT) {
             sm.hist_cnt[i] = 0;
             sm.hist_mass[i] = 0.0;
         }
+        const int rep = lane & (HIST_REP - 1);
         Sync::sync();
         // Each thread gathers runs of equal digits in registers and touches shared memory only
-        // when the digit changes: the leading digits of a row fall into two or three bins, and
+        // when the digit changes: the leading digits of a row fall into a handful of bins, and
         // a shared-memory fp64 add is a compare-and-swap loop that such crowding serialises.
+        // (Merging across the warp first -- one add per distinct digit among 32 lanes -- was
+        // tried and is 2-3x slower: the lower digits are all different.)
         int cur_d = -1, cur_n = 0;
         double cur_m = 0.0;
         for (int ci = warp; ci < nchunks; ci += NW) {
@@ -220,8 +224,8 @@ struct GenericLane {
                         const int d = (k[e] >> shift) & 255;
                         if (d != cur_d) {
                             if (cur_n) {
-                                atomicAdd(&sm.hist_cnt[cur_d], cur_n);
-                                if (MASS) atomicAdd(&sm.hist_mass[cur_d], cur_m);
+                                atomicAdd(&sm.hist_cnt[cur_d * HIST_REP + rep], cur_n);
+                                if (MASS) atomicAdd(&sm.hist_mass[cur_d * HIST_REP + rep], cur_m);
                             }
                             cur_d = d; cur_n = 0; cur_m = 0.0;
                         }
@@ -232,8 +236,8 @@ struct GenericLane {
             }
         }
         if (cur_n) {
-            atomicAdd(&sm.hist_cnt[cur_d], cur_n);
-            if (MASS) atomicAdd(&sm.hist_mass[cur_d], cur_m);
+            atomicAdd(&sm.hist_cnt[cur_d * HIST_REP + rep], cur_n);
+            if (MASS) atomicAdd(&sm.hist_mass[cur_d * HIST_REP + rep], cur_m);
         }
         Sync::sync();
     }
@@ -251,8 +255,13 @@ struct GenericLane {
             double lm = 0.0;
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                c[e] = sm.hist_cnt[lane * 8 + e];
-                m[e] = MASS ? sm.hist_mass[lane * 8 + e] : 0.0;
+                c[e] = 0;
+                m[e] = 0.0;
+#pragma unroll
+                for (int r = 0; r < HIST_REP; ++r) {
+                    c[e] += sm.hist_cnt[(lane * 8 + e) * HIST_REP + r];
+                    if (MASS) m[e] += sm.hist_mass[(lane * 8 + e) * HIST_REP + r];
+                }
                 lc += c[e];
                 lm += m[e];
             }
