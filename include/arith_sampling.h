@@ -218,7 +218,11 @@ int as_step_host_static(const void *h_logits, int dtype, int lanes, int V, long 
  *   temp, top_k, top_p   as in as_step, the same for every step
  *   d_seq         [S*N, T] i32 device, written (tokens, then -1 padding)
  *   d_len         [S*N] i32 device, written: tokens emitted (EOS included)
- *   d_codes_final NULL or [S*N] f64 device: each lane's code after its last step
+ *   d_codes_final NULL or [S*N] f64 device: each lane's code after its last step.
+ *                 It doubles as the loop's state: with a top-k / nucleus cut and this
+ *                 buffer given, the loop runs as one launch of the step kernel per
+ *                 step, rows gathered from the table by the previous tokens (several
+ *                 times faster than the single general kernel that runs otherwise)
  *   d_lane_status NULL or [S*N] i32 device: AS_OK, or the status that stopped the
  *                 lane early (a start/previous token outside [0,V) counts as
  *                 AS_ERR_NUMERIC)

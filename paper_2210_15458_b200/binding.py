@@ -233,7 +233,8 @@ def as_step_host_static(h_logits: torch.Tensor, h_codes: torch.Tensor, temp: flo
 def as_decode_bigram(table: torch.Tensor, start_tokens: torch.Tensor, N: int, u: float, T: int, eos: int,
                      temp: float = 1.0, top_k: int = 0, top_p: float = 1.0, V: Optional[int] = None,
                      codes_final: Optional[torch.Tensor] = None, lane_status: Optional[torch.Tensor] = None,
-                     seq: Optional[torch.Tensor] = None, length: Optional[torch.Tensor] = None, stream=None):
+                     seq: Optional[torch.Tensor] = None, length: Optional[torch.Tensor] = None, stream=None,
+                     per_step: bool = True):
     rows, width, ld = _logits_layout(table)
     V = width if V is None else V
     if rows < V:
@@ -241,6 +242,8 @@ def as_decode_bigram(table: torch.Tensor, start_tokens: torch.Tensor, N: int, u:
     S = start_tokens.numel()
     lanes = S * max(N, 0)
     dev = table.device
+    if codes_final is None and per_step:    # also the loop's state for the per-step kernels
+        codes_final = torch.empty(lanes, dtype=torch.float64, device=dev)
     if seq is None:
         seq = torch.empty((lanes, T), dtype=torch.int32, device=dev)
     if length is None:
@@ -255,13 +258,15 @@ def as_decode_bigram_codes(table: torch.Tensor, prev: torch.Tensor, codes_in: to
                            temp: float = 1.0, top_k: int = 0, top_p: float = 1.0, V: Optional[int] = None,
                            codes_final: Optional[torch.Tensor] = None,
                            lane_status: Optional[torch.Tensor] = None, seq: Optional[torch.Tensor] = None,
-                           length: Optional[torch.Tensor] = None, stream=None):
+                           length: Optional[torch.Tensor] = None, stream=None, per_step: bool = True):
     rows, width, ld = _logits_layout(table)
     V = width if V is None else V
     if rows < V:
         raise ValueError("bigram table needs at least V rows")
     lanes = prev.numel()
     dev = table.device
+    if codes_final is None and per_step:    # also the loop's state for the per-step kernels
+        codes_final = torch.empty(lanes, dtype=torch.float64, device=dev)
     if seq is None:
         seq = torch.empty((lanes, T), dtype=torch.int32, device=dev)
     if length is None:

@@ -105,13 +105,13 @@ static int launch_staged(const StepArgs& a, size_t smem, int sms, int want_per_s
     return AS_OK;
 }
 
-template <int DT, int CAPV, int MINB, bool UA>
+template <int DT, int CAPV, int MINB, bool UA, bool GATHER = false>
 static int launch_stream_ua(const StepArgs& a, int stages, int sms, int want_per_sm, cudaStream_t st) {
     static bool attr_set[64] = {false};
     static int per_sm_cache[64][SK_MAXSTAGES + 1] = {{0}};
     int dev = 0;
     cudaGetDevice(&dev);
-    auto kern = step_stream_kernel<DT, CAPV, MINB, UA>;
+    auto kern = step_stream_kernel<DT, CAPV, MINB, UA, GATHER>;
     cudaError_t e;
     if (!attr_set[dev]) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_OPTIN_MAX - 1024));
@@ -141,6 +141,7 @@ static int launch_stream_ua(const StepArgs& a, int stages, int sms, int want_per
 // copies each row from the boundary below its start
 template <int DT, int CAPV, int MINB>
 static int launch_stream(const StepArgs& a, bool unaligned, int stages, int sms, int want_per_sm, cudaStream_t st) {
+    if (a.row_idx) return launch_stream_ua<DT, CAPV, MINB, true, true>(a, stages, sms, want_per_sm, st);   // table rows: any alignment
     return unaligned ? launch_stream_ua<DT, CAPV, MINB, true>(a, stages, sms, want_per_sm, st)
                      : launch_stream_ua<DT, CAPV, MINB, false>(a, stages, sms, want_per_sm, st);
 }
@@ -297,6 +298,42 @@ encode_generic_kernel(const void* __restrict__ table, int V, long long ld, const
     }
 }
 
+// Decode loop as one launch of the streaming kernel per step (lanes with a top-k / nucleus cut):
+// set-up and wrap-up.  The state lives in the caller's outputs: the codes in codes_final, the
+// previous token in the sequence itself (column t-1; for step 0 the start tokens are parked in
+// `len`, which the wrap-up overwrites), a finished lane being one whose previous entry is the
+// padding or EOS.
+__global__ void decode_setup_kernel(const int* __restrict__ start_or_prev, const double* __restrict__ codes_in,
+                                    int lanes, int N, double u, int V, int T, int* __restrict__ idx0,
+                                    double* __restrict__ codes, int* __restrict__ seq, int* __restrict__ lane_status) {
+    const size_t total = (size_t)lanes * T;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) seq[i] = -1;
+    for (int ln = blockIdx.x * blockDim.x + threadIdx.x; ln < lanes; ln += gridDim.x * blockDim.x) {
+        int prev;
+        double c;
+        if (codes_in) {
+            prev = start_or_prev[ln];
+            c = codes_in[ln];
+        } else {
+            prev = start_or_prev[ln / N];
+            c = ((double)(ln % N) + u) / (double)N;
+            if (c >= 1.0) c -= 1.0;
+        }
+        const bool ok = prev >= 0 && prev < V;
+        idx0[ln] = ok ? prev : -1;
+        codes[ln] = c;
+        if (lane_status) lane_status[ln] = ok ? ST_OK : ST_NUMERIC;
+    }
+}
+
+__global__ void decode_wrapup_kernel(const int* __restrict__ seq, int lanes, int T, int* __restrict__ len) {
+    for (int ln = blockIdx.x * blockDim.x + threadIdx.x; ln < lanes; ln += gridDim.x * blockDim.x) {
+        int n = 0;
+        while (n < T && seq[(size_t)ln * T + n] >= 0) ++n;
+        len[ln] = n;
+    }
+}
+
 // ---------------------------------------------------------------------------
 // argument checks
 // ---------------------------------------------------------------------------
@@ -402,6 +439,30 @@ int as_lattice_codes_variant(int N, double b, int variant, double* d_codes, void
 
 }  // extern "C"
 
+// The streaming kernel for one step: one CTA per lane; rows of up to 6 stages (96 KB) stay resident
+// in the ring.  Sets a.fast.  AS_ERR_UNSUPPORTED (no message): this step is not for that kernel.
+static int launch_streaming(StepArgs& a, int dtype, bool unaligned, int sms, cudaStream_t st) {
+    const int E = dtype == AS_F32 ? 4 : 8;
+    const bool off_grid = unaligned || a.row_idx != nullptr;
+    const size_t row_bytes = (size_t)((a.V + (off_grid ? E - 1 : 0) + E - 1) / E) * 16;
+    const int nsl = (int)((row_bytes + SK_STAGE_BYTES - 1) / SK_STAGE_BYTES);
+    // rows of up to SK_RES_STAGES stages stay resident unless a smaller ring is asked for
+    const bool resident = nsl <= SK_RES_STAGES && !(g_tune_stages > 0 && g_tune_stages < nsl);
+    a.fast = (a.top_k > 0 && a.top_k <= (resident ? SK_K0_RESIDENT : SK_K0_STREAMED)) || (a.top_k == 0 && a.top_p < 1.0);
+    if (!(resident || a.fast)) return AS_ERR_UNSUPPORTED;
+    int stages = resident ? (nsl < 1 ? 1 : nsl) : (g_tune_stages > 0 ? g_tune_stages : 3);
+    if (!resident && stages >= nsl) stages = nsl - 1;
+    if (dtype == AS_F32) {
+        if (!resident && g_tune_minb != 2)
+            return launch_stream<DT_F32, 1536, 3>(a, unaligned, stages < 2 ? stages : 2, sms, g_tune_ctas, st);
+        return launch_stream<DT_F32, 2048, 2>(a, unaligned, stages, sms, g_tune_ctas, st);
+    }
+    // bf16 rows that stream: a 1024-entry hit list and <= 72 registers let three CTAs share an SM
+    if (!resident && g_tune_minb != 2)
+        return launch_stream<DT_BF16, 1024, 3>(a, unaligned, stages < 3 ? stages : 3, sms, g_tune_ctas, st);
+    return launch_stream<DT_BF16, 2048, 2>(a, unaligned, stages, sms, g_tune_ctas, st);
+}
+
 // as_step and as_step_lattice: lat_N = 0 reads d_codes, lat_N > 0 forms the lattice codes in the kernel
 static int step_common(const void* d_logits, int dtype, int lanes, int V, long long ld, const double* d_codes,
                        int lat_N, int lat_j0, double lat_u, double temp, int top_k, double top_p,
@@ -426,30 +487,15 @@ static int step_common(const void* d_logits, int dtype, int lanes, int V, long l
     a.ld = ld; a.inv_tau = inv_tau; a.top_p = top_p; a.scale2 = (float)(1.4426950408889634 / temp);
     a.lanes = lanes; a.V = V; a.top_k = top_k;
     a.lat_N = lat_N; a.lat_j0 = lat_j0; a.lat_u = lat_u;
+    a.row_idx = nullptr; a.idx_stride = 1; a.tok_stride = 1; a.eos = -1; a.rows = 0;
     const int E = dtype == AS_F32 ? 4 : 8;
     const size_t esz = dtype == AS_F32 ? 4 : 2;
     // some row starts off a 16-byte boundary: it is read from the boundary below, up to E-1 elements longer
     const bool unaligned = (reinterpret_cast<uintptr_t>(d_logits) & 15) != 0 || (((size_t)ld * esz) & 15) != 0;
     const size_t row_bytes = (size_t)((V + (unaligned && g_tune_path == 0 ? E - 1 : 0) + E - 1) / E) * 16;
     if (g_tune_path == 0) {
-        // streaming kernel: one CTA per lane; rows of up to 6 stages (96 KB) stay resident in the ring
-        const int nsl = (int)((row_bytes + SK_STAGE_BYTES - 1) / SK_STAGE_BYTES);
-        // rows of up to SK_RES_STAGES stages stay resident unless a smaller ring is asked for
-        const bool resident = nsl <= SK_RES_STAGES && !(g_tune_stages > 0 && g_tune_stages < nsl);
-        a.fast = (top_k > 0 && top_k <= (resident ? SK_K0_RESIDENT : SK_K0_STREAMED)) || (top_k == 0 && top_p < 1.0);
-        if (resident || a.fast) {
-            int stages = resident ? (nsl < 1 ? 1 : nsl) : (g_tune_stages > 0 ? g_tune_stages : 3);
-            if (!resident && stages >= nsl) stages = nsl - 1;
-            if (dtype == AS_F32) {
-                if (!resident && g_tune_minb != 2)
-                    return launch_stream<DT_F32, 1536, 3>(a, unaligned, stages < 2 ? stages : 2, di->sms, g_tune_ctas, st);
-                return launch_stream<DT_F32, 2048, 2>(a, unaligned, stages, di->sms, g_tune_ctas, st);
-            }
-            // bf16 rows that stream: a 1024-entry hit list and <= 72 registers let three CTAs share an SM
-            if (!resident && g_tune_minb != 2)
-                return launch_stream<DT_BF16, 1024, 3>(a, unaligned, stages < 3 ? stages : 3, di->sms, g_tune_ctas, st);
-            return launch_stream<DT_BF16, 2048, 2>(a, unaligned, stages, di->sms, g_tune_ctas, st);
-        }
+        rc = launch_streaming(a, dtype, unaligned, di->sms, st);
+        if (rc != AS_ERR_UNSUPPORTED) return rc;
     }
     if (g_tune_path == 2) {
         // cluster kernel: the row split over CS CTAs' shared memory
@@ -610,8 +656,46 @@ static int decode_common(const void* d_table, int dtype, int V, long long ld, co
     if (top_k < 0 || top_k >= V) top_k = 0;
     if (!(top_p > 0.0 && top_p < 1.0)) top_p = 1.0;
     const double inv_tau = 1.0 / temp;
-    const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
     cudaStream_t st = (cudaStream_t)stream;
+    if ((top_k > 0 || top_p < 1.0) && g_tune_path == 0 && d_codes_final && T > 0) {
+        // lanes with a cut: one launch of the streaming kernel per step, rows gathered from the table
+        StepArgs a;
+        a.logits = d_table; a.codes = d_codes_final; a.codes_out = d_codes_final;
+        a.diag = {nullptr, nullptr, nullptr, d_lane_status, nullptr};
+        a.ld = ld; a.inv_tau = inv_tau; a.top_p = top_p; a.scale2 = (float)(1.4426950408889634 / temp);
+        a.lanes = lanes; a.V = V; a.top_k = top_k;
+        a.lat_N = 0; a.lat_j0 = 0; a.lat_u = 0.0;
+        a.rows = V;
+        cudaError_t e;
+        bool served = true;
+        for (int t = 0; t < T && served; ++t) {
+            a.tokens = d_seq + t; a.tok_stride = T;
+            a.row_idx = t == 0 ? d_len : d_seq + (t - 1);
+            a.idx_stride = t == 0 ? 1 : T;
+            a.eos = (t == 0 || eos < 0) ? -1 : eos;          // a start token may equal EOS
+            if (t == 0) {
+                // is this a step for the streaming kernel at all?  (decided before anything is written)
+                StepArgs probe = a;
+                const int E = dtype == AS_F32 ? 4 : 8;
+                const size_t row_bytes = (size_t)((V + E - 1 + E - 1) / E) * 16;
+                const int nsl = (int)((row_bytes + SK_STAGE_BYTES - 1) / SK_STAGE_BYTES);
+                const bool resident = nsl <= SK_RES_STAGES && !(g_tune_stages > 0 && g_tune_stages < nsl);
+                probe.fast = (top_k > 0 && top_k <= (resident ? SK_K0_RESIDENT : SK_K0_STREAMED)) || (top_k == 0 && top_p < 1.0);
+                if (!(resident || probe.fast)) { served = false; break; }
+                const int sg = grid_for(lanes, di->sms, 8);
+                decode_setup_kernel<<<sg, 256, 0, st>>>(d_tok, d_codes_in, lanes, N, u, V, T, d_len, d_codes_final, d_seq, d_lane_status);
+                if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "decode set-up kernel launch");
+            }
+            rc = launch_streaming(a, dtype, true, di->sms, st);
+            if (rc != AS_OK) return rc == AS_ERR_UNSUPPORTED ? set_err(AS_ERR_CUDA, "streaming kernel refused a decode step") : rc;
+        }
+        if (served) {
+            decode_wrapup_kernel<<<grid_for(lanes, di->sms, 8), 256, 0, st>>>(d_seq, lanes, T, d_len);
+            if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "decode wrap-up kernel launch");
+            return AS_OK;
+        }
+    }
+    const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
     if (dtype == AS_F32)
         decode_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_table, V, ld, d_tok, d_codes_in, lanes, N, u, T, eos, inv_tau, top_k, top_p, d_seq, d_len, d_codes_final, d_lane_status);
     else

@@ -80,6 +80,15 @@ struct StepArgs {
     int lat_N;
     int lat_j0;
     double lat_u;
+    // Row gather (builds with GATHER; the decode loop over a table): lane ln reads row
+    // row_idx[ln * idx_stride] of `logits`; a lane whose index is negative, equal to `eos` or
+    // not below `rows` is skipped altogether (nothing read, nothing written).  Tokens go to
+    // tokens[ln * tok_stride].
+    const int* row_idx;
+    int idx_stride;
+    int tok_stride;
+    int eos;
+    int rows;
 };
 
 __device__ __forceinline__ double lane_code(const StepArgs& a, int ln) {

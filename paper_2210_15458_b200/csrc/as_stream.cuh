@@ -468,7 +468,7 @@ __device__ __forceinline__ void mask_lead(uint4& q, int lead) {
     q = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-template <int DT, int CAPV, int MINB, bool UA = false>
+template <int DT, int CAPV, int MINB, bool UA = false, bool GATHER = false>
 __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const StepArgs a, const int stages) {
     using StreamSmem = StreamSmemT<CAPV>;
     constexpr int SK_CAPV = CAPV;
@@ -492,8 +492,15 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
     const bool resident = nsl <= stages;
     const int S = resident ? max(nsl, 1) : stages;                     // ring length in use
 
+    // GATHER: the row comes from a table through an index; lanes without a usable index sit out
+    auto lane_row = [&](int ln) -> int { return GATHER ? a.row_idx[(size_t)ln * a.idx_stride] : ln; };
+    auto lane_active = [&](int ln) -> bool {
+        if (!GATHER) return true;
+        const int i = lane_row(ln);
+        return i >= 0 && i != a.eos && i < a.rows;
+    };
     auto row_of = [&](int ln) -> const char* {
-        return reinterpret_cast<const char*>(a.logits) + (size_t)ln * (size_t)a.ld * Tr::BYTES;
+        return reinterpret_cast<const char*>(a.logits) + (size_t)lane_row(ln) * (size_t)a.ld * Tr::BYTES;
     };
     auto staged_ok = [&](int ln) -> bool { return UA || (reinterpret_cast<uintptr_t>(row_of(ln)) & 15) == 0; };
     auto lead_of = [&](int ln) -> int {
@@ -516,6 +523,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
     int s_issue = 0;
     auto issue_some = [&](bool first_row_only) -> bool {   // false: a bounded wait ran out
         for (; ln_issue < a.lanes; ln_issue += gridDim.x, s_issue = 0) {
+            if (GATHER && !lane_active(ln_issue)) continue;
             if (!staged_ok(ln_issue)) continue;
             int bulk_bytes_i = bulk_bytes, nsl_i = nsl;
             const int lead_i = lead_of(ln_issue);
@@ -641,6 +649,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
     };
 
     for (int ln = blockIdx.x; ln < a.lanes; ln += gridDim.x) {
+        if (GATHER && !lane_active(ln)) continue;
         // the code is first looked at just before the epilogue: its 8-byte load queues behind the
         // row copies of the whole grid, and an earlier use would hold up the passes over the row
         const double c_in = lane_code(a, ln);
@@ -973,7 +982,15 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                 for (int s = 0; s < nsl_l; ++s) release(g + s);
         }
         if (resident && staged_ok(ln)) g += nsl_l;
-        if (tid == 0) write_result(a, ln, r, path);
+        if (tid == 0) {
+            if (GATHER) {
+                a.tokens[(size_t)ln * a.tok_stride] = r.token;
+                a.codes_out[ln] = r.code_out;
+                if (a.diag.lane_status && r.status != ST_OK) a.diag.lane_status[ln] = r.status;
+            } else {
+                write_result(a, ln, r, path);
+            }
+        }
         SyncC::sync();
         ASX_MARK(12);
     }

@@ -553,3 +553,38 @@ def test_step_rows_off_the_16_byte_grid_take_the_fast_path(B, orc, dtype, V, pad
             assert (d["path"].cpu().numpy() == B.PATH_COMPACT).sum() >= lanes - 3
     # no cut at all: the general routine, still correct
     check(B, orc, arr[:4], dtype, codes[:4], 1.0, 0, 1.0, what="off-grid rows, no cut")
+
+
+def test_decode_with_cuts_per_step_kernels_equal_the_single_kernel(B, orc):
+    # with a cut and a codes_final buffer the loop runs as one launch of the step kernel per step
+    # (rows gathered from the table); without the buffer, as one general kernel.  Both follow the
+    # same arithmetic up to rounding: sequences agree wherever the oracle's margins are safe.
+    rng = np.random.default_rng(77)
+    for dtype, V, ld, eos, temp, k, p in [(BF16, 3000, 3000, 5, 0.8, 12, 1.0), (F32, 2001, 2003, -1, 1.1, 0, 0.85),
+                                          (BF16, 70001, 70001, 0, 0.7, 40, 0.95)]:
+        x = rng.normal(0, 2.5, (V, ld)).astype(np.float32)
+        if eos >= 0:
+            x[:, eos] += 4.0
+        table = _store(x, dtype)
+        dev = to_dev(table, dtype)
+        lanes, T = 40, 10
+        prev = rng.integers(0, V, lanes).astype(np.int32)
+        prev[3] = V + 7                                             # out of range: status, no tokens
+        codes = rng.random(lanes)
+        outs = []
+        for per_step in (True, False):
+            st = torch.empty(lanes, dtype=torch.int32, device="cuda")
+            cf = torch.empty(lanes, dtype=torch.float64, device="cuda") if per_step else None
+            seq, ln = B.as_decode_bigram_codes(dev, torch.from_numpy(prev).cuda(), torch.from_numpy(codes).cuda(), T,
+                                               eos, temp, k, p, V=V, codes_final=cf, lane_status=st, per_step=per_step)
+            torch.cuda.synchronize()
+            outs.append((seq.cpu().numpy(), ln.cpu().numpy(), st.cpu().numpy()))
+        (s1, l1, t1), (s2, l2, t2) = outs
+        assert t1[3] == B.ERR_NUMERIC and t2[3] == B.ERR_NUMERIC and l1[3] == 0 and (s1[3] == -1).all()
+        # the first tokens can only differ inside the boundary band; count whole-prefix agreement
+        agree = [(s1[i, :4] == s2[i, :4]).all() for i in range(lanes)]
+        assert np.mean(agree) > 0.9
+        for i in range(lanes):
+            assert (s1[i, l1[i]:] == -1).all() and (s1[i, :l1[i]] >= 0).all()
+            if 0 < l1[i] < T:
+                assert s1[i, l1[i] - 1] == eos
