@@ -316,6 +316,25 @@ def bench_bigram(steps: int, warmup: int, S: int = 64, T: int = 128):
                      "mean_len": tokens / w.lanes,
                      "row_gbs_upper": tokens * w.V * w.elem_bytes / ms / 1e6,
                      "duplicate_prefix_rate": dup_rates(seq)}
+    # the same loop with a cut (Sec. 5.1 "Top-k sampling": k = 2 and 10; a nucleus): one launch of
+    # the streaming step kernel per step, rows gathered from the table
+    cf = torch.empty(w.lanes, dtype=torch.float64, device="cuda")
+    for name, k, p in (("top_k_2", 2, 1.0), ("top_k_10", 10, 1.0), ("top_p_0.9", 0, 0.9)):
+        fn = lambda: B.as_decode_bigram(table, starts, w.N, w.shift(), w.T, w.eos, w.temp, k, p, seq=seq, length=ln,
+                                        codes_final=cf)
+        for _ in range(max(1, warmup)):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(steps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / steps
+        tokens = int(ln.sum().item())
+        out["lattice_" + name] = {"ms_per_decode": ms, "tokens": tokens, "tokens_per_s": tokens / ms * 1e3,
+                                  "launches_per_decode": w.T + 2}
     # the other direction on the sequences just decoded: sequence -> interval, same tokens
     run_iid()
     fn = lambda: B.as_encode_bigram(table, prev, seq, ln, w.temp, w.top_k, w.top_p)
