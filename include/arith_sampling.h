@@ -24,9 +24,11 @@
  *   - There is no CPU implementation behind these calls: without a usable CUDA
  *     device they return AS_ERR_CUDA.
  *   - Logits are row-major [rows, ld] with ld >= V elements between rows, dtype
- *     AS_F32 (IEEE binary32) or AS_BF16 (bfloat16 bit patterns).  Rows whose
- *     address and pitch are multiples of 16 bytes take the bulk-copy path; other
- *     layouts are accepted and take a slower load path.
+ *     AS_F32 (IEEE binary32) or AS_BF16 (bfloat16 bit patterns).  The base
+ *     pointer and the pitch need only be element-aligned: rows that start off a
+ *     16-byte boundary are bulk-copied from the boundary below their start (the
+ *     bytes in front lie in the same 16-byte granule and are masked), at nearly
+ *     the speed of aligned rows.
  *   - Codes are fp64 in [0,1).  An input code of exactly 1.0 is read as the
  *     largest double below 1.  Rescaled codes are clamped to [0, 1 - 2^-53].
  *
