@@ -2,7 +2,7 @@
 // communication (lanes are independent: Remark after Proposition 1).
 //
 // CTA = 8 consumer warps + 1 producer warp.  The producer's lane 0 feeds a ring of
-// 16 KB shared-memory stages with bulk async copies (TMA, non-multicast; `full`
+// 16 KB shared-memory stages with bulk async copies (TMA, each into this CTA only; `full`
 // mbarrier per stage carries the byte count, `empty` mbarrier per stage collects
 // one arrival per consumer warp), running ahead across rows, so HBM reads never
 // wait for compute.  Consumers see each row exactly once (Algorithm 1 needs every
