@@ -200,8 +200,9 @@ __device__ __forceinline__ int warp_suffix_i(int v, int lane) {
 // degree-5 polynomial (truncation ~3e-17).  One fused multiply-add upstream forms t, so the
 // whole evaluation is 10 fp64 operations.  Arguments below -64000 (2^-1000) return 0.
 // ---------------------------------------------------------------------------
+template <bool GUARD = true>
 __device__ __forceinline__ double exp2_64th(double t, const double* __restrict__ tbl) {
-    if (!(t >= -64000.0)) return 0.0;
+    if (GUARD && !(t >= -64000.0)) return 0.0;     // (without the guard the caller vouches for t >= -64000)
     const double MAGIC = 6755399441055744.0;
     double r = t + MAGIC;
     const int k = __double2loint(r);
@@ -221,6 +222,11 @@ __device__ __forceinline__ double exp2_64th(double t, const double* __restrict__
 // ---------------------------------------------------------------------------
 // Packed NaN-propagating maxima and float views of one 16-byte vector.
 // ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t min_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("min.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
 __device__ __forceinline__ uint32_t max_nan_bf16x2(uint32_t a, uint32_t b) {
     uint32_t d;
     asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
@@ -279,6 +285,11 @@ template <> struct Pass<DT_BF16> {
         return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
     }
     __device__ static uint32_t key_of_f(float x) { return Traits<DT_BF16>::key_of(__float_as_uint(x) >> 16); }
+    // min of the 8 elements (NaN-free data; a NaN is caught by the max pass)
+    __device__ static float vmin(const uint4& q) {
+        const uint32_t m = min_bf16x2(min_bf16x2(q.x, q.y), min_bf16x2(q.z, q.w));
+        return fminf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+    }
 };
 template <> struct Pass<DT_F32> {
     struct Acc { float a, b; };
@@ -312,6 +323,10 @@ template <> struct Pass<DT_F32> {
                      fmaxf(__uint_as_float(q.z), __uint_as_float(q.w)));
     }
     __device__ static uint32_t key_of_f(float x) { return Traits<DT_F32>::key_of(__float_as_uint(x)); }
+    __device__ static float vmin(const uint4& q) {
+        return fminf(fminf(__uint_as_float(q.x), __uint_as_float(q.y)),
+                     fminf(__uint_as_float(q.z), __uint_as_float(q.w)));
+    }
 };
 
 // Result of one decode step for one lane, identical in every thread of the CTA.

@@ -344,18 +344,26 @@ struct GenericLane {
         if (c == 1.0) c = ASX_ONE_BELOW;
         // ---- 1. maximum (NaN and +inf propagate into it)
         typename P::Acc acc = P::init();
+        float vmn = __uint_as_float(0x7F800000u);                    // the row's minimum, for the plain case below
         const int nvf = (V * Tr::BYTES) >> 4;
-        for (int vi = tid; vi < nvf; vi += NT)
-            P::merge(acc, P::reduce(*reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row) + (size_t)vi * 16)));
-        for (int j = nvf * E + tid; j < V; j += NT) P::fold_scalar(acc, row, j);
+        for (int vi = tid; vi < nvf; vi += NT) {
+            const uint4 q = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row) + (size_t)vi * 16);
+            P::merge(acc, P::reduce(q));
+            vmn = fminf(vmn, P::vmin(q));
+        }
+        for (int j = nvf * E + tid; j < V; j += NT) {
+            P::fold_scalar(acc, row, j);
+            vmn = fminf(vmn, P::load_f(row, j));
+        }
         uint32_t k0, k1;
         P::keys(acc, k0, k1);
         uint32_t kmax = warp_max_u(max(k0, k1));
-        if (lane == 0) sm.red_u[warp] = kmax;
+        uint32_t kmin = warp_min_u(P::key_of_f(vmn));
+        if (lane == 0) { sm.red_u[warp] = kmax; sm.red_u2[warp] = kmin; }
         if (tid == 0) sm.b_i[2] = 0;
         Sync::sync();
-        kmax = 0;
-        for (int w = 0; w < NW; ++w) kmax = max(kmax, sm.red_u[w]);
+        kmax = 0; kmin = 0xFFFFFFFFu;
+        for (int w = 0; w < NW; ++w) { kmax = max(kmax, sm.red_u[w]); kmin = min(kmin, sm.red_u2[w]); }
         if (code_bad || kmax >= Tr::KEY_PINF || kmax <= Tr::KEY_NINF) {
             Sync::sync();
             return fail(c_in, ST_NUMERIC);
@@ -363,6 +371,10 @@ struct GenericLane {
         lmax = (double)Tr::value_f(kmax);
         const double s64 = inv_tau * 0x1.71547652b82fep+6;          // 64 log2(e) / temp
         const double c64 = -lmax * s64;
+        // The plain case -- no masked token, and no mass below 2^-1000 of the largest: every token
+        // is kept and the exponential needs no underflow guard, which shortens the loop that every
+        // logit of every step goes through.
+        const bool plain = kmin > Tr::KEY_NINF && fma((double)Tr::value_f(kmin), s64, c64) >= -64000.0;
         // ---- 2. per-chunk masses in index order
         int nfin = 0;
         for (int ci = warp; ci < nchunks; ci += NW) {
@@ -371,10 +383,15 @@ struct GenericLane {
                 float x[E];
                 int base;
                 chunk_floats(ci, r, x, base);
+                if (plain && base + E <= V) {        // (a vector reaching past V holds -inf padding: guarded)
 #pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    local += exp2_64th(fma((double)x[e], s64, c64), sm.exp_tbl);
-                    nfin += (x[e] > __uint_as_float(0xFF800000u));
+                    for (int e = 0; e < E; ++e) local += exp2_64th<false>(fma((double)x[e], s64, c64), sm.exp_tbl);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        local += exp2_64th(fma((double)x[e], s64, c64), sm.exp_tbl);
+                        nfin += (x[e] > __uint_as_float(0xFF800000u));
+                    }
                 }
             }
             local = warp_sum_d(local);
@@ -387,7 +404,7 @@ struct GenericLane {
         // ---- 3. the chunk, then the element, whose interval holds c * Z
         const double Z = sm.chunk_sum[nchunks];
         const double t = c * Z;
-        const int n_kept = sm.b_i[2];
+        const int n_kept = plain ? V : sm.b_i[2];
         if (tid == 0) { sm.b_i[0] = INT_MAX; sm.b_i[1] = -1; }
         Sync::sync();
         for (int ci = tid; ci < nchunks; ci += NT) {
@@ -679,17 +696,25 @@ struct GenericLane {
         inv_tau = inv_tau_;
         fill_exp_table(sm.exp_tbl, tid);
         typename P::Acc acc = P::init();
+        float vmn = __uint_as_float(0x7F800000u);
         const int nvf = (V * Tr::BYTES) >> 4;
-        for (int vi = tid; vi < nvf; vi += NT)
-            P::merge(acc, P::reduce(*reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row) + (size_t)vi * 16)));
-        for (int j = nvf * E + tid; j < V; j += NT) P::fold_scalar(acc, row, j);
+        for (int vi = tid; vi < nvf; vi += NT) {
+            const uint4 q = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row) + (size_t)vi * 16);
+            P::merge(acc, P::reduce(q));
+            vmn = fminf(vmn, P::vmin(q));
+        }
+        for (int j = nvf * E + tid; j < V; j += NT) {
+            P::fold_scalar(acc, row, j);
+            vmn = fminf(vmn, P::load_f(row, j));
+        }
         uint32_t k0, k1;
         P::keys(acc, k0, k1);
         uint32_t kmax = warp_max_u(max(k0, k1));
-        if (lane == 0) sm.red_u[warp] = kmax;
+        uint32_t kmin = warp_min_u(P::key_of_f(vmn));
+        if (lane == 0) { sm.red_u[warp] = kmax; sm.red_u2[warp] = kmin; }
         Sync::sync();
-        kmax = 0;
-        for (int w = 0; w < NW; ++w) kmax = max(kmax, sm.red_u[w]);
+        kmax = 0; kmin = 0xFFFFFFFFu;
+        for (int w = 0; w < NW; ++w) { kmax = max(kmax, sm.red_u[w]); kmin = min(kmin, sm.red_u2[w]); }
         if (kmax >= Tr::KEY_PINF || kmax <= Tr::KEY_NINF) {
             Sync::sync();
             return fail(0.0, ST_NUMERIC);
@@ -697,11 +722,25 @@ struct GenericLane {
         lmax = (double)Tr::value_f(kmax);
         const double s64 = inv_tau * 0x1.71547652b82fep+6;          // 64 log2(e) / temp
         const double c64 = -lmax * s64;
+        // plain rows (no masked token, nothing below 2^-1000 of the largest mass): no underflow guard,
+        // every token counts, and whole vectors on one side of the token need no per-element test
+        const bool plain = kmin > Tr::KEY_NINF && fma((double)Tr::value_f(kmin), s64, c64) >= -64000.0;
         double all = 0.0, below = 0.0, e_tok = 0.0;
         int has = 0, nfin = 0;
         for (int vi = tid; vi < nvec; vi += NT) {
             float x[E];
             const int base = vi * E;
+            if (plain && base + E <= V && (base + E <= tok || base > tok)) {
+                const uint4 q = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row) + (size_t)base * Tr::BYTES);
+                P::floats(q, x);
+                double vsum = 0.0;
+#pragma unroll
+                for (int e = 0; e < E; ++e) vsum += exp2_64th<false>(fma((double)x[e], s64, c64), sm.exp_tbl);
+                all += vsum;
+                if (base < tok) below += vsum;
+                nfin += E;
+                continue;
+            }
             if (base + E <= V) {
                 const uint4 q = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row) + (size_t)base * Tr::BYTES);
                 P::floats(q, x);
