@@ -383,26 +383,27 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2,
     uint32_t depth_key = P::key_of_f(t1f);
     if (Tr::value_f(depth_key) < t1f) depth_key += 1;     // smallest key whose value is >= t1
     SyncC::sync();
-    // ---- 3. collect afresh
-    float tail = 0.f;
+    // ---- 3. collect afresh.  The mass outside the new list is the old one less the tokens that
+    //         join now (those below the old threshold): an exponential for a few hundred elements,
+    //         not for the whole row again.
+    float joined = 0.f;
     visit([&](float x, int j) {
-        bool hit = false;
         if (x >= t1f) {
             const uint32_t key = P::key_of_f(x);
             if (key > Tr::KEY_NINF) {
-                hit = true;
                 const int slot = atomicAdd(&sm.cand_count, 1);
                 if (slot < SK_CAP) sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)j;
+                if (x < t0f) joined += ex2_approx((x - lmaxf) * scale2);
             }
         }
-        if (!hit) tail += ex2_approx((x - lmaxf) * scale2);
     });
-    const double td = warp_sum_d((double)tail);
+    const double td = warp_sum_d((double)joined);
     if (lane == 0) sm.red_d[warp] = td;
     SyncC::sync();
-    double tsum = 0.0;
+    double tsum = tailsum;
 #pragma unroll
-    for (int w = 0; w < SK_NW; ++w) tsum += sm.red_d[w];
+    for (int w = 0; w < SK_NW; ++w) tsum -= sm.red_d[w];
+    if (tsum < 0.0) tsum = 0.0;
     const int C = sm.cand_count;
     if (C <= 0 || C > SK_CAP || !(tsum == tsum) || !(tsum < 1e300)) { ASX_COUNT(3); return false; }
     const bool ok2 = epilogue_ranked<DT, NT, SyncC, StreamSmem>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, depth_key, c,
