@@ -7,7 +7,7 @@ A step is one pass of the decode hot path over one batch of synthetic input: a f
 shifted lattice of codes and one decode step for every lane, in one launch (as_step_lattice
 forms the codes in the step kernel; the two-call form is timed beside it).
 The default workload is the 256-lane x 32000-token bf16 step (temperature 0.7, top_k 40).
-Rank 0 prints ONE JSON line; see README/DESIGN for the keys.  With N > 1 (torchrun) every
+Rank 0 prints ONE JSON line.  With N > 1 (torchrun) every
 rank decodes its own batch (lanes never communicate), so scaling is weak and there is no
 data-path collective: only the timing is reduced (max over ranks).
 

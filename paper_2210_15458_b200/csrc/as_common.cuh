@@ -144,21 +144,10 @@ __device__ __forceinline__ double warp_sum_d(double v) {
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
     return v;
 }
-__device__ __forceinline__ int warp_sum_i(int v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
-    return v;
-}
-__device__ __forceinline__ unsigned warp_max_u(unsigned v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(FULL, v, o));
-    return v;
-}
-__device__ __forceinline__ unsigned warp_min_u(unsigned v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(FULL, v, o));
-    return v;
-}
+// 32-bit integer reductions: one redux.sync instruction each instead of five shuffle steps
+__device__ __forceinline__ int warp_sum_i(int v) { return __reduce_add_sync(FULL, v); }
+__device__ __forceinline__ unsigned warp_max_u(unsigned v) { return __reduce_max_sync(FULL, v); }
+__device__ __forceinline__ unsigned warp_min_u(unsigned v) { return __reduce_min_sync(FULL, v); }
 // inclusive scans over lanes 0..31 in lane order
 __device__ __forceinline__ double warp_incl_scan_d(double v, int lane) {
 #pragma unroll

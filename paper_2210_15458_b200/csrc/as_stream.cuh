@@ -84,9 +84,25 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 
 // m-th largest (1-based) of the 64 16-bit keys held two per lane, by a search on the value, two
 // bits per step: the largest v with count(keys >= v) >= m (0 if fewer than m keys are positive).
+// Up to SEL_PEEL_MAX the maximum is taken off the top m times instead.
+constexpr int SEL_PEEL_MAX = 12;
 __device__ __forceinline__ uint32_t warp_select16(uint32_t a16, uint32_t b16, int m, uint32_t lo16 = 0) {
     // Only an answer above lo16 (the threshold already in force) is of use, and it cannot exceed the
     // warp's maximum: search the bits below their common prefix.  0 = no bound above lo16.
+    if (m <= SEL_PEEL_MAX) {
+        // small m: take the maximum off the top m times (one redux and one ballot per round, against
+        // six ballots per two bits of the search below); duplicates count once each, as they must
+        uint32_t v = 0;
+#pragma unroll 1
+        for (int r = 0; r < m; ++r) {
+            const uint32_t mx = max(a16, b16);
+            v = warp_max_u(mx);
+            if (v <= lo16) return 0;             // (also: fewer than m positive keys)
+            const int owner = __ffs(__ballot_sync(FULL, mx == v)) - 1;
+            if ((int)(threadIdx.x & 31) == owner) { if (a16 == v) a16 = 0; else b16 = 0; }
+        }
+        return v;
+    }
     const uint32_t hi16 = warp_max_u(max(a16, b16));
     if (hi16 <= lo16) return 0;
     int nb = 32 - __clz(lo16 ^ hi16);            // differing low bits
@@ -120,23 +136,40 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
     // (src[C..C+3] are zero: the caller zero-fills the array before collecting candidates)
     // ---- ranks by (value desc, index asc): composites are distinct -> a permutation; each
     //      thread also computes the mass of its own candidate and stores it by rank
-    for (int i = tid; i < C; i += NT) {
-        const unsigned long long ci = src[i];
-        int r = 0;
+    //      A short list is shared out G threads to a candidate (G a power of two, the G threads
+    //      adjacent lanes of one warp): each counts a G-th of the list, the counts are added by
+    //      shuffles, one of them stores the composite and another the mass.
+    const int kmax = (top_k > 0 && top_k < C) ? top_k : C;
+    const bool topk_only = !(top_p < 1.0);
+    {
+        const int G = C <= NT / 8 ? 8 : C <= NT / 4 ? 4 : C <= NT / 2 ? 2 : 1;
+        const int sub = tid & (G - 1);
+        for (int i0 = 0; i0 < C; i0 += NT / G) {
+            const int i = i0 + tid / G;
+            const bool valid = i < C;
+            const unsigned long long ci = valid ? src[i] : ~0ull;
+            int r = 0;
 #pragma unroll 1
-        for (int j = 0; j < C; j += 4)
-            r += (src[j] > ci) + (src[j + 1] > ci) + (src[j + 2] > ci) + (src[j + 3] > ci);
-        dst[r] = ci;
-        e[r] = exp_nonpos(((double)Tr::value_f((uint32_t)(ci >> 32)) - lmax) * inv_tau, sm.exp_tbl);
+            for (int j = sub * 4; j < C; j += G * 4)
+                r += (src[j] > ci) + (src[j + 1] > ci) + (src[j + 2] > ci) + (src[j + 3] > ci);
+            for (int o = G >> 1; o > 0; o >>= 1) r += __shfl_xor_sync(FULL, r, o);
+            if (valid) {
+                // with a top-k alone nothing past rank kmax is looked at again: zeros there, which
+                // the index loop below relies on
+                if (sub == 0) dst[r] = (topk_only && r >= kmax) ? 0ull : ci;
+                if (sub == (G > 1 ? 1 : 0))
+                    e[r] = exp_nonpos(((double)Tr::value_f((uint32_t)(ci >> 32)) - lmax) * inv_tau, sm.exp_tbl);
+            }
+        }
     }
     ASX_MARK(6);
-    const int kmax = (top_k > 0 && top_k < C) ? top_k : C;
     if (tid < 4) dst[C + tid] = 0ull;             // ~0 = index 0xFFFFFFFF: never "smaller"
     Sync::sync();
+    int n_final, ok;
     if (top_p < 1.0) {
         if (warp == 0) {
             // prefix masses in rank order: nucleus on the distribution renormalised over the survivors
-            int n_final = kmax, ok = 1;
+            int nf = kmax, okw = 1;
             const int per = (kmax + 31) / 32;
             const int b = min(lane * per, kmax), en = min(b + per, kmax);
             double s = 0.0;
@@ -151,40 +184,43 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
             for (int r = b; r < en; ++r) { run += e[r]; below += (run < target); }
             below = warp_sum_i(below);
             if (below >= kmax) {
-                if (top_k == 0) ok = 0;        // nucleus-only: it reaches past the list
+                if (top_k == 0) okw = 0;       // nucleus-only: it reaches past the list
             } else {
-                n_final = below + 1;
+                nf = below + 1;
             }
-            if (ok && (uint32_t)(dst[n_final - 1] >> 32) < depth_key) ok = 0;   // cut below the exact depth
+            if (okw && (uint32_t)(dst[nf - 1] >> 32) < depth_key) okw = 0;   // cut below the exact depth
             __syncwarp();
             if (lane == 0) {
-                sm.b_i[0] = n_final; sm.b_i[1] = ok;
+                sm.b_i[0] = nf; sm.b_i[1] = okw;
                 // entries past the kept ranks must not count in the index loop
-                if (n_final < C) { dst[n_final] = 0ull; dst[n_final + 1] = 0ull; dst[n_final + 2] = 0ull; dst[n_final + 3] = 0ull; }
+                if (nf < C) { dst[nf] = 0ull; dst[nf + 1] = 0ull; dst[nf + 2] = 0ull; dst[nf + 3] = 0ull; }
             }
         }
         Sync::sync();
+        n_final = sm.b_i[0];
+        ok = sm.b_i[1];
     } else {
-        // top-k only: the answer follows from kmax alone
-        if (tid == 0) { sm.b_i[0] = kmax; sm.b_i[1] = ((uint32_t)(dst[kmax - 1] >> 32) >= depth_key) ? 1 : 0; }
-        if (kmax < C) {
-            Sync::sync();
-            if (tid < 4) dst[kmax + tid] = 0ull;  // entries past the kept ranks must not count below
-        }
-        Sync::sync();
+        // top-k only: the answer follows from kmax alone, every thread sees it; the entries past
+        // the kept ranks were stored as zeros
+        n_final = kmax;
+        ok = ((uint32_t)(dst[kmax - 1] >> 32) >= depth_key) ? 1 : 0;
     }
     ASX_MARK(7);
-    const int n_final = sm.b_i[0];
-    if (sm.b_i[1]) {
+    if (ok) {
         // ---- index order among the kept: src is free now, it receives (index << 32) | rank
-        for (int r = tid; r < n_final; r += NT) {
-            const uint32_t idx = ~(uint32_t)dst[r];
+        const int G = n_final <= NT / 8 ? 8 : n_final <= NT / 4 ? 4 : n_final <= NT / 2 ? 2 : 1;
+        const int sub = tid & (G - 1);
+        for (int r0 = 0; r0 < n_final; r0 += NT / G) {
+            const int r = r0 + tid / G;
+            const bool valid = r < n_final;
+            const uint32_t idx = valid ? ~(uint32_t)dst[r] : 0u;
             int ir = 0;
 #pragma unroll 1
-            for (int q = 0; q < n_final; q += 4)
+            for (int q = sub * 4; q < n_final; q += G * 4)
                 ir += (~(uint32_t)dst[q] < idx) + (~(uint32_t)dst[q + 1] < idx) +
                       (~(uint32_t)dst[q + 2] < idx) + (~(uint32_t)dst[q + 3] < idx);
-            src[ir] = ((unsigned long long)idx << 32) | (uint32_t)r;
+            for (int o = G >> 1; o > 0; o >>= 1) ir += __shfl_xor_sync(FULL, ir, o);
+            if (valid && sub == 0) src[ir] = ((unsigned long long)idx << 32) | (uint32_t)r;
         }
         Sync::sync();
         ASX_MARK(8);
@@ -257,7 +293,7 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
     Sync::sync();
     ASX_MARK(10);
     out = sm.res;
-    return sm.b_i[1] != 0;
+    return ok != 0;
 }
 
 // One more pass over a 16-byte aligned row in global memory, f(vector, vector index), thread t
@@ -649,6 +685,37 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         }
     };
 
+    // Elements of one vector that pass the final threshold -> candidate list, token index base + e.
+    // One slot reservation per vector: a reservation per element made up to E dependent atomic round
+    // trips per warp pass (the hits of a warp's lanes sit at different e), which cost more than the
+    // passes over the row.  With with_tail the other elements join the fp32 tail.
+    auto push_vec = [&](const uint4& q, int base, float t0f, uint32_t t0key, bool with_tail, float ref, float& tail) {
+        float x[E];
+        P::floats(q, x);
+        unsigned em = 0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            bool hit = false;
+            if (x[e] >= t0f) {
+                const uint32_t key = P::key_of_f(x[e]);
+                hit = key >= t0key && key > Tr::KEY_NINF;
+            }
+            em |= (hit ? 1u : 0u) << e;
+            if (with_tail && !hit) tail += ex2_approx((x[e] - ref) * scale2);
+        }
+        if (em) {
+            int slot = atomicAdd(&sm.cand_count, __popc(em));
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                if ((em >> e) & 1u) {
+                    if (slot < SK_CAP)
+                        sm.u.ep.cand[slot] = ((unsigned long long)P::key_of_f(x[e]) << 32) | (uint32_t)~(uint32_t)(base + e);
+                    ++slot;
+                }
+            }
+        }
+    };
+
     for (int ln = blockIdx.x; ln < a.lanes; ln += gridDim.x) {
         if (GATHER && !lane_active(ln)) continue;
         // the code is first looked at just before the epilogue: its 8-byte load queues behind the
@@ -799,20 +866,8 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                         hm &= hm - 1;
                         const int s = i / SK_VPT, v = (i % SK_VPT) * NT + tid;
                         const uint4 q = ringv[(size_t)((g + s) % S) * SK_STAGE_VEC + v];
-                        float x[E];
-                        P::floats(q, x);
-#pragma unroll
-                        for (int e = 0; e < E; ++e) {
-                            if (x[e] >= t0f) {
-                                const uint32_t key = P::key_of_f(x[e]);
-                                if (key >= t0key && key > Tr::KEY_NINF) {
-                                    const int slot = atomicAdd(&sm.cand_count, 1);
-                                    if (slot < SK_CAP)
-                                        sm.u.ep.cand[slot] = ((unsigned long long)key << 32) |
-                                                             (uint32_t)~(uint32_t)((s * SK_STAGE_VEC + v) * E + e - lead);
-                                }
-                            }
-                        }
+                        float unused = 0.f;
+                        push_vec(q, (s * SK_STAGE_VEC + v) * E - lead, t0f, t0key, false, ref, unused);
                     }
                 } else {
 #pragma unroll 1
@@ -886,42 +941,10 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                 const uint4 q = sm.u.ep.v.cvec[i];
                 // most listed vectors came in under an earlier, lower threshold
                 if (!want_tail && !(P::part_max(P::reduce(q)) >= t0f)) continue;
-                const int base = sm.u.ep.cidx[i] * E - lead;
-                float x[E];
-                P::floats(q, x);
-#pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    bool hit = false;
-                    if (x[e] >= t0f) {
-                        const uint32_t key = P::key_of_f(x[e]);
-                        if (key >= t0key && key > Tr::KEY_NINF) {
-                            hit = true;
-                            const int slot = atomicAdd(&sm.cand_count, 1);
-                            if (slot < SK_CAP)
-                                sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)(base + e);
-                        }
-                    }
-                    if (want_tail && !hit) tail += ex2_approx((x[e] - ref) * scale2);
-                }
+                push_vec(q, sm.u.ep.cidx[i] * E - lead, t0f, t0key, want_tail, ref, tail);
             }
-            if (tail_elems_l > 0 && tid == 0) {      // the ragged last vector lives in thread 0's registers
-                float x[E];
-                P::floats(qt, x);
-#pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    bool hit = false;
-                    if (x[e] >= t0f) {
-                        const uint32_t key = P::key_of_f(x[e]);
-                        if (key >= t0key && key > Tr::KEY_NINF) {
-                            hit = true;
-                            const int slot = atomicAdd(&sm.cand_count, 1);
-                            if (slot < SK_CAP)
-                                sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)(bulk_vec_l * E + e - lead);
-                        }
-                    }
-                    if (want_tail && !hit) tail += ex2_approx((x[e] - ref) * scale2);
-                }
-            }
+            // the ragged last vector lives in thread 0's registers
+            if (tail_elems_l > 0 && tid == 0) push_vec(qt, bulk_vec_l * E - lead, t0f, t0key, want_tail, ref, tail);
         }
         if (!list_ok && !decided && !general_row && nvh > SK_CAPV && !(UA && lead) && !*(volatile int*)&sm.poisoned) {
             // more hit vectors than the list holds: take the candidates in one more pass, against
