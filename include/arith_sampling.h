@@ -326,6 +326,11 @@ int as_reward_mean(const int32_t *d_seq, const int32_t *d_len, int S, int N, int
  *   AS_TUNE_MIN_CTAS      streaming kernel build for bf16 rows that do not fit the ring:
  *                         3 = three CTAs per SM (1024-entry hit list, <= 72 registers; default),
  *                         2 = two CTAs per SM (2048-entry hit list)
+ *   AS_TUNE_SERIAL_LAUNCH 1 = launch the streaming kernel as an ordinary stream-ordered kernel.
+ *                         By default it is launched so that its CTAs may be set up while the
+ *                         kernel before it on the stream drains (programmatic dependent launch;
+ *                         it still waits for that kernel's completion before it reads or
+ *                         writes global memory, so results do not depend on this key)
  * Returns AS_ERR_INVALID_ARG for an unknown key or value.
  */
 #define AS_TUNE_STEP_PATH 1
@@ -333,6 +338,7 @@ int as_reward_mean(const int32_t *d_seq, const int32_t *d_len, int S, int N, int
 #define AS_TUNE_CTAS_PER_SM 3
 #define AS_TUNE_STAGES 4
 #define AS_TUNE_MIN_CTAS 5
+#define AS_TUNE_SERIAL_LAUNCH 6
 int as_tune(int key, int value);
 
 /* Text of the calling thread's most recent error ("" if none). Never NULL. */

@@ -44,11 +44,22 @@ constexpr long long ST_WAIT_CYCLES = 4000000000LL;   // ~2 s: bound on any mbarr
 #ifdef ASX_PROFILE
 __device__ long long g_asx_marks[32];
 __device__ unsigned long long g_asx_counts[16];
+__device__ unsigned long long g_asx_span[4];      // first / last CTA start, first / last CTA end (globaltimer, ns)
+__device__ __forceinline__ void asx_span(int i) {
+    if (threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        atomicMin(&g_asx_span[i], t);
+        atomicMax(&g_asx_span[i + 1], t);
+    }
+}
+#define ASX_SPAN(i) asx_span(i)
 #define ASX_MARK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_asx_marks[i] = clock64(); } while (0)
 #define ASX_COUNT(i) do { if (threadIdx.x == 0) atomicAdd(&g_asx_counts[i], 1ull); } while (0)
 #else
 #define ASX_MARK(i) do {} while (0)
 #define ASX_COUNT(i) do {} while (0)
+#define ASX_SPAN(i) do {} while (0)
 #endif
 
 struct DiagOut {

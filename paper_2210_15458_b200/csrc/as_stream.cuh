@@ -78,6 +78,12 @@ struct StreamSmemT {
     LaneResult res;
 };
 
+// Programmatic dependent launch.  allow_next: the next kernel on the stream may begin its own
+// set-up while this grid still runs.  wait_prev: returns once the kernel before this one has
+// completed and its writes are visible (at once if this launch does not overlap anything).
+__device__ __forceinline__ void pdl_allow_next() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_prev() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -520,6 +526,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     ASX_MARK(13);
+    ASX_SPAN(0);
     const int V = a.V;
     const int row_bytes = (V + (UA ? E - 1 : 0)) * Tr::BYTES;          // UA: the longest a row gets with its lead
     const int bulk_bytes = row_bytes & ~15;
@@ -585,6 +592,10 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         }
         return true;
     };
+    // Set-up that touches no global memory comes first: it may run while the kernel before this
+    // one on the stream is still draining.  Everything after pdl_wait_prev() sees that kernel's
+    // writes (logits, codes, the previous step's tokens in a decode loop).
+    pdl_allow_next();
     if (is_producer) {
         for (int i = 0; i < S; ++i) {
             mbar_init(smem_u32(&sm.full_bar[i]), 1);
@@ -592,9 +603,10 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         }
         fence_mbar_init();
         sm.poisoned = 0;
-        issue_some(true);                         // fills the ring without waiting
     }
     fill_exp_table(sm.exp_tbl, tid);
+    pdl_wait_prev();
+    if (is_producer) issue_some(true);            // fills the ring without waiting
     __syncthreads();
 
     // =========================== producer warp ===========================
@@ -692,6 +704,27 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
     auto push_vec = [&](const uint4& q, int base, float t0f, uint32_t t0key, bool with_tail, float ref, float& tail) {
         float x[E];
         P::floats(q, x);
+        if (!with_tail) {
+            // lean form: one float compare per element; the exact key test and the reservation run
+            // only for the one or two elements that pass (~55 instructions per vector against ~170)
+            unsigned m = 0;
+#pragma unroll
+            for (int e = 0; e < E; ++e) m |= (x[e] >= t0f ? 1u : 0u) << e;
+#pragma unroll 1
+            while (m) {
+                const int e = __ffs(m) - 1;
+                m &= m - 1;
+                float xe = x[0];
+#pragma unroll
+                for (int k = 1; k < E; ++k) xe = (e == k) ? x[k] : xe;
+                const uint32_t key = P::key_of_f(xe);
+                if (key >= t0key && key > Tr::KEY_NINF) {
+                    const int slot = atomicAdd(&sm.cand_count, 1);
+                    if (slot < SK_CAP) sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)(base + e);
+                }
+            }
+            return;
+        }
         unsigned em = 0;
 #pragma unroll
         for (int e = 0; e < E; ++e) {
@@ -1019,6 +1052,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         ASX_MARK(12);
     }
     ASX_MARK(14);
+    ASX_SPAN(2);
 }
 
 }  // namespace asx
