@@ -394,6 +394,9 @@ int as_debug_span(unsigned long long* h_out, int reset) {
     if (reset) return cudaMemcpyToSymbol(g_asx_span, init, sizeof(init)) == cudaSuccess ? AS_OK : AS_ERR_CUDA;
     return cudaMemcpyFromSymbol(h_out, g_asx_span, sizeof(init)) == cudaSuccess ? AS_OK : AS_ERR_CUDA;
 }
+int as_debug_cta(unsigned long long* h_out) {
+    return cudaMemcpyFromSymbol(h_out, g_asx_cta, sizeof(unsigned long long) * 1024 * 8) == cudaSuccess ? AS_OK : AS_ERR_CUDA;
+}
 int as_debug_counts(unsigned long long* h_out) {
     return cudaMemcpyFromSymbol(h_out, g_asx_counts, sizeof(unsigned long long) * 16) == cudaSuccess ? AS_OK : AS_ERR_CUDA;
 }

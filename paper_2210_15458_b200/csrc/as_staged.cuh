@@ -54,12 +54,22 @@ __device__ __forceinline__ void asx_span(int i) {
     }
 }
 #define ASX_SPAN(i) asx_span(i)
+__device__ unsigned long long g_asx_cta[1024][8];  // per-CTA phase times of its first lane (globaltimer, ns)
+__device__ __forceinline__ void asx_cta(int i) {
+    if (threadIdx.x == 0 && blockIdx.x < 1024) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        g_asx_cta[blockIdx.x][i] = t;
+    }
+}
+#define ASX_CTA(i) asx_cta(i)
 #define ASX_MARK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_asx_marks[i] = clock64(); } while (0)
 #define ASX_COUNT(i) do { if (threadIdx.x == 0) atomicAdd(&g_asx_counts[i], 1ull); } while (0)
 #else
 #define ASX_MARK(i) do {} while (0)
 #define ASX_COUNT(i) do {} while (0)
 #define ASX_SPAN(i) do {} while (0)
+#define ASX_CTA(i) do {} while (0)
 #endif
 
 struct DiagOut {

@@ -527,6 +527,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     ASX_MARK(13);
     ASX_SPAN(0);
+    ASX_CTA(0);
     const int V = a.V;
     const int row_bytes = (V + (UA ? E - 1 : 0)) * Tr::BYTES;          // UA: the longest a row gets with its lead
     const int bulk_bytes = row_bytes & ~15;
@@ -562,7 +563,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
     // The producer lane initialises the barriers of the stages in use and starts the first copies
     // before the block-wide barrier, so the first row is in flight while the rest of the CTA sets up.
     const bool is_producer = (warp == SK_NW && lane == 0);
-    unsigned g_issued = 0;                        // producer: slices issued so far
+    unsigned p_st = 0, p_round = 0;               // producer: slices issued so far = p_round * S + p_st
     int ln_issue = blockIdx.x;                    // producer: lane whose slices come next
     int s_issue = 0;
     auto issue_some = [&](bool first_row_only) -> bool {   // false: a bounded wait ran out
@@ -573,12 +574,12 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             const int lead_i = lead_of(ln_issue);
             if (UA) { int bv, te; geom(lead_i, bulk_bytes_i, bv, te, nsl_i); }
             const char* src = row_of(ln_issue) - lead_i * Tr::BYTES;
-            for (; s_issue < nsl_i; ++s_issue, ++g_issued) {
-                const int st = g_issued % S;
-                if (g_issued >= (unsigned)S) {    // the stage must have been drained by every consumer warp
+            for (; s_issue < nsl_i; ++s_issue, p_st = (p_st + 1 == (unsigned)S ? (++p_round, 0u) : p_st + 1)) {
+                const int st = (int)p_st;
+                if (p_round >= 1) {               // the stage must have been drained by every consumer warp
                     if (first_row_only) return true;
                     if (*(volatile int*)&sm.poisoned) return false;
-                    if (!mbar_wait_bounded(smem_u32(&sm.empty_bar[st]), ((g_issued / S) - 1) & 1)) {
+                    if (!mbar_wait_bounded(smem_u32(&sm.empty_bar[st]), (p_round - 1) & 1)) {
                         *(volatile int*)&sm.poisoned = 1;
                         return false;
                     }
@@ -620,7 +621,12 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
     const int m_sel = (K0 + SK_NW - 1) / SK_NW;
     const float scale2 = a.scale2;
     const uint32_t ninf_word = (DT == DT_BF16) ? 0xFF80FF80u : 0xFF800000u;
-    unsigned g = 0;
+    // consumer's position in the ring: the slice counter g is kept as stage (g mod S) and phase
+    // parity ((g / S) & 1) and advanced by additions; a division by S per use cost more
+    // instructions than the work between two uses
+    unsigned g_st = 0, g_par = 0;
+    auto stage_of = [&](int off) -> unsigned { const unsigned st = g_st + off; return st >= (unsigned)S ? st - S : st; };
+    auto advance = [&](int n) { g_st += n; if (g_st >= (unsigned)S) { g_st -= S; g_par ^= 1u; } };   // n <= S
     int thr_calls = 0;
 
     // block step: max so far and (optionally) threshold from the subset maxima held in `acc`;
@@ -808,13 +814,14 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         float t0f = 0.f;
         const bool cut = a.fast && (a.top_k > 0 || a.top_p < 1.0);
 
-        auto wait_full = [&](unsigned gg) {
+        auto wait_full = [&](int off) {            // slice g + off, off < S
             if (*(volatile int*)&sm.poisoned) return;
-            if (!mbar_wait_bounded(smem_u32(&sm.full_bar[gg % S]), (gg / S) & 1)) *(volatile int*)&sm.poisoned = 1;
+            const unsigned par = g_par ^ (g_st + off >= (unsigned)S ? 1u : 0u);
+            if (!mbar_wait_bounded(smem_u32(&sm.full_bar[stage_of(off)]), par)) *(volatile int*)&sm.poisoned = 1;
         };
-        auto release = [&](unsigned gg) {
+        auto release = [&](int off) {
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sm.empty_bar[gg % S]));
+            if (lane == 0) mbar_arrive(smem_u32(&sm.empty_bar[stage_of(off)]));
         };
         auto load_slice = [&](const uint4* sv, int nv, uint4 (&q)[SK_VPT]) -> unsigned {
             unsigned valid = 0;
@@ -829,6 +836,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         };
 
         ASX_MARK(0);
+        ASX_CTA(1);
         if (general_row) {
             // nothing was staged for this lane
         } else if (resident) {
@@ -838,38 +846,44 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
 #pragma unroll
             for (int s = 0; s < SK_RES_STAGES; ++s) {
                 if (s < nsl_l) {
-                    wait_full(g + s);
+                    wait_full(s);
                     ASX_MARK(1);
                     uint4 q[SK_VPT];
-                    load_slice(ringv + (size_t)((g + s) % S) * SK_STAGE_VEC, min(SK_STAGE_VEC, bulk_vec_l - s * SK_STAGE_VEC), q);
+                    const unsigned valid = load_slice(ringv + (size_t)stage_of(s) * SK_STAGE_VEC,
+                                                      min(SK_STAGE_VEC, bulk_vec_l - s * SK_STAGE_VEC), q);
                     if (UA && s == 0 && tid == 0 && lead) {
                         // the elements in front of the row: masked here and in the ring (this thread
                         // alone reads that vector again; the next bulk copy into the stage is
                         // ordered after the store by the proxy fence)
                         mask_lead<DT>(q[0], lead);
-                        reinterpret_cast<uint4*>(ring)[(size_t)(g % S) * SK_STAGE_VEC] = q[0];
+                        reinterpret_cast<uint4*>(ring)[(size_t)g_st * SK_STAGE_VEC] = q[0];
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     }
 #pragma unroll
                     for (int j = 0; j < SK_VPT; ++j) {
                         const typename P::Acc part = P::reduce(q[j]);
                         P::merge(acc, part);
-                        pm[s * SK_VPT + j] = P::part_max(part);      // -inf for vectors past the row
+                        // NaN for vectors past the row: they must not pass any threshold, not even
+                        // -inf (a row with fewer than K0 elements), or the hit loop below would read
+                        // stages that do not exist
+                        pm[s * SK_VPT + j] = ((valid >> j) & 1u) ? P::part_max(part) : __uint_as_float(0x7FC00000u);
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < SK_VPT; ++j) pm[s * SK_VPT + j] = __uint_as_float(0xFF800000u);
+                    for (int j = 0; j < SK_VPT; ++j) pm[s * SK_VPT + j] = __uint_as_float(0x7FC00000u);
                 }
             }
             if (tid == 0) P::merge(acc, P::reduce(qt));
             ASX_MARK(2);
+            ASX_CTA(2);
             threshold(acc, gmax, t0key, cut, 0u);
             ASX_MARK(3);
+            ASX_CTA(3);
             const bool bad = gmax >= Tr::KEY_PINF || gmax <= Tr::KEY_NINF;
             if (bad) {
                 r = failed_lane(c_in, ST_NUMERIC);
                 decided = true;
-                for (int s = 0; s < nsl_l; ++s) release(g + s);
+                for (int s = 0; s < nsl_l; ++s) release(s);
             } else if (!cut) {
                 // no cut: every token is kept; the general routine scans the row in shared memory
                 if (UA && lead) {
@@ -898,7 +912,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                         const int i = __ffs(hm) - 1;
                         hm &= hm - 1;
                         const int s = i / SK_VPT, v = (i % SK_VPT) * NT + tid;
-                        const uint4 q = ringv[(size_t)((g + s) % S) * SK_STAGE_VEC + v];
+                        const uint4 q = ringv[(size_t)stage_of(s) * SK_STAGE_VEC + v];
                         float unused = 0.f;
                         push_vec(q, (s * SK_STAGE_VEC + v) * E - lead, t0f, t0key, false, ref, unused);
                     }
@@ -906,12 +920,12 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
 #pragma unroll 1
                     for (int s = 0; s < nsl_l; ++s) {
                         uint4 q[SK_VPT];
-                        const unsigned valid = load_slice(ringv + (size_t)((g + s) % S) * SK_STAGE_VEC,
+                        const unsigned valid = load_slice(ringv + (size_t)stage_of(s) * SK_STAGE_VEC,
                                                           min(SK_STAGE_VEC, bulk_vec_l - s * SK_STAGE_VEC), q);
                         slice_pass(q, s * SK_STAGE_VEC + tid, valid, false, acc, t0f, ref, tail);
                     }
                 }
-                for (int s = 0; s < nsl_l; ++s) release(g + s);     // the producer may refill: next row
+                for (int s = 0; s < nsl_l; ++s) release(s);     // the producer may refill: next row
             }
         } else {
             // ---- streamed: slice -> registers -> stage released; T0 at slices 0, 1, 2, 4, 8, ...
@@ -924,13 +938,13 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
 #define ASX_ACC(var) do {} while (0)
 #endif
 #pragma unroll 1
-            for (int s = 0; s < nsl_l; ++s, ++g) {
-                wait_full(g);
+            for (int s = 0; s < nsl_l; ++s, advance(1)) {
+                wait_full(0);
                 ASX_ACC(pw);
                 uint4 q[SK_VPT];
-                const unsigned valid = load_slice(ringv + (size_t)(g % S) * SK_STAGE_VEC,
+                const unsigned valid = load_slice(ringv + (size_t)g_st * SK_STAGE_VEC,
                                                   min(SK_STAGE_VEC, bulk_vec_l - s * SK_STAGE_VEC), q);
-                release(g);
+                release(0);
                 if (UA && s == 0 && tid == 0 && lead) mask_lead<DT>(q[0], lead);
                 ASX_ACC(pl);
                 if (s == 0) {
@@ -1006,6 +1020,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         // the tail was summed against `ref` (<= lmax); bring it to the true maximum
         if (want_tail) tailsum *= exp_nonpos(((double)ref - lmax) * a.inv_tau, sm.exp_tbl);
         ASX_MARK(5);
+        ASX_CTA(5);
 #ifdef ASX_PROFILE
         if (blockIdx.x == 0 && tid == 0) { g_asx_marks[20] = nvh; g_asx_marks[21] = C; }
 #endif
@@ -1036,9 +1051,9 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             r = gl.run(c_in, a.inv_tau, a.top_k, a.top_p);
             path = PATH_GENERAL;
             if (general_release)
-                for (int s = 0; s < nsl_l; ++s) release(g + s);
+                for (int s = 0; s < nsl_l; ++s) release(s);
         }
-        if (resident && staged_ok(ln)) g += nsl_l;
+        if (resident && staged_ok(ln)) advance(nsl_l);
         if (tid == 0) {
             if (GATHER) {
                 a.tokens[(size_t)ln * a.tok_stride] = r.token;
@@ -1050,9 +1065,11 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         }
         SyncC::sync();
         ASX_MARK(12);
+        ASX_CTA(6);
     }
     ASX_MARK(14);
     ASX_SPAN(2);
+    ASX_CTA(7);
 }
 
 }  // namespace asx

@@ -555,6 +555,35 @@ def test_step_rows_off_the_16_byte_grid_take_the_fast_path(B, orc, dtype, V, pad
     check(B, orc, arr[:4], dtype, codes[:4], 1.0, 0, 1.0, what="off-grid rows, no cut")
 
 
+@pytest.mark.parametrize("dtype", [F32, BF16])
+@pytest.mark.parametrize("V", [2, 5, 24, 200, 4096 + 40])
+def test_step_rows_with_fewer_tokens_than_the_cut_asks_for(B, orc, dtype, V):
+    # fewer finite tokens than top_k (or than the list aims at): the threshold falls to -inf.  Only
+    # vectors that exist may then count as hits: the ring holds one stage for such a row, and the
+    # space behind a short row is whatever the previous launch left there.  The list must decide
+    # these lanes itself (no detour through the general routine), masked tokens staying out.
+    rng = np.random.default_rng(300 + V)
+    lanes = 21
+    x = rng.normal(0, 3, (lanes, V)).astype(np.float32)
+    if V > 8:
+        x[:, rng.choice(V, V // 3, replace=False)] = -np.inf
+    arr = _store(x, dtype)
+    codes = rng.random(lanes)
+    codes[0], codes[1] = 0.0, 1.0
+    dev = to_dev(arr, dtype)                               # aligned rows when V * size is a multiple of 16
+    for temp, k, p in [(1.0, 1, 1.0), (0.8, V - 1 if V > 2 else 1, 1.0), (0.7, min(V - 1, 250), 0.9), (1.2, 0, 0.6)]:
+        if k > 256:
+            continue
+        d = {}
+        ref = orc.step(arr, dtype, codes, temp, k, p, threads=8)
+        tok, c2 = B.as_step(dev, torch.from_numpy(codes).cuda(), temp, k, p, diag=d)
+        torch.cuda.synchronize()
+        compare_step(ref, tok.cpu().numpy(), c2.cpu().numpy(), d["p_tok"].cpu().numpy(), d["n_kept"].cpu().numpy(),
+                     d["lane_status"].cpu().numpy(), what="short rows V=%d %s" % (V, (temp, k, p)))
+        if k > 0:
+            assert (d["path"].cpu().numpy() == B.PATH_COMPACT).all()
+
+
 def test_decode_with_cuts_per_step_kernels_equal_the_single_kernel(B, orc):
     # with a cut and a codes_final buffer the loop runs as one launch of the step kernel per step
     # (rows gathered from the table); without the buffer, as one general kernel.  Both follow the
