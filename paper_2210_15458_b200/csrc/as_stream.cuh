@@ -75,7 +75,6 @@ struct StreamSmemT {
     int cand_count;
     int poisoned;        // a bounded wait ran out: stop issuing / stop waiting
     int b_i[4];
-    LaneResult res;
 };
 
 // Programmatic dependent launch.  allow_next: the next kernel on the stream may begin its own
@@ -131,7 +130,8 @@ __device__ __forceinline__ uint32_t warp_select16(uint32_t a16, uint32_t b16, in
 
 // Exact decode on a candidate list src[0..C) (composites, any order); dst is scratch of C + 4
 // entries.  depth_key: every element of the row with key >= depth_key is in the list, so ranks
-// are exact down to that key.  Returns false if the list cannot decide the lane.
+// are exact down to that key.  Returns false if the list cannot decide the lane (uniformly in all
+// threads); `out` is set in thread 0 only.
 template <int DT, int NT, class Sync, class StreamSmem>
 __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long* src, unsigned long long* dst,
                                              double* e, int C, uint32_t depth_key, double c, double lmax,
@@ -291,14 +291,14 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
                 LaneResult r;
                 r.token = (int)(src[pick] >> 32); r.status = ST_OK; r.n_kept = n_final; r.code_out = cn;
                 r.p_tok = p_tok; r.cdf_lo = cdf_lo;
-                sm.res = r;
+                out = r;
             }
         }
     }
     ASX_MARK(9);
-    Sync::sync();
     ASX_MARK(10);
-    out = sm.res;
+    // No barrier here: the result lives in thread 0, which is also the one that writes it out, and
+    // every caller passes a block barrier before shared memory is written again.
     return ok != 0;
 }
 
