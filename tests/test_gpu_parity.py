@@ -584,6 +584,30 @@ def test_step_rows_with_fewer_tokens_than_the_cut_asks_for(B, orc, dtype, V):
             assert (d["path"].cpu().numpy() == B.PATH_COMPACT).all()
 
 
+def test_step_overlapped_launches_give_the_same_results(B):
+    # launches of one row per CTA may start while the launch before them drains (programmatic
+    # dependent launch): a chain of steps, each reading the codes the one before wrote, must give
+    # bit for bit what the same chain gives as ordinary launches
+    from paper_2210_15458_b200 import synth
+    w = synth.StepWorkload("chain", lanes=200, V=32000, dtype=synth.BF16, sigma=3.0, temp=0.7, top_k=40,
+                           top_p=1.0, seed_logits=71, seed_perm=72, seed_shift=73)
+    logits = to_dev(w.logits(), BF16)
+    results = []
+    for serial in (1, 0):
+        B.as_tune(B.TUNE_SERIAL_LAUNCH, serial)
+        try:
+            codes = B.as_lattice_codes(w.N, w.shift())
+            toks = torch.empty((12, w.lanes), dtype=torch.int32, device="cuda")
+            for t in range(12):                      # back to back, no host synchronisation between
+                B.as_step(logits, codes, w.temp, w.top_k, w.top_p, tokens=toks[t], codes_out=codes)
+            torch.cuda.synchronize()
+            results.append((toks.cpu().numpy(), codes.cpu().numpy()))
+        finally:
+            B.as_tune(B.TUNE_SERIAL_LAUNCH, 0)
+    assert np.array_equal(results[0][0], results[1][0])
+    assert np.array_equal(results[0][1], results[1][1])
+
+
 def test_decode_with_cuts_per_step_kernels_equal_the_single_kernel(B, orc):
     # with a cut and a codes_final buffer the loop runs as one launch of the step kernel per step
     # (rows gathered from the table); without the buffer, as one general kernel.  Both follow the

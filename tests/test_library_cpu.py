@@ -89,6 +89,7 @@ def test_invalid_arguments_are_rejected_on_the_host(L):
     assert rm(V=0) == B.ERR_INVALID_ARG and rm(r=None) == B.ERR_INVALID_ARG and rm(mean=None) == B.ERR_INVALID_ARG
     assert rm(S=0) == B.OK
     assert L.as_tune(99, 0) == B.ERR_INVALID_ARG and L.as_tune(B.TUNE_CLUSTER, 3) == B.ERR_INVALID_ARG
+    assert L.as_tune(B.TUNE_SERIAL_LAUNCH, 2) == B.ERR_INVALID_ARG and L.as_tune(B.TUNE_SERIAL_LAUNCH, 0) == B.OK
     assert L.as_step_host_work_bytes(0, 4, 10) >= 4 * 10 * 4 + 4 * 24
 
 
