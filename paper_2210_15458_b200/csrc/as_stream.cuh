@@ -43,7 +43,7 @@ constexpr int SK_MAXSTAGES = 12;
 constexpr int SK_RES_STAGES = 6;           // rows of up to this many stages (96 KB) stay resident
 constexpr int SK_K0_RESIDENT = 256;        // largest top_k served by the list, resident rows
 constexpr int SK_K0_STREAMED = 96;         // ... streamed rows (hits grow like K0 ln(V / K0))
-constexpr int SK_KP = 96;                  // K0 for nucleus-only lanes
+constexpr int SK_KP = 64;                  // K0 for nucleus-only lanes
 
 using SyncC = SyncNamed<SK_NT>;
 
