@@ -14,8 +14,8 @@
 //       max and tested against the current T0; T0 is recomputed at slices
 //       0, 1, 2, 4, 8, ... and only ever rises.
 // T0 is a lower bound on the K0-th largest logit: each warp takes the m-th
-// largest (m = ceil(K0 / 8)) of its 64 per-thread subset maxima by a ballot
-// search, and T0 is the smallest of the 8 warp values, so at least K0 elements
+// largest (m = ceil(K0 / 8)) of its 64 per-thread subset maxima (warp_select16),
+// and T0 is the smallest of the 8 warp values, so at least K0 elements
 // are >= T0.  The hot loop costs one packed max and one compare per 16-byte
 // vector; a vector holding an element >= T0 is copied (warp-aggregated, one
 // atomic per warp) to a small list.  Once per row the listed vectors are
@@ -43,7 +43,7 @@ constexpr int SK_MAXSTAGES = 12;
 constexpr int SK_RES_STAGES = 6;           // rows of up to this many stages (96 KB) stay resident
 constexpr int SK_K0_RESIDENT = 256;        // largest top_k served by the list, resident rows
 constexpr int SK_K0_STREAMED = 96;         // ... streamed rows (hits grow like K0 ln(V / K0))
-constexpr int SK_KP = 64;                  // K0 for nucleus-only lanes
+constexpr int SK_KP = 48;                  // K0 for nucleus-only lanes
 
 using SyncC = SyncNamed<SK_NT>;
 
