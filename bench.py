@@ -1,24 +1,29 @@
 #!/usr/bin/env python
 """Benchmark of the arithmetic-sampling decode step on B200.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c5|c4] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5|c2|c3|c4] [--lanes L]
+                  [--impl reference] [--no-extras]
 
-A step is one pass of the decode hot path over one batch of synthetic input: a fresh
-shifted lattice of codes and one decode step for every lane, in one launch (as_step_lattice
-forms the codes in the step kernel; the two-call form is timed beside it).
-The default workload is the 256-lane x 32000-token bf16 step (temperature 0.7, top_k 40).
-Rank 0 prints ONE JSON line.  With N > 1 (torchrun) every
-rank decodes its own batch (lanes never communicate), so scaling is weak and there is no
-data-path collective: only the timing is reduced (max over ranks).
+A step is one pass of the decode hot path over one batch of synthetic input: a fresh shifted
+lattice of codes and one decode step for every lane, in one launch (as_step_lattice forms the
+codes in the step kernel).  The default workload is the largest single-GPU step configuration:
+8192 lanes x 256000 bf16 logits, temperature 0.8, top_k 64 and top_p 0.95 together.  Rank 0
+prints ONE JSON line; `rooflines` in it holds one block per configuration (bytes per launch,
+median and minimum time per launch over >= 20 graph replays, fraction of the measured copy
+bandwidth and of the nominal 8 TB/s).  With N > 1 every rank decodes its own batch (lanes never
+communicate), so scaling is weak and there is no data-path collective: only the timing is
+reduced (max over ranks).  `--gpus N` without a torchrun environment starts the N ranks itself.
 
-`--impl reference` times the CPU oracle (oracle/, test infrastructure) on host cores for
-the same workload; it is a deliberately plain program and serves as a reported baseline.
+`--impl reference` times the CPU oracle (oracle/, test infrastructure) on host cores for the
+same workload; it is a deliberately plain program and serves as a reported baseline.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import re
+import socket
 import subprocess
 import sys
 import threading
@@ -33,10 +38,9 @@ if ROOT not in sys.path:
 from paper_2210_15458_b200 import synth  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the step kernel on the default
-# workload, from the ncu capture summarised in profiles/as_step_stream_c2.md
-NCU_TRAFFIC_BYTES = {"c2": 16472576}
-RING_BYTES = 3 * L2_BYTES          # rotating input buffers: each launch reads from HBM
+RING_BYTES = 3 * L2_BYTES          # small inputs rotate through this much memory
+REPLAYS = 20                       # graph replays behind every median / minimum
+NOMINAL_GBS = 8000.0
 
 
 # ----------------------------------------------------------------------------- helpers
@@ -46,6 +50,18 @@ def measured_peaks():
         with open(path) as f:
             return float(json.load(f)["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def captured_traffic(kernel_file: str, key: str):
+    """DRAM bytes per lane of a kernel from its ncu summary under profiles/ (a line
+    `traffic_bytes_per_lane[<key>]: <number>` written with the capture), or None."""
+    path = os.path.join(ROOT, "profiles", kernel_file)
+    try:
+        with open(path) as f:
+            m = re.search(r"traffic_bytes_per_lane\[%s\]:\s*([0-9.eE+]+)" % re.escape(key), f.read())
+        return float(m.group(1)) if m else None
+    except OSError:
+        return None
 
 
 class ClockSampler:
@@ -119,11 +135,52 @@ def barrier(world: int):
         dist.barrier()
 
 
+def check_world(gpus: int, world: int) -> None:
+    """--gpus must agree with the ranks that were actually started."""
+    if gpus != world:
+        raise SystemExit("bench.py: --gpus %d but WORLD_SIZE is %d: start it as `python bench.py --gpus %d` "
+                         "(it spawns the ranks) or under torchrun with --nproc-per-node %d" % (gpus, world, gpus, gpus))
+
+
+def spawn_ranks(gpus: int) -> int:
+    """`python bench.py --gpus N` outside torchrun: start the N ranks (one per GPU) on this node."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def to_dev(arr, dtype):
     import torch
     if dtype == synth.BF16:
         return torch.from_numpy(np.ascontiguousarray(arr).view(np.int16)).cuda().view(torch.bfloat16)
     return torch.from_numpy(np.ascontiguousarray(arr)).cuda()
+
+
+def device_rows(rows: int, V: int, sigma: float, dtype: int, seed: int, bias):
+    """rows x V logits ~ N(0, sigma^2) + bias, drawn on the device (torch's seeded generator) in the
+    workload's distribution and rounded to its storage type: the host recipe of synth.py yields the
+    same distribution but takes minutes for gigabytes of rows."""
+    import torch
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    tdt = torch.bfloat16 if dtype == synth.BF16 else torch.float32
+    out = torch.empty((rows, V), dtype=tdt, device="cuda")
+    b = torch.from_numpy(bias).cuda() if bias is not None else None
+    step = max(1, (64 << 20) // V)
+    for r0 in range(0, rows, step):
+        r1 = min(rows, r0 + step)
+        x = torch.randn((r1 - r0, V), generator=g, device="cuda", dtype=torch.float32) * sigma
+        if b is not None:
+            x += b[None, :]
+        out[r0:r1] = x.to(tdt)
+    return out
+
+
+def median_min(xs):
+    return float(np.median(xs)), float(np.min(xs))
 
 
 # ----------------------------------------------------------------------------- step workloads
@@ -133,68 +190,84 @@ def step_workload(name: str, lanes=None):
     if name == "c3":
         return synth.c3() if lanes is None else synth.c3(lanes)
     if name == "c5":
-        return synth.c5(1024 if lanes is None else lanes)
+        return synth.c5(8192 if lanes is None else lanes)
     raise ValueError(name)
 
 
-def step_bytes(w) -> int:
-    """Algorithmic bytes of one step: each row read once, code in, code out, token out."""
-    return w.lanes * (w.V * w.elem_bytes + 8 + 8 + 4)
+def step_key(w) -> str:
+    return "c5_%d" % w.lanes if w.name == "c5" else w.name
+
+
+def step_bytes(w, stored_codes: bool = True) -> int:
+    """Algorithmic bytes of one step: each row read once, code in (unless formed in the kernel),
+    code out, token out."""
+    return w.lanes * (w.V * w.elem_bytes + (8 if stored_codes else 0) + 8 + 4)
+
+
+def workload_text(w, lanes=None) -> str:
+    return "%s: %d lanes x V=%d %s logits, temp %g, top_k %d, top_p %g, fp64 lattice codes" % (
+        w.name, w.lanes if lanes is None else lanes, w.V, "bf16" if w.dtype else "f32", w.temp, w.top_k, w.top_p)
 
 
 class StepBench:
-    """Device-resident inputs for a step workload: a ring of distinct logits buffers larger
-    than 3x L2, so that consecutive launches never find their rows in cache."""
+    """Device-resident inputs of a step workload.  Inputs smaller than 4x L2 rotate through a ring
+    of distinct buffers larger than 3x L2, so that no launch finds its rows in cache; larger ones
+    are their own flush."""
 
-    def __init__(self, w, rank: int, base_lanes=None):
+    def __init__(self, w, rank: int):
         import torch
         from paper_2210_15458_b200 import binding as B
         self.B, self.w, self.torch = B, w, torch
-        # host generation is the slow part: for many-lane workloads the first base_lanes rows are
-        # generated and repeated with a per-copy rotation of the lanes
-        gen = w.lanes if base_lanes is None else min(w.lanes, base_lanes)
-        base = w.logits(gen, seed_offset=rank)
-        first = to_dev(base, w.dtype)
-        if gen < w.lanes:
-            first = torch.cat([torch.roll(first, shifts=i, dims=0) for i in range(w.lanes // gen)], dim=0)
-        total = first.numel() * first.element_size()
+        bias = synth.zipf_bias(w.V, w.seed_perm)
+        total = w.lanes * w.V * w.elem_bytes
         nbuf = 1 if total > 4 * L2_BYTES else max(2, -(-RING_BYTES // total))
-        self.ring = [first] + [torch.roll(first, shifts=i, dims=0) for i in range(1, nbuf)]
-        self.host_base = base
+        self.ring = [device_rows(w.lanes, w.V, w.sigma, w.dtype, w.seed_logits + 1000 * rank + 7 * i, bias)
+                     for i in range(nbuf)]
         self.ring_bytes = nbuf * total
         self.shifts = np.random.default_rng(1234 + rank).random(4096)
-        self.codes = B.as_lattice_codes(w.N, float(self.shifts[0]))      # for the calls that read stored codes
+        self.codes = B.as_lattice_codes(w.N, float(self.shifts[0]))[: w.lanes].contiguous()
+        self.iid = torch.from_numpy(synth.iid_codes(w.lanes, 4321 + rank)).cuda()
         self.tokens = torch.empty(w.lanes, dtype=torch.int32, device="cuda")
         self.codes_out = torch.empty(w.lanes, dtype=torch.float64, device="cuda")
         self.i = 0
+
+    def l2_note(self) -> str:
+        if len(self.ring) == 1:
+            return "one input of %.0f MB (> L2) read end to end by every launch" % (self.ring_bytes / 1e6)
+        return "inputs rotate through %d buffers (%.0f MB > 3x L2)" % (len(self.ring), self.ring_bytes / 1e6)
+
+    def _next(self):
+        buf = self.ring[self.i % len(self.ring)]
+        self.i += 1
+        return buf
 
     def step(self):
         """One pass of the hot path: the lattice codes of a fresh shift, formed in the step kernel
         (as_step_lattice: the same values as_lattice_codes would write), and the decode step."""
         B, w = self.B, self.w
-        B.as_step_lattice(self.ring[self.i % len(self.ring)], w.N, float(self.shifts[self.i % 4096]), 0,
-                          w.temp, w.top_k, w.top_p, tokens=self.tokens, codes_out=self.codes_out)
-        self.i += 1
+        B.as_step_lattice(self._next(), w.N, float(self.shifts[self.i % 4096]), 0, w.temp, w.top_k, w.top_p,
+                          tokens=self.tokens, codes_out=self.codes_out)
 
     def step_two_calls(self):
         """The same pass as two launches: as_lattice_codes, then as_step on the stored codes."""
         B, w = self.B, self.w
         B.as_lattice_codes(w.N, float(self.shifts[self.i % 4096]), out=self.codes)
-        B.as_step(self.ring[self.i % len(self.ring)], self.codes[: w.lanes], w.temp, w.top_k, w.top_p,
-                  tokens=self.tokens, codes_out=self.codes_out)
-        self.i += 1
+        B.as_step(self._next(), self.codes, w.temp, w.top_k, w.top_p, tokens=self.tokens, codes_out=self.codes_out)
 
-    def step_kernel_only(self):
-        """as_step on stored codes (every step after the first in a decode loop)."""
+    def step_stored(self):
+        """as_step on stored lattice codes (every step after the first in a decode loop)."""
         B, w = self.B, self.w
-        B.as_step(self.ring[self.i % len(self.ring)], self.codes[: w.lanes], w.temp, w.top_k, w.top_p,
-                  tokens=self.tokens, codes_out=self.codes_out)
-        self.i += 1
+        B.as_step(self._next(), self.codes, w.temp, w.top_k, w.top_p, tokens=self.tokens, codes_out=self.codes_out)
 
-    def timed(self, fn, n: int) -> float:
-        """Device time of n calls of fn.  The calls are captured once into a CUDA graph (the step
-        is launch-bound from Python: a ctypes call costs more than the kernel) and the graph
-        is replayed; the inputs still rotate through the ring inside the graph."""
+    def step_iid(self):
+        """The same kernel on iid uniform codes: ordinary ancestral sampling by inverse CDF."""
+        B, w = self.B, self.w
+        B.as_step(self._next(), self.iid, w.temp, w.top_k, w.top_p, tokens=self.tokens, codes_out=self.codes_out)
+
+    def graph(self, fn, n: int):
+        """n calls of fn captured into one CUDA graph (a ctypes call from Python costs more than
+        a small kernel, so a Python launch loop would time the interpreter); the inputs still
+        rotate through the ring inside the graph."""
         torch = self.torch
         g = torch.cuda.CUDAGraph()
         side = torch.cuda.Stream()
@@ -204,9 +277,10 @@ class StepBench:
                 for _ in range(n):
                     fn()
         torch.cuda.current_stream().wait_stream(side)
-        self.last_graph = g
-        for _ in range(3):              # untimed: the first replay uploads the graph
-            g.replay()
+        return g
+
+    def replay_ms(self, g) -> float:
+        torch = self.torch
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         a.record()
@@ -215,18 +289,56 @@ class StepBench:
         torch.cuda.synchronize()
         return a.elapsed_time(b)
 
+    def per_launch_us(self, fn, replays: int = REPLAYS):
+        """Median and minimum time of one launch of fn over `replays` replays of a graph that holds
+        enough launches to last about 2 ms (at least 2, and a whole turn of the input ring)."""
+        for _ in range(3):
+            fn()
+        self.torch.cuda.synchronize()
+        probe = self.graph(fn, 2)
+        self.replay_ms(probe)
+        one = max(self.replay_ms(probe) / 2, 1e-3)
+        n = int(min(400, max(2, len(self.ring), round(2.0 / one))))
+        g = self.graph(fn, n)
+        self.replay_ms(g)
+        xs = [self.replay_ms(g) / n * 1e3 for _ in range(replays)]
+        return median_min(xs) + (n,)
+
+
+def roofline_block(w, med_us, min_us, launches, peak, bytes_per_launch, traffic_per_lane=None, kernel=None):
+    gbs = bytes_per_launch / (med_us * 1e-6) / 1e9
+    blk = {"bound": "hbm", "workload": workload_text(w), "bytes_per_launch": bytes_per_launch,
+           "us_per_launch_median": med_us, "us_per_launch_min": min_us,
+           "replays": REPLAYS, "launches_per_replay": launches,
+           "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+           "frac_of_8TBs_nominal": gbs / NOMINAL_GBS, "frac_at_min": bytes_per_launch / (min_us * 1e-6) / 1e9 / peak,
+           "logits_per_s": w.lanes * w.V / (med_us * 1e-6), "lane_steps_per_s": w.lanes / (med_us * 1e-6),
+           "traffic": None if traffic_per_lane is None else traffic_per_lane * w.lanes}
+    if kernel:
+        blk["kernel"] = kernel
+    return blk
+
+
+def stream_kernel_name(w) -> str:
+    resident = w.V * w.elem_bytes <= 6 * 16384
+    return "step_stream_kernel (%s rows)" % ("ring-resident" if resident else "streamed")
+
 
 def e2e_step(w, steps: int, warmup: int):
     """Same metric through the host-buffer entry point: every step copies the logits and codes
     from pinned host memory, runs the step and copies tokens and codes back."""
     import torch
     from paper_2210_15458_b200 import binding as B
-    base = w.logits()
-    view = base.view(np.int16) if w.dtype == synth.BF16 else base
-    nslots = 4
-    h_logits = [torch.from_numpy(np.roll(view, i, axis=0).copy()).pin_memory() for i in range(nslots)]
-    if w.dtype == synth.BF16:
-        h_logits = [h.view(torch.bfloat16) for h in h_logits]
+    bias = synth.zipf_bias(w.V, w.seed_perm)
+    tdt = torch.bfloat16 if w.dtype == synth.BF16 else torch.float32
+    total = w.lanes * w.V * w.elem_bytes
+    nslots = 1 if total > (1 << 30) else 4
+    h_logits = []
+    for i in range(nslots):
+        h = torch.empty((w.lanes, w.V), dtype=tdt, pin_memory=True)
+        h.copy_(device_rows(w.lanes, w.V, w.sigma, w.dtype, 900 + i, bias))
+        h_logits.append(h)
+    torch.cuda.empty_cache()
     codes = np.random.default_rng(99).random(w.lanes)
     h_codes = torch.from_numpy(codes).pin_memory()
     h_tok = torch.empty(w.lanes, dtype=torch.int32).pin_memory()
@@ -249,16 +361,14 @@ def e2e_step(w, steps: int, warmup: int):
     return ms, h2d, d2h
 
 
-def cpu_baseline_step(w, budget_s: float = 12.0):
-    """The oracle as it stands, on host cores, on a bounded sample of the same workload."""
+def oracle_rate(w, lanes: int, budget_s: float):
+    """logits/s of the oracle as it stands on `lanes` rows of the workload (host recipe), all host cores."""
     from oracle import oracle
     cores = os.cpu_count() or 1
-    lanes = min(w.lanes, 256)
     arr = w.logits(lanes)
     codes = oracle.lattice_codes(w.N, w.shift())[:lanes]
     threads = min(cores, lanes)
-    oracle.step(arr[: min(lanes, threads)], w.dtype, codes[: min(lanes, threads)], w.temp, w.top_k, w.top_p,
-                threads=threads)
+    oracle.step(arr[:threads], w.dtype, codes[:threads], w.temp, w.top_k, w.top_p, threads=threads)
     t0 = time.perf_counter()
     reps = 0
     while True:
@@ -267,104 +377,94 @@ def cpu_baseline_step(w, budget_s: float = 12.0):
         dt = time.perf_counter() - t0
         if dt > budget_s or reps >= 20:
             break
-    return {"value": reps * lanes * w.V / dt, "unit": "logits/s", "cores": threads, "kind": "oracle",
+    return reps * lanes * w.V / dt, threads, reps, dt
+
+
+def cpu_baseline_step(w, budget_s: float = 12.0):
+    """The oracle as it stands, on host cores, on a bounded sample of the same workload."""
+    lanes = min(w.lanes, 64 if w.V > 100000 else 256)
+    rate, threads, reps, dt = oracle_rate(w, lanes, budget_s)
+    return {"value": rate, "unit": "logits/s", "cores": threads, "kind": "oracle",
             "sample": "%d x the first %d lanes of %s (V=%d), %.1f s" % (reps, lanes, w.name, w.V, dt)}
 
 
 # ----------------------------------------------------------------------------- bigram workload (c4)
-def bench_bigram(steps: int, warmup: int, S: int = 64, T: int = 128):
+def bench_bigram(reps: int, warmup: int, S: int = 64, T: int = 128, eos_variant: bool = True):
     """tokens/s of the full decode loop over the 32128 x 32128 bf16 bigram table, lattice
     codes versus iid codes (ordinary ancestral sampling through the same kernel)."""
     import torch
     from paper_2210_15458_b200 import binding as B
     w = synth.c4(S=S, T=T)
-    table = to_dev(w.table(), w.dtype)
+    table = device_rows(w.V, w.V, w.sigma, w.dtype, w.seed_table, w.column_bias())
     starts = torch.from_numpy(w.starts()).cuda()
     out = {}
     seq = torch.empty((w.lanes, w.T), dtype=torch.int32, device="cuda")
     ln = torch.empty(w.lanes, dtype=torch.int32, device="cuda")
     prev = starts.repeat_interleave(w.N).contiguous()
     iid = torch.from_numpy(synth.iid_codes(w.lanes, 77)).cuda()
+    peak, _ = measured_peaks()
 
-    def run_lattice():
-        B.as_decode_bigram(table, starts, w.N, w.shift(), w.T, w.eos, w.temp, w.top_k, w.top_p, seq=seq, length=ln)
-
-    def run_iid():
-        B.as_decode_bigram_codes(table, prev, iid, w.T, w.eos, w.temp, w.top_k, w.top_p, seq=seq, length=ln)
+    def timed(fn):
+        for _ in range(max(1, warmup)):
+            fn()
+        xs = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            xs.append(a.elapsed_time(b))
+        return median_min(xs)
 
     def dup_rates(s):
         s = s.cpu().numpy().reshape(w.S, w.N, w.T)
         res = {}
-        for L in (1, 2, 4, 8, 128):
+        for L in (1, 2, 4, 8, 16, 32, w.T):
             r = [1.0 - len({tuple(x[:L]) for x in grp}) / w.N for grp in s]
             res[str(L)] = float(np.mean(r))
         return res
 
-    for name, fn in (("lattice", run_lattice), ("iid", run_iid)):
-        for _ in range(max(1, warmup)):
-            fn()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        a.record()
-        for _ in range(steps):
-            fn()
-        b.record()
-        torch.cuda.synchronize()
-        ms = a.elapsed_time(b) / steps
+    def decode_entry(fn, tbl_note=None):
+        med, mn = timed(fn)
         tokens = int(ln.sum().item())
-        out[name] = {"ms_per_decode": ms, "tokens": tokens, "tokens_per_s": tokens / ms * 1e3,
-                     "mean_len": tokens / w.lanes,
-                     "row_gbs_upper": tokens * w.V * w.elem_bytes / ms / 1e6,
-                     "duplicate_prefix_rate": dup_rates(seq)}
+        gbs = tokens * w.V * w.elem_bytes / med / 1e6
+        e = {"ms_per_decode_median": med, "ms_per_decode_min": mn, "repetitions": reps, "tokens": tokens,
+             "tokens_per_s": tokens / med * 1e3, "mean_len": tokens / w.lanes,
+             "row_gbs": gbs, "row_frac_of_peak": gbs / peak,
+             "duplicate_prefix_rate": dup_rates(seq)}
+        if tbl_note:
+            e["table"] = tbl_note
+        return e
+
+    def run_lattice(tbl=table):
+        B.as_decode_bigram(tbl, starts, w.N, w.shift(), w.T, w.eos, w.temp, w.top_k, w.top_p, seq=seq, length=ln)
+
+    def run_iid(tbl=table):
+        B.as_decode_bigram_codes(tbl, prev, iid, w.T, w.eos, w.temp, w.top_k, w.top_p, seq=seq, length=ln)
+
+    out["lattice"] = decode_entry(run_lattice)
+    out["iid"] = decode_entry(run_iid)
     # the same loop with a cut (Sec. 5.1 "Top-k sampling": k = 2 and 10; a nucleus): one launch of
     # the streaming step kernel per step, rows gathered from the table
     cf = torch.empty(w.lanes, dtype=torch.float64, device="cuda")
     for name, k, p in (("top_k_2", 2, 1.0), ("top_k_10", 10, 1.0), ("top_p_0.9", 0, 0.9)):
-        fn = lambda: B.as_decode_bigram(table, starts, w.N, w.shift(), w.T, w.eos, w.temp, k, p, seq=seq, length=ln,
-                                        codes_final=cf)
-        for _ in range(max(1, warmup)):
-            fn()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        a.record()
-        for _ in range(steps):
-            fn()
-        b.record()
-        torch.cuda.synchronize()
-        ms = a.elapsed_time(b) / steps
+        med, mn = timed(lambda: B.as_decode_bigram(table, starts, w.N, w.shift(), w.T, w.eos, w.temp, k, p, seq=seq,
+                                                   length=ln, codes_final=cf))
         tokens = int(ln.sum().item())
-        out["lattice_" + name] = {"ms_per_decode": ms, "tokens": tokens, "tokens_per_s": tokens / ms * 1e3,
-                                  "launches_per_decode": w.T + 2}
+        out["lattice_" + name] = {"ms_per_decode_median": med, "ms_per_decode_min": mn, "tokens": tokens,
+                                  "tokens_per_s": tokens / med * 1e3, "launches_per_decode": w.T + 2,
+                                  "row_gbs": tokens * w.V * w.elem_bytes / med / 1e6}
     # the other direction on the sequences just decoded: sequence -> interval, same tokens
     run_iid()
-    fn = lambda: B.as_encode_bigram(table, prev, seq, ln, w.temp, w.top_k, w.top_p)
-    for _ in range(max(1, warmup)):
-        fn()
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    a.record()
-    for _ in range(steps):
-        fn()
-    b.record()
-    torch.cuda.synchronize()
-    ms = a.elapsed_time(b) / steps
+    med, mn = timed(lambda: B.as_encode_bigram(table, prev, seq, ln, w.temp, w.top_k, w.top_p))
     tokens = int(ln.sum().item())
-    out["encode"] = {"ms_per_encode": ms, "tokens": tokens, "tokens_per_s": tokens / ms * 1e3}
+    out["encode"] = {"ms_per_encode_median": med, "ms_per_encode_min": mn, "tokens": tokens,
+                     "tokens_per_s": tokens / med * 1e3, "row_gbs": tokens * w.V * w.elem_bytes / med / 1e6}
     # what is computed from the decoded groups: n-gram diversity (Sec. 5.1) and the sample-mean
     # estimator of an additive synthetic reward (Sec. 4.2 / 5.2), lattice codes against iid codes
     r = torch.from_numpy(synth.reward_table(w.V, 78)).cuda()
-
-    def timed_call(fn, reps=20):
-        fn()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        a.record()
-        for _ in range(reps):
-            fn()
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / reps
-
     K = 16
     fits = w.N * w.T <= B.NGRAM_MAX_ITEMS          # one group's tokens and hash table in shared memory
     shifts = np.random.default_rng(79).random(K)
@@ -384,17 +484,90 @@ def bench_bigram(steps: int, warmup: int, S: int = 64, T: int = 128):
         means = torch.stack(means)
         stats[name] = {"estimator_sd_over_%d_runs_mean_over_groups" % K: float(means.std(dim=0).mean().item()),
                        "ngram_diversity_mean": float(torch.stack(divs).mean().item()) if fits else None}
-    stats["ms_ngram_diversity"] = timed_call(lambda: B.as_ngram_diversity(seq, ln, w.N)) if fits else None
-    stats["ms_reward_mean"] = timed_call(lambda: B.as_reward_mean(seq, ln, w.N, r))
+    stats["ms_ngram_diversity"] = timed(lambda: B.as_ngram_diversity(seq, ln, w.N))[0] if fits else None
+    stats["ms_reward_mean"] = timed(lambda: B.as_reward_mean(seq, ln, w.N, r))[0]
     out["groups"] = stats
+    if eos_variant:
+        # SUPPLEMENTARY variant, not the configuration as specified: with a random permutation the
+        # EOS column's bias makes P(EOS) ~ 1e-10 and no lane ever stops early; here that column's
+        # bias is raised (on the device: fp32 add, rounded to bf16 again) so that lanes stop after
+        # ~30 tokens on average and per-lane early stop, padding and ragged lengths are timed
+        eb = -3.0
+        col = table[:, w.eos].float() - float(w.column_bias()[w.eos]) + eb
+        tbl2 = table.clone()
+        tbl2[:, w.eos] = col.to(table.dtype)
+        note = "EOS column bias raised from %.2f to %.2f" % (float(w.column_bias()[w.eos]), eb)
+        out["eos_raised_lattice"] = decode_entry(lambda: run_lattice(tbl2), note)
+        out["eos_raised_iid"] = decode_entry(lambda: run_iid(tbl2), note)
+        del tbl2
     out["workload"] = "c4: bf16 bigram table 32128x32128, %d starts x 32 codes, T<=%d, temp 0.8, EOS 1" % (S, T)
     return out
 
 
 # ----------------------------------------------------------------------------- arms
+def side_measurements(B, peak, skip_key):
+    """One roofline block per step configuration (the headline's is measured by the caller), the
+    iid-code run of the step kernel beside the lattice run, the cluster kernel beside the streaming
+    kernel, two shapes outside the configurations, and the bigram loop."""
+    import torch
+    blocks, extras = {}, {}
+    for name, lanes in (("c2", None), ("c3", None), ("c5", 1024), ("c5", 4096), ("c5", 8192)):
+        w = step_workload(name, lanes)
+        key = step_key(w)
+        if key == skip_key:
+            continue
+        sb = StepBench(w, 0)
+        med, mn, n = sb.per_launch_us(sb.step_stored)
+        tpl = captured_traffic("as_step_stream_%s.md" % w.name, w.name)
+        blocks[key] = roofline_block(w, med, mn, n, peak, step_bytes(w), tpl, stream_kernel_name(w))
+        imed, imn, _ = sb.per_launch_us(sb.step_iid)
+        blocks[key]["iid_codes_us_per_launch_median"] = imed
+        blocks[key]["iid_codes_us_per_launch_min"] = imn
+        if key == "c2":
+            fmed, fmn, _ = sb.per_launch_us(sb.step)
+            tmed, tmn, _ = sb.per_launch_us(sb.step_two_calls)
+            blocks[key]["fused_first_step_us_median"] = fmed          # as_step_lattice
+            blocks[key]["two_calls_us_median"] = tmed                 # as_lattice_codes + as_step
+        if key == "c5_1024":
+            # the row split over a thread-block cluster (4 and 8 CTAs per lane) beside the default
+            for cs in (4, 8):
+                try:
+                    B.as_tune(B.TUNE_STEP_PATH, 2)
+                    B.as_tune(B.TUNE_CLUSTER, cs)
+                    cmed, cmn, _ = sb.per_launch_us(sb.step_stored)
+                finally:
+                    B.as_tune(B.TUNE_CLUSTER, 0)
+                    B.as_tune(B.TUNE_STEP_PATH, 0)
+                blocks[key]["cluster_kernel_cs%d_us_median" % cs] = cmed
+                blocks[key]["cluster_kernel_cs%d_us_min" % cs] = cmn
+        del sb
+        torch.cuda.empty_cache()
+    # shapes outside the configurations: many lanes of a 32000-token vocabulary, flat rows with a wide
+    # nucleus, and a step without any cut (every token kept)
+    for key, w in (("many_lanes_4096x32000_top_k_40",
+                    synth.StepWorkload("x1", 4096, 32000, synth.BF16, 3.0, 0.7, 40, 1.0, 20, 21, 22)),
+                   ("no_cut_2048x32128_temp_0.8",
+                    synth.StepWorkload("x2", 2048, 32128, synth.BF16, 2.5, 0.8, 0, 1.0, 40, 41, 43))):
+        sb = StepBench(w, 0)
+        med, mn, n = sb.per_launch_us(sb.step_stored)
+        extras[key] = roofline_block(w, med, mn, n, peak, step_bytes(w))
+        del sb
+        torch.cuda.empty_cache()
+    w = synth.StepWorkload("x3", 1024, 128256, synth.BF16, 3.0, 0.8, 0, 0.9, 60, 61, 62)
+    sb = StepBench(w, 0)
+    sb.ring = [device_rows(w.lanes, w.V, w.sigma, w.dtype, 60, None)]      # no Zipf bias: flat rows
+    med, mn, n = sb.per_launch_us(sb.step_stored, replays=5)
+    extras["wide_nucleus_flat_1024x128256_top_p_0.9"] = roofline_block(w, med, mn, n, peak, step_bytes(w))
+    del sb
+    torch.cuda.empty_cache()
+    extras["bigram_decode"] = bench_bigram(10, 2)
+    return blocks, extras
+
+
 def run_ours(args):
     import torch
     rank, local_rank, world = dist_env()
+    check_world(args.gpus, world)
     torch.cuda.set_device(local_rank)
     if world > 1:
         import torch.distributed as dist
@@ -402,88 +575,74 @@ def run_ours(args):
     from paper_2210_15458_b200 import binding as B
     B.lib()
     w = step_workload(args.workload, args.lanes)
+    key = step_key(w)
     sb = StepBench(w, rank)
     for _ in range(args.warmup):
         sb.step()
+    g = sb.graph(sb.step, args.steps)              # the timed region: exactly K steps
+    sb.replay_ms(g)                                # untimed: the first replay uploads the graph
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
     barrier(world)
-    ms = sb.timed(sb.step, args.steps)
+    ms = sb.replay_ms(g)
     barrier(world)
     if rank == 0:
-        # the timed replay lasts a few tens of ms; keep the same graph running for ~0.5 s so that
-        # nvidia-smi (100 ms period) sees the clocks under this load
-        t_end = time.perf_counter() + 0.5
+        # keep the same load running for ~0.6 s so that nvidia-smi (100 ms period) sees its clocks
+        t_end = time.perf_counter() + 0.6
         while time.perf_counter() < t_end:
-            sb.last_graph.replay()
-        torch.cuda.synchronize()
+            g.replay()
+            torch.cuda.synchronize()
     ms = max_over_ranks(ms, world, torch.device("cuda", local_rank))
-    # the step is a single launch of the step kernel: its duration is the step's; the same kernel
-    # on stored codes (as_step) and the two-launch form are timed beside it
-    for _ in range(3):
-        sb.step_kernel_only()
-    kern_launches = max(args.steps, 200)
-    kms = sb.timed(sb.step, kern_launches) / kern_launches
-    kms_stored = sb.timed(sb.step_kernel_only, kern_launches) / kern_launches
-    ms2 = sb.timed(sb.step_two_calls, kern_launches) / kern_launches
     clocks = sampler.stop() if rank == 0 else None
+    del g
     if rank != 0:
         if world > 1:
             torch.distributed.destroy_process_group()
         return
     peak, peak_kind = measured_peaks()
-    logits_per_step = w.lanes * w.V * world
-    value = logits_per_step * args.steps / (ms / 1e3)
-    lattice_step_bytes = step_bytes(w) - 8 * w.lanes          # the codes are not read from memory
-    achieved = lattice_step_bytes / (kms / 1e3) / 1e9
+    # the dominant kernel: the step is a single launch of the step kernel, timed launch by launch
+    med, mn, n = sb.per_launch_us(sb.step)
+    tpl = captured_traffic("as_step_stream_%s.md" % w.name, w.name)
+    head = roofline_block(w, med, mn, n, peak, step_bytes(w, stored_codes=False), tpl,
+                          stream_kernel_name(w) + " via as_step_lattice")
+    head["peak_kind"] = peak_kind
+    smed, smn, _ = sb.per_launch_us(sb.step_stored)
+    imed, imn, _ = sb.per_launch_us(sb.step_iid)
+    head["stored_lattice_codes_us_per_launch_median"] = smed
+    head["iid_codes_us_per_launch_median"] = imed
+    head["iid_codes_us_per_launch_min"] = imn
+    value = w.lanes * w.V * world * args.steps / (ms / 1e3)
     line = {
         "metric": "logits decoded/s", "value": value, "unit": "logits/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "%s: %d lanes x V=%d %s logits, temp %g, top_k %d, top_p %g, fp64 lattice codes"
-                               % (w.name, w.lanes, w.V, "bf16" if w.dtype else "f32", w.temp, w.top_k, w.top_p),
-                   "lanes_per_gpu": w.lanes, "V": w.V, "l2": "inputs rotate through %d buffers (%.0f MB > 3x L2)"
-                                                             % (len(sb.ring), sb.ring_bytes / 1e6),
+        "config": {"workload": workload_text(w), "lanes_per_gpu": w.lanes, "V": w.V, "l2": sb.l2_note(),
                    "step": "one as_step_lattice launch: lattice codes of a fresh shift formed in the step kernel",
-                   "timing": "K steps captured in one CUDA graph, replayed once between events",
+                   "timing": "the K steps captured in one CUDA graph, replayed once between CUDA events; per-launch "
+                             "median / min from %d replays of a shorter graph" % REPLAYS,
+                   "inputs": "drawn on the device in the configuration's distribution (seeded)",
                    "parallelism": "lanes sharded, no collective"},
         "lane_steps_per_s": w.lanes * world * args.steps / (ms / 1e3),
+        "hbm_gbs": step_bytes(w, stored_codes=False) * world * args.steps / (ms / 1e3) / 1e9,
         "gpu_launches": args.steps,
-        "ms_per_step_two_calls": ms2,          # as_lattice_codes + as_step on the stored codes
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "step_stream_kernel (as_step_lattice)", "achieved": achieved,
-                     "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_kind": peak_kind, "frac_of_8TBs_nominal": achieved / 8000.0,
-                     "us_per_launch": kms * 1e3, "bytes_per_launch": lattice_step_bytes,
-                     "us_per_launch_stored_codes": kms_stored * 1e3,
-                     "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+        "roofline": head,
     }
+    del sb
+    torch.cuda.empty_cache()
     if world == 1:
-        e_ms, h2d, d2h = e2e_step(w, args.steps, args.warmup)
-        line["e2e"] = {"value": w.lanes * w.V * args.steps / (e_ms / 1e3), "unit": "logits/s",
-                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e_ms / args.steps}
+        e_steps = max(1, min(args.steps, 3 if w.lanes * w.V * w.elem_bytes > (1 << 30) else 50))
+        e_ms, h2d, d2h = e2e_step(w, e_steps, 1 if e_steps <= 3 else 3)
+        line["e2e"] = {"value": w.lanes * w.V * e_steps / (e_ms / 1e3), "unit": "logits/s",
+                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e_ms / e_steps,
+                       "steps": e_steps, "entry_point": "as_step_host (pinned host buffers)"}
+        torch.cuda.empty_cache()
         line["cpu_baseline"] = cpu_baseline_step(w)
+        line["rooflines"] = {key: head}
         if not args.no_extras:
-            extras = {}
-            for name, lanes in (("c3", None), ("c5", 1024), ("c5", 4096), ("c5", 8192)):
-                if name == w.name:
-                    continue
-                del sb
-                torch.cuda.empty_cache()
-                ww = step_workload(name, lanes)
-                sb = StepBench(ww, 0, base_lanes=1024)
-                for _ in range(3):
-                    sb.step_kernel_only()
-                n = 2 * len(sb.ring) if len(sb.ring) > 1 else 6
-                k = sb.timed(sb.step_kernel_only, n) / n
-                gbs = step_bytes(ww) / (k / 1e3) / 1e9
-                key = name if lanes in (None, 1024) else "%s_%d" % (name, lanes)
-                extras[key] = {"lanes": ww.lanes, "V": ww.V, "us_per_launch": k * 1e3, "GBs": gbs,
-                               "frac_of_peak": gbs / peak, "logits_per_s": ww.lanes * ww.V / (k / 1e3)}
-            del sb
-            torch.cuda.empty_cache()
-            extras["bigram_decode"] = bench_bigram(2, 1)
+            blocks, extras = side_measurements(B, peak, key)
+            line["rooflines"].update(blocks)
             line["other_workloads"] = extras
     else:
         line["e2e"] = None
@@ -498,7 +657,11 @@ def run_reference(args):
     from oracle import oracle
     w = step_workload(args.workload, args.lanes)
     cores = os.cpu_count() or 1
-    lanes = min(w.lanes, 256)
+    # each step is a bounded sample of the workload's lanes, sized from a short probe so that the
+    # K steps take about a minute
+    probe = min(w.lanes, 32)
+    rate, _, _, _ = oracle_rate(w, probe, 2.0)
+    lanes = int(max(1, min(w.lanes, 256, rate * 60.0 / (max(args.steps, 1) * w.V))))
     arr = w.logits(lanes)
     threads = min(cores, lanes)
     shifts = np.random.default_rng(1234).random(4096)
@@ -518,8 +681,7 @@ def run_reference(args):
         "impl": "reference", "metric": "logits decoded/s", "value": value, "unit": "logits/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "%s: %d lanes x V=%d %s logits, temp %g, top_k %d, top_p %g (CPU oracle, %s)"
-                               % (w.name, lanes, w.V, "bf16" if w.dtype else "f32", w.temp, w.top_k, w.top_p, sample)},
+        "config": {"workload": workload_text(w) + " (CPU oracle, %s)" % sample},
         "cpu_baseline": {"value": value, "unit": "logits/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "logits/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
@@ -528,21 +690,25 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c5", "c4"],
+    ap.add_argument("--workload", default="c5", choices=["c2", "c3", "c5", "c4"],
                     help="c4 prints the bigram decode / encode loop's own line (a side measurement)")
     ap.add_argument("--lanes", type=int, default=None,
-                    help="lanes for c3 / c5 / c4 (default: the configured size; c4: a multiple of 32)")
+                    help="lanes for c3 / c5 / c4 (default: c5 8192, c3 1024, c4 2048; c4: a multiple of 32)")
     ap.add_argument("--T", type=int, default=128, help="c4 only: maximum steps per lane (512-1024: summarisation-sized outputs)")
-    ap.add_argument("--no-extras", action="store_true", help="skip the other workloads' short measurements")
+    ap.add_argument("--no-extras", action="store_true", help="skip the other configurations' blocks")
     args = ap.parse_args()
     args.warmup = max(3, args.warmup)
+    if args.gpus < 1:
+        raise SystemExit("--gpus must be >= 1")
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus))
     if args.workload == "c4":
         if args.impl == "reference" or dist_env()[2] > 1:
             raise SystemExit("--workload c4 is a single-GPU side measurement of the CUDA path")
-        print(json.dumps(bench_bigram(min(args.steps, 20), min(args.warmup, 3), S=(args.lanes or 2048) // 32,
+        print(json.dumps(bench_bigram(min(args.steps, 10), min(args.warmup, 3), S=(args.lanes or 2048) // 32,
                                       T=args.T)))
     elif args.impl == "reference":
         run_reference(args)

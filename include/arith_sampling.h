@@ -314,8 +314,8 @@ int as_reward_mean(const int32_t *d_seq, const int32_t *d_len, int S, int N, int
                    int32_t *d_group_status, void *stream);
 
 /*
- * Launch-shape overrides for measurement sweeps (process-wide, not thread-safe;
- * 0 restores the built-in choice).  Keys:
+ * Launch-shape overrides for measurement sweeps and tests (0 restores the built-in
+ * choice).  Keys:
  *   AS_TUNE_STEP_PATH     0 = streaming kernel (one CTA per lane), 1 = general kernel only,
  *                         2 = cluster kernel (row split over the CTAs of a cluster)
  *   AS_TUNE_CLUSTER       CTAs per lane for the cluster kernel (1, 2, 4, 8)
@@ -331,7 +331,16 @@ int as_reward_mean(const int32_t *d_seq, const int32_t *d_len, int S, int N, int
  *                         kernel before it on the stream drains (programmatic dependent launch;
  *                         it still waits for that kernel's completion before it reads or
  *                         writes global memory, so results do not depend on this key)
- * Returns AS_ERR_INVALID_ARG for an unknown key or value.
+ *   AS_TUNE_WAIT_KCYCLES  bound on every on-device wait for a copy, in units of 1000 clock
+ *                         cycles (default: 2,000,000 = about one second).  A wait that runs out
+ *                         ends the lane with status AS_ERR_TIMEOUT (token -1, code unchanged);
+ *                         the kernel returns normally and later calls are not affected
+ *   AS_TUNE_DEBUG_NO_COPY 1 = the copy-issuing thread of the step kernels issues nothing, so
+ *                         every wait runs out: exists only so that a test can exercise the
+ *                         AS_ERR_TIMEOUT path without any copy in flight; use it with a small
+ *                         AS_TUNE_WAIT_KCYCLES
+ * Returns AS_ERR_INVALID_ARG for an unknown key or value.  The keys are process-wide; a launch
+ * reads each once (concurrent calls see the old or the new value).
  */
 #define AS_TUNE_STEP_PATH 1
 #define AS_TUNE_CLUSTER 2
@@ -339,6 +348,8 @@ int as_reward_mean(const int32_t *d_seq, const int32_t *d_len, int S, int N, int
 #define AS_TUNE_STAGES 4
 #define AS_TUNE_MIN_CTAS 5
 #define AS_TUNE_SERIAL_LAUNCH 6
+#define AS_TUNE_WAIT_KCYCLES 7
+#define AS_TUNE_DEBUG_NO_COPY 8
 int as_tune(int key, int value);
 
 /* Text of the calling thread's most recent error ("" if none). Never NULL. */

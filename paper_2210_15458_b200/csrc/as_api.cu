@@ -3,6 +3,7 @@
 #include "as_stream.cuh"
 #include "as_metrics.cuh"
 
+#include <atomic>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -14,7 +15,20 @@ namespace asx {
 // host-side state
 // ---------------------------------------------------------------------------
 static thread_local char g_err[512] = "";
-static int g_tune_path = 0, g_tune_cluster = 0, g_tune_ctas = 0, g_tune_stages = 0, g_tune_minb = 0, g_tune_serial = 0;
+// launch-shape overrides (as_tune): each is read once per launch; relaxed atomics make a
+// concurrent as_tune well-defined (a launch sees the old or the new value)
+struct Tune {
+    std::atomic<int> v{0};
+    operator int() const { return v.load(std::memory_order_relaxed); }
+    void operator=(int x) { v.store(x, std::memory_order_relaxed); }
+};
+static Tune g_tune_path, g_tune_cluster, g_tune_ctas, g_tune_stages, g_tune_minb, g_tune_serial,
+    g_tune_wait_kcycles, g_tune_no_copy;
+
+static long long wait_cycles_now() {
+    const int k = g_tune_wait_kcycles;
+    return k > 0 ? (long long)k * 1000 : ST_WAIT_CYCLES;
+}
 
 static int set_err(int code, const char* fmt, ...) {
     va_list ap;
@@ -431,6 +445,14 @@ int as_tune(int key, int value) {
             if (value < 0 || value == 1 || value > SK_MAXSTAGES) return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_STAGES takes 0 or 2..12");
             g_tune_stages = value;
             return AS_OK;
+        case AS_TUNE_WAIT_KCYCLES:
+            if (value < 0) return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_WAIT_KCYCLES takes 0 (default) or a positive count of 1000 cycles");
+            g_tune_wait_kcycles = value;
+            return AS_OK;
+        case AS_TUNE_DEBUG_NO_COPY:
+            if (value != 0 && value != 1) return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_DEBUG_NO_COPY takes 0 or 1");
+            g_tune_no_copy = value;
+            return AS_OK;
         default:
             return set_err(AS_ERR_INVALID_ARG, "unknown tuning key %d", key);
     }
@@ -520,6 +542,7 @@ static int step_common(const void* d_logits, int dtype, int lanes, int V, long l
     a.lanes = lanes; a.V = V; a.top_k = top_k;
     a.lat_N = lat_N; a.lat_j0 = lat_j0; a.lat_u = lat_u;
     a.row_idx = nullptr; a.idx_stride = 1; a.tok_stride = 1; a.eos = -1; a.rows = 0;
+    a.wait_cycles = wait_cycles_now(); a.debug_no_copy = g_tune_no_copy;
     const int E = dtype == AS_F32 ? 4 : 8;
     const size_t esz = dtype == AS_F32 ? 4 : 2;
     // some row starts off a 16-byte boundary: it is read from the boundary below, up to E-1 elements longer
@@ -618,7 +641,11 @@ int as_step_host(const void* h_logits, int dtype, int lanes, int V, long long ld
     if ((e = cudaMemcpyAsync(d_codes, h_codes, (size_t)lanes * 8, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "copy codes to device");
     as_step_diag dg = {nullptr, nullptr, nullptr, d_status, nullptr};
     rc = as_step(d_logits, dtype, lanes, V, d_ld, d_codes, temp, top_k, top_p, d_tokens, d_codes_out, &dg, stream);
-    if (rc != AS_OK) return rc;
+    if (rc != AS_OK) {
+        // the copies above are queued on the work buffer: do not hand it back while they run
+        cudaStreamSynchronize(st);
+        return rc;
+    }
     if ((e = cudaMemcpyAsync(h_tokens, d_tokens, (size_t)lanes * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "copy tokens to host");
     if ((e = cudaMemcpyAsync(h_codes_out, d_codes_out, (size_t)lanes * 8, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "copy codes to host");
     if (h_lane_status && (e = cudaMemcpyAsync(h_lane_status, d_status, (size_t)lanes * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "copy status to host");
@@ -698,6 +725,7 @@ static int decode_common(const void* d_table, int dtype, int V, long long ld, co
         a.lanes = lanes; a.V = V; a.top_k = top_k;
         a.lat_N = 0; a.lat_j0 = 0; a.lat_u = 0.0;
         a.rows = V;
+        a.wait_cycles = wait_cycles_now(); a.debug_no_copy = g_tune_no_copy;
         cudaError_t e;
         bool served = true;
         for (int t = 0; t < T && served; ++t) {

@@ -17,8 +17,8 @@ constexpr int ST_NUMERIC = -5;
 #define ASX_ONE_BELOW 0x1.fffffffffffffp-1
 
 // ---------------------------------------------------------------------------
-// Keys: an unsigned integer whose order equals the order of the stored float.
-// -inf maps to KEY_NINF (masked token); anything below it is a negative NaN,
+// Keys: an unsigned integer whose order equals the order of the stored float
+// (the two zeros share one key).  -inf maps to KEY_NINF (masked token); anything below it is a negative NaN,
 // anything >= KEY_PINF is +inf or a positive NaN.
 // ---------------------------------------------------------------------------
 template <int DT> struct Traits;
@@ -29,7 +29,9 @@ template <> struct Traits<DT_F32> {
     static constexpr int KEYBITS = 32;
     static constexpr uint32_t KEY_NINF = 0x007FFFFFu;
     static constexpr uint32_t KEY_PINF = 0xFF800000u;
+    // (-0.0 gets the key of +0.0: the two compare equal, so they must tie and fall to the index)
     __device__ __forceinline__ static uint32_t key_of(uint32_t bits) {
+        if (bits == 0x80000000u) bits = 0u;
         return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
     }
     __device__ __forceinline__ static float value_f(uint32_t key) {
@@ -51,6 +53,7 @@ template <> struct Traits<DT_BF16> {
     static constexpr uint32_t KEY_NINF = 0x007Fu;
     static constexpr uint32_t KEY_PINF = 0xFF80u;
     __device__ __forceinline__ static uint32_t key_of(uint32_t b16) {
+        if (b16 == 0x8000u) b16 = 0u;                   // -0.0 ties with +0.0
         return (b16 & 0x8000u) ? (~b16 & 0xFFFFu) : (b16 | 0x8000u);
     }
     __device__ __forceinline__ static float value_f(uint32_t key) {

@@ -38,7 +38,7 @@ constexpr int ST_CHUNK_BYTES = ST_CHUNK_VEC * 16;
 constexpr int ST_MAXCHUNK = 27;        // 27 * 8 KB = 216 KB
 constexpr int ST_M = 2 * ST_NT;        // subset maxima per CTA
 constexpr int ST_KP = 256;             // candidates aimed at for nucleus-only lanes
-constexpr long long ST_WAIT_CYCLES = 4000000000LL;   // ~2 s: bound on any mbarrier wait
+constexpr long long ST_WAIT_CYCLES = 2000000000LL;   // ~1 s: default bound on any mbarrier wait
 
 // Phase timestamps of CTA 0 for profiling builds (-DASX_PROFILE); compiled out otherwise.
 #ifdef ASX_PROFILE
@@ -110,6 +110,10 @@ struct StepArgs {
     int tok_stride;
     int eos;
     int rows;
+    // bound on every mbarrier wait, in clock cycles; when it runs out the lane reports ST_TIMEOUT
+    long long wait_cycles;
+    // test of the time-out path only: the copy-issuing thread issues nothing, so every wait runs out
+    int debug_no_copy;
 };
 
 __device__ __forceinline__ double lane_code(const StepArgs& a, int ln) {
@@ -144,15 +148,15 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-// waits for the phase with the given parity; gives up after ST_WAIT_CYCLES
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+// waits for the phase with the given parity; gives up after `limit` clock cycles
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, long long limit) {
     const long long t0 = clock64();
     for (;;) {
         uint32_t ok;
         asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
                      " selp.u32 %0, 1, 0, p;\n}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
         if (ok) return true;
-        if (clock64() - t0 > ST_WAIT_CYCLES) return false;
+        if (clock64() - t0 > limit) return false;
     }
 }
 // ---------------------------------------------------------------------------
@@ -401,7 +405,7 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
     // bring this CTA's slice of lane ln's row into shared memory
     auto issue = [&](int ln) {
         const char* src = row_of(ln) + (size_t)elem0 * Tr::BYTES;
-        if (tid == 0 && !poisoned) {
+        if (tid == 0 && !poisoned && !a.debug_no_copy) {
             fence_proxy_async();
             for (int i = 0; i < nchunk; ++i) {
                 const uint32_t bytes = (uint32_t)min(ST_CHUNK_BYTES, bulk_bytes - i * ST_CHUNK_BYTES);
@@ -452,7 +456,7 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
         typename P::Acc acc = P::init();
         bool timed_out = poisoned;
         for (int i = 0; i < nchunk; ++i) {
-            if (!poisoned && !mbar_wait_bounded(smem_u32(&sm.bars[i]), phase & 1)) timed_out = true;
+            if (!poisoned && !timed_out && !mbar_wait_bounded(smem_u32(&sm.bars[i]), phase & 1, a.wait_cycles)) timed_out = true;
             const int v = i * ST_CHUNK_VEC + tid;
             if (v < bulk_vec) P::fold(acc, rowv[v]);
         }
@@ -611,9 +615,9 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
         }
         ASX_MARK(12);
     }
-    if (poisoned && tid == 0) {
+    if (poisoned && tid == 0 && !a.debug_no_copy) {
         // copies issued before the wait ran out may still be in flight: give them one more bounded wait
-        for (int i = 0; i < nchunk; ++i) mbar_wait_bounded(smem_u32(&sm.bars[i]), (phase - 1) & 1);
+        for (int i = 0; i < nchunk; ++i) mbar_wait_bounded(smem_u32(&sm.bars[i]), (phase - 1) & 1, a.wait_cycles);
     }
     if (CS > 1) cluster.sync();     // no CTA leaves while a peer may still write into its shared memory
 }

@@ -74,6 +74,8 @@ struct StreamSmemT {
     int vec_count;
     int cand_count;
     int poisoned;        // a bounded wait ran out: stop issuing / stop waiting
+    int prod_done;       // the copy-issuing thread has left; prod_st / prod_round say what it armed
+    unsigned prod_st, prod_round;
     int b_i[4];
 };
 
@@ -579,13 +581,14 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                 if (p_round >= 1) {               // the stage must have been drained by every consumer warp
                     if (first_row_only) return true;
                     if (*(volatile int*)&sm.poisoned) return false;
-                    if (!mbar_wait_bounded(smem_u32(&sm.empty_bar[st]), (p_round - 1) & 1)) {
+                    if (!mbar_wait_bounded(smem_u32(&sm.empty_bar[st]), (p_round - 1) & 1, a.wait_cycles)) {
                         *(volatile int*)&sm.poisoned = 1;
                         return false;
                     }
                 }
                 const uint32_t bytes = (uint32_t)min(SK_STAGE_BYTES, bulk_bytes_i - s_issue * SK_STAGE_BYTES);
                 const uint32_t bar = smem_u32(&sm.full_bar[st]);
+                if (a.debug_no_copy) return false;    // (time-out test: nothing is armed, nothing is in flight)
                 mbar_expect_tx(bar, bytes);
                 bulk_g2s(smem_u32(ring + (size_t)st * SK_STAGE_BYTES), src + (size_t)s_issue * SK_STAGE_BYTES, bytes, bar);
             }
@@ -604,6 +607,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         }
         fence_mbar_init();
         sm.poisoned = 0;
+        sm.prod_done = 0;
     }
     fill_exp_table(sm.exp_tbl, tid);
     pdl_wait_prev();
@@ -612,7 +616,14 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
 
     // =========================== producer warp ===========================
     if (warp == SK_NW) {
-        if (lane == 0) issue_some(false);
+        if (lane == 0) {
+            issue_some(false);
+            // what has been armed, for the consumers' drain should a wait run out
+            sm.prod_st = p_st;
+            sm.prod_round = p_round;
+            __threadfence_block();
+            *(volatile int*)&sm.prod_done = 1;
+        }
         return;
     }
     // =========================== consumer warps ===========================
@@ -817,7 +828,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         auto wait_full = [&](int off) {            // slice g + off, off < S
             if (*(volatile int*)&sm.poisoned) return;
             const unsigned par = g_par ^ (g_st + off >= (unsigned)S ? 1u : 0u);
-            if (!mbar_wait_bounded(smem_u32(&sm.full_bar[stage_of(off)]), par)) *(volatile int*)&sm.poisoned = 1;
+            if (!mbar_wait_bounded(smem_u32(&sm.full_bar[stage_of(off)]), par, a.wait_cycles)) *(volatile int*)&sm.poisoned = 1;
         };
         auto release = [&](int off) {
             __syncwarp();
@@ -1066,6 +1077,22 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         SyncC::sync();
         ASX_MARK(12);
         ASX_CTA(6);
+    }
+    if (tid == 0 && *(volatile int*)&sm.poisoned) {
+        // A wait ran out.  Copies armed before that may still be in flight into this CTA's shared
+        // memory: the CTA does not leave before each armed stage has landed or its own bounded
+        // wait has run out as well.  (The copy-issuing thread stops at its next wait once it sees
+        // the flag, and says what it had armed.)
+        const long long t0 = clock64();
+        while (!*(volatile int*)&sm.prod_done && clock64() - t0 <= 2 * a.wait_cycles + 1000000) { }
+        if (*(volatile int*)&sm.prod_done) {
+            __threadfence_block();
+            const unsigned pst = sm.prod_st, prd = sm.prod_round;
+            for (unsigned st = 0; st < (unsigned)S; ++st) {
+                const int rnd = (int)prd - (st < pst ? 0 : 1);       // the last round that armed this stage
+                if (rnd >= 0 && !mbar_wait_bounded(smem_u32(&sm.full_bar[st]), (unsigned)rnd & 1u, a.wait_cycles)) break;
+            }
+        }
     }
     ASX_MARK(14);
     ASX_SPAN(2);

@@ -152,30 +152,68 @@ def test_c2_full(B, orc):
     check(B, orc, arr, BF16, iid, w.temp, w.top_k, w.top_p, what="c2 iid")
 
 
-def _sampled_full_size(B, orc, w, sample, seed):
+def _sampled_full_size(B, orc, w, sample, seed, extra=None):
+    """The whole configuration through the CUDA path in the launch shape the benchmark times;
+    `sample` lanes spread over the whole range (plus those `extra` picks from the GPU's own
+    diagnostics) go through the oracle one by one; every lane gets range checks."""
     arr = w.logits()
     codes = orc.lattice_codes(w.N, w.shift())[: w.lanes]
-    tok, c2, p, nk, st = gpu_step(B, arr, w.dtype, codes, w.temp, w.top_k, w.top_p)
-    idx = np.sort(np.random.default_rng(seed).choice(w.lanes, sample, replace=False))
+    d = {}
+    tok, c2 = B.as_step(to_dev(arr, w.dtype), torch.from_numpy(codes).cuda(), w.temp, w.top_k, w.top_p, diag=d)
+    torch.cuda.synchronize()
+    tok, c2 = tok.cpu().numpy(), c2.cpu().numpy()
+    p, nk, st, path = (d[k].cpu().numpy() for k in ("p_tok", "n_kept", "lane_status", "path"))
+    rng = np.random.default_rng(seed)
+    # one lane from each of `sample` equal stretches: early and late rows of every persistent CTA
+    edges = np.linspace(0, w.lanes, sample + 1).astype(np.int64)
+    idx = set(int(rng.integers(edges[i], edges[i + 1])) for i in range(sample))
+    if extra is not None:
+        idx |= set(int(i) for i in extra(nk, path))
+    idx = np.array(sorted(idx))
     ref = orc.step(np.ascontiguousarray(arr[idx]), w.dtype, codes[idx], w.temp, w.top_k, w.top_p, threads=8)
     r = compare_step(ref, tok[idx], c2[idx], p[idx], nk[idx], st[idx], what=w.name)
     assert (st == 0).all() and (tok >= 0).all() and (tok < w.V).all()
     assert (c2 >= 0).all() and (c2 < 1).all() and (nk >= 1).all()
     if w.top_k:
         assert (nk <= w.top_k).all()
+    r["sampled"] = len(idx)
     return r
 
 
 def test_c3_full_size_sampled(B, orc):
     from paper_2210_15458_b200 import synth
-    r = _sampled_full_size(B, orc, synth.c3(), 64, 1)
+
+    def deep_lanes(nk, path):
+        # the lanes with the largest kept sets are the ones whose nucleus reached below the first
+        # threshold (the list was deepened) or that went to the general routine
+        return list(np.argsort(-nk)[:24]) + list(np.nonzero(path == B.PATH_GENERAL)[0][:16])
+    r = _sampled_full_size(B, orc, synth.c3(), 128, 1, extra=deep_lanes)
+    assert r["sampled"] >= 128 and r["compared"] >= 0.9 * r["sampled"]
+
+
+@pytest.mark.parametrize("lanes", [1024, 4096, 8192])
+def test_c5_full_size_sampled(B, orc, lanes):
+    from paper_2210_15458_b200 import synth
+    r = _sampled_full_size(B, orc, synth.c5(lanes), 64, 2 + lanes)
     assert r["compared"] >= 56
 
 
-def test_c5_full_size_sampled(B, orc):
+@pytest.mark.parametrize("cluster", [4, 8])
+def test_c5_rows_through_the_cluster_kernel(B, orc, cluster):
+    # the row split over the CTAs of a thread-block cluster (slices in distributed shared memory)
+    # at the full vocabulary of the large-vocabulary configuration
     from paper_2210_15458_b200 import synth
-    r = _sampled_full_size(B, orc, synth.c5(1024), 48, 2)
-    assert r["compared"] >= 40
+    w = synth.c5(96)
+    arr = w.logits()
+    codes = orc.lattice_codes(w.N, w.shift())
+    try:
+        B.as_tune(B.TUNE_STEP_PATH, 2)
+        B.as_tune(B.TUNE_CLUSTER, cluster)
+        r = check(B, orc, arr, BF16, codes, w.temp, w.top_k, w.top_p, what="c5 cluster=%d" % cluster)
+        assert r["compared"] >= 88
+    finally:
+        B.as_tune(B.TUNE_CLUSTER, 0)
+        B.as_tune(B.TUNE_STEP_PATH, 0)
 
 
 # --------------------------------------------------------------------------- bigram decode loop
@@ -354,6 +392,11 @@ def test_c4_full_size_sampled(B, orc):
         assert (seq[i, :upto] == ref.seq[n, :upto]).all()
         compared += upto
     assert compared >= 5 * len(lanes)
+    # the same table with a cut: the loop then runs as one launch of the step kernel per step with
+    # the rows gathered from the table (Sec. 5.1 "Top-k sampling"), teacher-forced against the oracle
+    for k, p in [(10, 1.0), (0, 0.9), (40, 0.95)]:
+        ref, nsafe, nsteps = _teacher_forced(B, orc, table, BF16, dev, prev[:12], codes[:12], 10, w.eos, w.temp, k, p)
+        assert nsafe > 0.9 * nsteps and nsteps >= 100
 
 
 # --------------------------------------------------------------------------- launch shapes
@@ -641,3 +684,51 @@ def test_decode_with_cuts_per_step_kernels_equal_the_single_kernel(B, orc):
             assert (s1[i, l1[i]:] == -1).all() and (s1[i, :l1[i]] >= 0).all()
             if 0 < l1[i] < T:
                 assert s1[i, l1[i] - 1] == eos
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_step_signed_zeros_tie_and_fall_to_the_lower_index(B, orc, dtype):
+    # -0.0 and +0.0 are the same logit: where a top-k or nucleus boundary falls between them the
+    # lower index wins, whatever the signs
+    rng = np.random.default_rng(12)
+    V, lanes = 4099, 16
+    x = rng.normal(-4, 1, (lanes, V)).astype(np.float32)
+    for i in range(lanes):
+        z = rng.choice(V, 6, replace=False)
+        x[i, z] = np.where(rng.random(6) < 0.5, -0.0, 0.0).astype(np.float32)   # the six largest, signs mixed
+    x[0, :2] = [-0.0, 0.0]
+    arr = _store(x, dtype)
+    codes = rng.random(lanes)
+    for temp, k, p in [(1.0, 1, 1.0), (1.0, 3, 1.0), (0.8, 0, 0.4), (1.0, 5, 0.5)]:
+        check(B, orc, arr, dtype, codes, temp, k, p, what="signed zeros %s" % ((temp, k, p),))
+    tok, _ = B.as_step(to_dev(arr, dtype), torch.from_numpy(codes).cuda(), 1.0, 1, 1.0)
+    ref = orc.step(arr, dtype, codes, 1.0, 1, 1.0)
+    assert np.array_equal(tok.cpu().numpy(), ref.tokens)           # top_k = 1: no band, exact
+
+
+@pytest.mark.parametrize("path,V", [(0, 32000), (0, 140000), (2, 40000)])
+def test_a_wait_that_runs_out_reports_timeout_and_the_next_call_is_fine(B, orc, path, V):
+    # every wait for a copy is bounded.  With the copy-issuing thread told to issue nothing (so no
+    # copy is in flight) and a limit of a million cycles, the wait runs out: the lane must come back
+    # with AS_ERR_TIMEOUT, token -1 and its code unchanged, the kernel returns normally, and the
+    # next ordinary call gives the oracle's result.
+    rng = np.random.default_rng(V)
+    arr = _store(rng.normal(0, 3, (3, V)), BF16)
+    dev = to_dev(arr, BF16)
+    codes = np.array([0.25, 0.5, 0.75])
+    try:
+        B.as_tune(B.TUNE_STEP_PATH, path)
+        B.as_tune(B.TUNE_WAIT_KCYCLES, 1000)
+        B.as_tune(B.TUNE_DEBUG_NO_COPY, 1)
+        d = {}
+        tok, c2 = B.as_step(dev, torch.from_numpy(codes).cuda(), 0.8, 20, 1.0, diag=d)
+        torch.cuda.synchronize()
+        assert (d["lane_status"].cpu().numpy() == B.ERR_TIMEOUT).all()
+        assert (tok.cpu().numpy() == -1).all() and np.array_equal(c2.cpu().numpy(), codes)
+    finally:
+        B.as_tune(B.TUNE_DEBUG_NO_COPY, 0)
+        B.as_tune(B.TUNE_WAIT_KCYCLES, 0)
+    try:
+        check(B, orc, arr, BF16, codes, 0.8, 20, 1.0, what="after a time-out")
+    finally:
+        B.as_tune(B.TUNE_STEP_PATH, 0)

@@ -595,3 +595,99 @@ def test_naive_codebook_example_is_biased_but_consistent(orc):
         codes = orc.lattice_codes_variant(N, 0.0, 2)
         o = orc.decode_bigram_codes(table, F32, np.zeros(N, np.int32), codes, 1, -1)
         assert abs((o.seq[:, 0] == 1).mean() - 0.4) <= 1.0 / N
+
+
+# --------------------------------------------------------------------------- d_tok, the gate of every GPU comparison
+def test_d_tok_is_the_distance_to_the_nearest_cdf_boundary_exact(orc):
+    # Algorithm 1's interval (m, M) of the chosen token: d_tok = min(c - m, M - c).  With equal
+    # logits every kept token has probability 1/n exactly; for n a power of two the CDF values
+    # k/n and the codes below are dyadic, so every quantity is exact in fp64 and the oracle must
+    # return the distance bit for bit (a division by Z too many, a wrong end, a swapped sign fail).
+    ninf = -np.inf
+    for row, kept in [([0.5] * 8, list(range(8))),
+                      ([1.25, ninf, 1.25, 1.25, ninf, ninf, 1.25, ninf], [0, 2, 3, 6])]:
+        n = len(kept)
+        codes = (np.arange(256) + 0.25) / 256
+        o = orc.step(np.repeat(_rows([row]), len(codes), 0), F32, codes, temp=0.7)
+        assert (o.status == 0).all()
+        for c, tok, d, lo, p in zip(codes, o.tokens, o.d_tok, o.cdf_lo, o.p_tok):
+            i = int(c * n)                                   # position among the kept tokens
+            assert tok == kept[i] and p == 1.0 / n and lo == i / n
+            assert d == min(c - i / n, (i + 1) / n - c)
+
+
+def test_d_tok_against_the_decimal_cdf(orc):
+    # the same quantity on rows of unequal probabilities, against the CDF in 60-digit decimals,
+    # with temperature and both cuts
+    rng = np.random.default_rng(91)
+    for temp, k, tp in [(1.0, 0, 1.0), (0.6, 4, 1.0), (1.4, 0, 0.8), (0.9, 5, 0.7)]:
+        row = _rows([rng.normal(0, 2, 9)])
+        p = ex.conditional([float(v) for v in row[0]], temp, k, tp)
+        cdf = [Decimal(0)]
+        for x in p:
+            cdf.append(cdf[-1] + x)
+        codes = rng.random(300)
+        o = orc.step(np.repeat(row, len(codes), 0), F32, codes, temp=temp, top_k=k, top_p=tp)
+        checked = 0
+        for c, tok, d in zip(codes, o.tokens, o.d_tok):
+            cd = ex.D(c)
+            want = [j for j in range(9) if cdf[j] <= cd < cdf[j + 1]][0]
+            dist = min(cd - cdf[want], cdf[want + 1] - cd)
+            if dist < Decimal("1e-12"):
+                continue
+            checked += 1
+            assert tok == want
+            assert d == pytest.approx(float(dist), abs=1e-14)
+        assert checked > 290
+
+
+# --------------------------------------------------------------------------- encode under a cut, Sec. 4.1 with Sec. 5.1's top-k
+@pytest.mark.parametrize("kw", [{"top_k": 3}, {"top_p": 0.7, "temp": 1.2}, {"top_k": 4, "top_p": 0.8}])
+def test_encode_under_cuts_matches_the_enumerated_codebook(orc, kw):
+    # every sequence of the truncated model owns the interval the brute-force codebook gives it;
+    # a sequence with a token outside the kept set has probability zero: status NUMERIC, and the
+    # interval returned is that of the prefix before the offending token
+    V, T, start, eos = 6, 3, 2, 0
+    table = _tiny_model(V, seed=123)
+    book = _book(table, start, T, eos, **kw)
+    assert len(book) < V ** T                                  # the cut really removes sequences
+    seqs = np.full((len(book), T), -1, np.int32)
+    lens = np.zeros(len(book), np.int32)
+    for i, (s, _, _) in enumerate(book):
+        seqs[i, :len(s)] = s
+        lens[i] = len(s)
+    prev = np.full(len(book), start, np.int32)
+    lo, width, st = orc.encode_bigram(table, F32, prev, seqs, lens, **kw)
+    assert (st == 0).all()
+    for i, (_, l, w) in enumerate(book):
+        assert lo[i] == pytest.approx(float(l), abs=1e-14)
+        assert width[i] == pytest.approx(float(w), rel=1e-13)
+    # the intervals tile [0, 1) in dictionary order
+    order = np.argsort(lo, kind="stable")
+    np.testing.assert_allclose(lo[order][1:], (lo + width)[order][:-1], atol=1e-14)
+    assert (lo + width)[order][-1] == pytest.approx(1.0, abs=1e-14)
+    # sequences outside the truncated model
+    have = {s for s, _, _ in book}
+    bad = []
+    for a in range(V):
+        for b in range(V):
+            for c in range(V):
+                s = (a, b, c)
+                cut = s if eos not in s else s[:s.index(eos) + 1]
+                if cut not in have:
+                    bad.append(cut + (-1,) * (T - len(cut)))
+    bad = np.array(sorted(set(bad)), np.int32)
+    assert len(bad) > 0
+    blen = np.array([int((r >= 0).sum()) for r in bad], np.int32)
+    lo2, w2, st2 = orc.encode_bigram(table, F32, np.full(len(bad), start, np.int32), bad, blen, **kw)
+    assert (st2 == orc.ERR_NUMERIC).all()
+    pre = {}
+    for s, l, w in book:                                       # interval of a prefix = union of its sequences
+        for n in range(len(s) + 1):
+            a = pre.setdefault(s[:n], [l, Decimal(0)])
+            a[1] += w
+    for r, l, w in zip(bad, lo2, w2):
+        s = tuple(int(x) for x in r if x >= 0)
+        n = max(n for n in range(len(s)) if s[:n] in pre)      # longest prefix with positive probability
+        assert l == pytest.approx(float(pre[s[:n]][0]), abs=1e-14)
+        assert w == pytest.approx(float(pre[s[:n]][1]), rel=1e-12)

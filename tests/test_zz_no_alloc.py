@@ -5,7 +5,9 @@ Some users of this library get a stream from a host application but no right to 
 every stream of the device.  For them the library carries its own work buffer.  This test calls
 that entry point through the C ABI twice in a row (the buffer keeps the first call's contents,
 the second call must not be disturbed by them) and compares with as_step_host, which uses a
-caller-supplied buffer; it also checks that an oversized request is refused.  It is collected
+caller-supplied buffer -- the same kernel on the same bytes, so the results must be equal bit
+for bit; it checks that the device's free memory is the same before and after the calls, and
+that an oversized request is refused.  It is collected
 last so that a run stopping at the first failure has already run everything else."""
 import numpy as np
 import pytest
@@ -44,15 +46,24 @@ def test_static_work_buffer_matches_caller_buffer_twice(B):
         B.as_step_host(logits, codes, temp, k, p, tok, c, st, work)
         inputs.append((logits, codes))
         wanted.append((tok, c, st))
+    # a first call on this device (it looks up the buffer's address), then the measured ones
+    lanes, V, temp, k, p = cases[0]
+    warm = (torch.empty(lanes, dtype=torch.int32), torch.empty(lanes, dtype=torch.float64))
+    B.as_step_host_static(inputs[0][0], inputs[0][1], temp, k, p, warm[0], warm[1], None)
+    outs = [(torch.full((c[0],), -7, dtype=torch.int32), torch.full((c[0],), -7.0, dtype=torch.float64),
+             torch.full((c[0],), -7, dtype=torch.int32)) for c in cases]
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
     # two calls in a row on the built-in buffer: the second finds the first one's bytes in it
-    for (lanes, V, temp, k, p), (logits, codes), (want_tok, want_c, want_st) in zip(cases, inputs, wanted):
-        got_tok = torch.full((lanes,), -7, dtype=torch.int32)
-        got_c = torch.full((lanes,), -7.0, dtype=torch.float64)
-        got_st = torch.full((lanes,), -7, dtype=torch.int32)
+    for (lanes, V, temp, k, p), (logits, codes), (got_tok, got_c, got_st) in zip(cases, inputs, outs):
         B.as_step_host_static(logits, codes, temp, k, p, got_tok, got_c, got_st)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "as_step_host_static changed the device's free memory"
+    for (got_tok, got_c, got_st), (want_tok, want_c, want_st) in zip(outs, wanted):
         assert (got_st == 0).all() and torch.equal(got_st, want_st)
         assert torch.equal(got_tok, want_tok)
-        np.testing.assert_allclose(got_c.numpy(), want_c.numpy(), rtol=1e-6, atol=1e-12)
+        assert torch.equal(got_c, want_c)                  # same kernel, same bytes: bit for bit
 
 
 def test_static_work_buffer_refuses_what_does_not_fit(B):
