@@ -251,6 +251,44 @@ int as_decode_bigram_codes(const void *d_table, int dtype, int V, long long ld,
                            int32_t *d_lane_status, void *stream);
 
 /*
+ * Decoding with extended-precision codes.  Algorithm 1's update c <- (c - m)/(M - m) is real
+ * arithmetic; in fp64 every step spends -log2 p_i of the code's 53 bits, so after a few dozen
+ * tokens a lane is no longer steered by its lattice code and the properties of Sec. 4.3 / 4.4
+ * hold for a prefix only.  A lattice code (j + u)/N is a rational number, though, whose binary
+ * digits never run out: these two calls carry it as the state of an arithmetic decoder.
+ *
+ * Lane state: four 64-bit words [range, code, q, packed] -- the current interval has `range`
+ * units, in (2^62, 2^63]; `code` < range is the code's offset inside it; q and packed hold the
+ * source of the code's further digits (the unread part of its first 53 bits, their number in
+ * the upper half of packed, and in the lower half the remainder of the long division by N that
+ * yields every later digit).  Each step cuts the interval into 2^32 cells of range >> 32 units;
+ * with P_j the prefix sums (vocabulary-index order) of the kept tokens' masses under the same
+ * temperature / top-k / nucleus treatment as as_step and F(P) = floor(P * 2^32 / Z), token j owns
+ * the cells [F(P_j), F(P_{j+1})), the last token with mass ending at 2^32; the token whose cells
+ * hold the code is emitted, the interval becomes that token's, and digits are shifted in until
+ * range > 2^62 again.  All of it is integer arithmetic on cell boundaries that depend on the row
+ * alone: the sequences of a lattice are exactly those whose intervals in this subdivision hold
+ * the codes, at any length.  A token of probability below 2^-32 may own no cell.
+ *
+ * as_xp_lattice_state writes the state of the codes (j + u')/N, j = j0 .. j0+count-1, with
+ * u' = floor(u 2^53) / 2^53 (the shift read to 53 fractional bits), S times over:
+ *   d_state [S*count, 4] u64 device, lane = s*count + (j - j0)
+ * Errors: AS_ERR_INVALID_ARG (N < 1, u outside [0,1), j0 / count outside [0, N], S < 0, NULL).
+ *
+ * as_decode_bigram_xp runs Algorithm 1's loop (as as_decode_bigram_codes) from d_prev[lanes] and
+ * d_state[lanes, 4], which it updates in place, so that a decode can be split and resumed.
+ *   N   the lattice size the states were made for (it drives the digit source)
+ *   d_lane_status NULL or [lanes]: AS_OK, or AS_ERR_NUMERIC (unusable row, previous token
+ *       outside [0, V), state outside its domain); the lane stops there
+ * Errors: as as_decode_bigram_codes.
+ */
+int as_xp_lattice_state(int N, double u, int j0, int count, int S, uint64_t *d_state, void *stream);
+int as_decode_bigram_xp(const void *d_table, int dtype, int V, long long ld, const int32_t *d_prev,
+                        uint64_t *d_state, int lanes, int N, int T, int eos, double temp, int top_k,
+                        double top_p, int32_t *d_seq, int32_t *d_len, int32_t *d_lane_status,
+                        void *stream);
+
+/*
  * Sequence -> interval, the codebook of Sec. 4.1 read in the other direction:
  * in dictionary order every sequence owns the interval [lo, lo + P(sequence)),
  * and a code decodes to that sequence exactly when it falls inside.  For lane i

@@ -32,6 +32,13 @@
  *   orc_reward_mean       the sample-mean estimator (1/N) sum_i s(x_i) of Sec. 4.2
  *                         (Proposition on its unbiasedness) for an additive
  *                         reward s(x) = sum_t r[x_t].
+ *   orc_xp_*              Algorithm 1 with the code carried to unlimited precision:
+ *                         c <- (c - m)/(M - m) is real arithmetic in the paper, and a
+ *                         lattice code (j + u)/N is a rational whose binary digits never
+ *                         run out.  The step is that of an arithmetic decoder: the CDF of
+ *                         each step is quantised to 2^32 cells, the interval (m, M) of the
+ *                         chosen token becomes an integer sub-range, and further digits of
+ *                         the code are shifted in as the range narrows.
  *
  * Readings taken where the paper is silent (all also stated in the design
  * notes): intervals are half-open [F_{i-1}, F_i); order of modifiers is
@@ -101,30 +108,28 @@ typedef struct {
 } step_result;
 
 /*
- * One step for one lane (Algorithm 1, loop body).  row points at V stored
- * logits.  Work arrays l, e (V doubles), keep (V bytes), rk (V ranked) are
- * supplied by the caller.
+ * The modified next-token distribution of one row (steps 1-6 of the loop body of
+ * Algorithm 1 with the logit modifiers): on return keep[j] marks the kept tokens,
+ * e[j] holds their unnormalised masses exp(l_j/temp - max) (0 for the others) and
+ * *Z_out their sum in index order.  Work arrays l, e (V doubles), keep (V bytes),
+ * rk (V ranked) are supplied by the caller.  Returns ORC_OK or ORC_ERR_NUMERIC
+ * (NaN / +inf logit, no finite logit); fills n_kept, d_topp, tie_topk of `out`.
  */
-static void step_lane(const void *row, int dtype, long V, double c, double temp,
-                      long top_k, double top_p, double *l, double *e, char *keep,
-                      ranked *rk, step_result *out)
+static int kept_masses(const void *row, int dtype, long V, double temp, long top_k, double top_p,
+                       double *l, double *e, char *keep, ranked *rk, double *Z_out,
+                       step_result *out)
 {
     long j, nK = 0;
-    out->token = -1; out->code_out = c; out->p_tok = 0.0; out->cdf_lo = 0.0;
-    out->d_tok = 0.0; out->d_topp = INFINITY; out->n_kept = 0; out->tie_topk = 0;
-    out->status = ORC_ERR_NUMERIC;
-
-    if (!(c >= 0.0 && c <= 1.0)) return;          /* also rejects NaN */
-    if (c == 1.0) c = ORC_ONE_BELOW;              /* code domain is [0,1) */
+    out->d_topp = INFINITY; out->n_kept = 0; out->tie_topk = 0;
 
     /* 1-2: widen exactly; masked = -inf; NaN / +inf are errors */
     for (j = 0; j < V; ++j) {
         l[j] = load_logit(row, dtype, j);
-        if (isnan(l[j]) || l[j] == INFINITY) return;
+        if (isnan(l[j]) || l[j] == INFINITY) return ORC_ERR_NUMERIC;
         keep[j] = (l[j] > -INFINITY);
         nK += keep[j];
     }
-    if (nK == 0) return;
+    if (nK == 0) return ORC_ERR_NUMERIC;
 
     /* 3: top-k on the logits, order (value desc, index asc) */
     if (top_k > 0 && top_k < nK) {
@@ -160,7 +165,7 @@ static void step_lane(const void *row, int dtype, long V, double c, double temp,
             after = nsum_val(&run);
             if (after >= target) { cut = r + 1; break; }
         }
-        for (r = cut; r < n; ++r) keep[rk[r].idx] = 0;
+        for (r = cut; r < n; ++r) { keep[rk[r].idx] = 0; e[rk[r].idx] = 0.0; }
         if (cut < n || after >= target) {
             double a = fabs(target - before), b = fabs(after - target);
             out->d_topp = (a < b ? a : b) / Z1;
@@ -171,7 +176,32 @@ static void step_lane(const void *row, int dtype, long V, double c, double temp,
     /* 6: renormalise over the final kept set, summed in index order */
     nsum z = {0.0, 0.0};
     for (j = 0; j < V; ++j) if (keep[j]) nsum_add(&z, e[j]);
-    double Z = nsum_val(&z);
+    *Z_out = nsum_val(&z);
+    out->n_kept = (int32_t)nK;
+    return ORC_OK;
+}
+
+/*
+ * One step for one lane (Algorithm 1, loop body).  row points at V stored
+ * logits.  Work arrays as for kept_masses.
+ */
+static void step_lane(const void *row, int dtype, long V, double c, double temp,
+                      long top_k, double top_p, double *l, double *e, char *keep,
+                      ranked *rk, step_result *out)
+{
+    long j;
+    double Z;
+    out->token = -1; out->code_out = c; out->p_tok = 0.0; out->cdf_lo = 0.0;
+    out->d_tok = 0.0; out->d_topp = INFINITY; out->n_kept = 0; out->tie_topk = 0;
+    out->status = ORC_ERR_NUMERIC;
+
+    if (!(c >= 0.0 && c <= 1.0)) return;          /* also rejects NaN */
+    if (c == 1.0) c = ORC_ONE_BELOW;              /* code domain is [0,1) */
+
+    if (kept_masses(row, dtype, V, temp, top_k, top_p, l, e, keep, rk, &Z, out) != ORC_OK) {
+        out->n_kept = 0; out->d_topp = INFINITY; out->tie_topk = 0;
+        return;
+    }
 
     /* 7: first kept j (ascending index) with c*Z < S_j (inclusive prefix) */
     double t = c * Z, S_excl = 0.0;
@@ -200,7 +230,6 @@ static void step_lane(const void *row, int dtype, long V, double c, double temp,
     out->p_tok = e[chosen] / Z;
     out->cdf_lo = lo;
     out->d_tok = da < db ? da : db;
-    out->n_kept = (int32_t)nK;
     out->status = ORC_OK;
 }
 
@@ -530,4 +559,184 @@ int orc_reward_mean(const int32_t *seq, const int32_t *len, long S, long N, long
     return ORC_OK;
 }
 
-int orc_version(void) { return 1; }
+
+/* ------------------------------------------------------------------------------------------
+ * Extended-precision codes (Algorithm 1 in exact arithmetic).
+ *
+ * The code of lane j is the rational c = (j + u')/N with u' = floor(u 2^53)/2^53 (the shift
+ * read to 53 fractional bits).  With A = j 2^53 + floor(u 2^53), q0 = A div N, rem = A mod N:
+ *   c = q0 / 2^53 + (rem / N) / 2^53,
+ * so its binary digits are the 53 bits of q0 followed by the digits of rem/N, which long
+ * division produces one at a time for ever.
+ *
+ * Lane state, four 64-bit words:
+ *   [0] range   the current interval has `range` units; (2^62, 2^63] after every step
+ *   [1] code    the code's offset inside it, in the same units, < range
+ *   [2] q       the bits of q0 not yet shifted in (right-aligned)
+ *   [3] (nq << 32) | rem    how many those are, and the long-division remainder
+ * One step: r = range >> 32 is the size of one of 2^32 cells; the code lies in cell
+ * t = min(code div r, 2^32 - 1).  With P_0 = 0 <= P_1 <= ... the prefix sums of the kept masses
+ * in index order and F(P) = floor(P * (2^32 / Z)) (F of the last one := 2^32), token j owns
+ * the cells [F(P_j), F(P_{j+1})): the token is the first kept j with F(P_{j+1}) > t; then
+ * code -= r F(P_j), range = r (F(P_{j+1}) - F(P_j)) -- the last kept token also takes the
+ * range mod 2^32 units left over -- and digits of c are shifted in until range > 2^62 again.
+ * All of this is integer arithmetic: the decoded sequence is exactly the one whose interval
+ * in this nested subdivision holds c.
+ * ------------------------------------------------------------------------------------------ */
+#define XP_CELLS 4294967296.0          /* 2^32 */
+#define XP_RANGE_TOP (1ull << 63)
+#define XP_RANGE_LOW (1ull << 62)
+
+static uint64_t xp_next_bit(uint64_t *st, uint64_t N)
+{
+    uint64_t nq = st[3] >> 32, rem = st[3] & 0xFFFFFFFFull, bit;
+    if (nq > 0) {
+        --nq;
+        bit = (st[2] >> nq) & 1ull;
+        st[2] &= (nq ? ((1ull << nq) - 1ull) : 0ull);
+    } else {
+        rem <<= 1;
+        bit = rem >= N;
+        if (bit) rem -= N;
+    }
+    st[3] = (nq << 32) | rem;
+    return bit;
+}
+
+/* state of the lattice codes (j + u)/N for j = j0 .. j0 + count - 1, written S times over
+ * (one copy per start token: lane = s*count + (j - j0)) */
+int orc_xp_lattice_state(long N, double u, long j0, long count, long S, uint64_t *state)
+{
+    long i, s, k;
+    if (N < 1 || N > 0x7FFFFFFFL || S < 0 || j0 < 0 || count < 0 || j0 + count > N || !state ||
+        !(u >= 0.0 && u < 1.0))
+        return ORC_ERR_INVALID_ARG;
+    uint64_t U = (uint64_t)floor(u * 9007199254740992.0);            /* floor(u 2^53), exact */
+    for (i = 0; i < count; ++i) {
+        unsigned __int128 A = ((unsigned __int128)(uint64_t)(j0 + i) << 53) + U;
+        uint64_t st[4];
+        st[0] = XP_RANGE_TOP;
+        st[1] = 0;
+        st[2] = (uint64_t)(A / (uint64_t)N);
+        st[3] = ((uint64_t)53 << 32) | (uint64_t)(A % (uint64_t)N);
+        for (k = 0; k < 63; ++k) st[1] = (st[1] << 1) | xp_next_bit(st, (uint64_t)N);
+        for (s = 0; s < S; ++s) memcpy(state + ((size_t)s * (size_t)count + (size_t)i) * 4, st, sizeof st);
+    }
+    return ORC_OK;
+}
+
+/* cell boundaries of one row: cells[j] = F(P_j) for j = 0..V, cells[V] = 2^32; a token that is
+ * not kept owns no cell (cells[j+1] == cells[j]).  Returns the status of the row. */
+static int xp_row_cells(const void *row, int dtype, long V, double temp, long top_k, double top_p,
+                        workspace *w, uint64_t *cells, step_result *info)
+{
+    long j, last = -1;
+    double Z;
+    int rc = kept_masses(row, dtype, V, temp, top_k, top_p, w->l, w->e, w->keep, w->rk, &Z, info);
+    if (rc != ORC_OK) return rc;
+    const double K = XP_CELLS / Z;
+    nsum run = {0.0, 0.0};
+    cells[0] = 0;
+    for (j = 0; j < V; ++j) {
+        if (w->keep[j]) {
+            nsum_add(&run, w->e[j]);
+            double f = nsum_val(&run) * K;
+            uint64_t F = f >= XP_CELLS ? 0x100000000ull : (uint64_t)f;
+            if (F < cells[j]) F = cells[j];            /* (the sums are non-decreasing; kept for safety) */
+            cells[j + 1] = F;
+            last = j;
+        } else {
+            cells[j + 1] = cells[j];
+        }
+    }
+    for (j = last; j < V; ++j) cells[j + 1] = 0x100000000ull;   /* the last kept token ends at 2^32 */
+    return ORC_OK;
+}
+
+int orc_xp_row_cells(const void *row, int dtype, long V, double temp, long top_k, double top_p,
+                     uint64_t *cells)
+{
+    workspace w;
+    step_result info;
+    if (!row || !cells || !check_params(V, temp, top_k, top_p)) return ORC_ERR_INVALID_ARG;
+    if (!ws_alloc(&w, V)) { ws_free(&w); return ORC_ERR_INVALID_ARG; }
+    int rc = xp_row_cells(row, dtype, V, temp, top_k, top_p, &w, cells, &info);
+    ws_free(&w);
+    return rc;
+}
+
+/*
+ * Algorithm 1's loop with extended-precision codes over a bigram model, lanes
+ * [lane_begin, lane_end): lane i starts from previous token prev[i] and state[4 i .. 4 i + 3]
+ * (updated in place, so a decode can be split and resumed).  seq, len, status as for
+ * orc_decode_bigram_codes.  Optional traces, each [lanes, T]: the position of the code inside
+ * the step's distribution, (code / r) / 2^32, and its distance to the nearest end of the
+ * chosen token's cell range, both before the step.
+ */
+int orc_xp_decode_bigram(const void *table, int dtype, long V, long ld, const int32_t *prev,
+                         uint64_t *state, long lanes, long N, long T, long eos, double temp,
+                         long top_k, double top_p, int32_t *seq, int32_t *len, int32_t *status,
+                         double *trace_pos, double *trace_d_tok, long lane_begin, long lane_end)
+{
+    workspace w;
+    long i, t, j;
+    size_t esz = dtype == ORC_BF16 ? 2 : 4;
+    if (!table || !prev || !state || !seq || lanes < 0 || T < 0 || ld < V || N < 1 || N > 0x7FFFFFFFL ||
+        !check_params(V, temp, top_k, top_p))
+        return ORC_ERR_INVALID_ARG;
+    if (dtype != ORC_F32 && dtype != ORC_BF16) return ORC_ERR_INVALID_ARG;
+    if (lane_begin < 0 || lane_end > lanes) return ORC_ERR_INVALID_ARG;
+    if (!ws_alloc(&w, V)) { ws_free(&w); return ORC_ERR_INVALID_ARG; }
+    uint64_t *cells = (uint64_t *)malloc(sizeof(uint64_t) * (size_t)(V + 1));
+    if (!cells) { ws_free(&w); return ORC_ERR_INVALID_ARG; }
+    for (i = lane_begin; i < lane_end; ++i) {
+        uint64_t *st = state + (size_t)i * 4;
+        long p = prev[i], n = 0;
+        int32_t rc = ORC_OK;
+        for (t = 0; t < T; ++t) {
+            seq[i * T + t] = -1;
+            if (trace_pos) trace_pos[i * T + t] = NAN;
+            if (trace_d_tok) trace_d_tok[i * T + t] = NAN;
+        }
+        for (t = 0; t < T; ++t) {
+            step_result info;
+            if (p < 0 || p >= V || st[0] <= XP_RANGE_LOW || st[0] > XP_RANGE_TOP || st[1] >= st[0]) {
+                rc = ORC_ERR_NUMERIC;
+                break;
+            }
+            const char *row = (const char *)table + (size_t)p * (size_t)ld * esz;
+            rc = xp_row_cells(row, dtype, V, temp, top_k, top_p, &w, cells, &info);
+            if (rc != ORC_OK) break;
+            const uint64_t r = st[0] >> 32;
+            uint64_t tcell = st[1] / r;
+            if (tcell > 0xFFFFFFFFull) tcell = 0xFFFFFFFFull;
+            long tok = -1;
+            for (j = 0; j < V; ++j) if (cells[j + 1] > tcell) { tok = j; break; }
+            /* (cells[V] = 2^32 > tcell: a token is always found) */
+            const uint64_t lo = cells[tok], hi = cells[tok + 1];
+            if (trace_pos || trace_d_tok) {
+                double pos = ((double)st[1] / (double)r) / XP_CELLS;
+                double a = pos - (double)lo / XP_CELLS, b = (double)hi / XP_CELLS - pos;
+                if (trace_pos) trace_pos[i * T + t] = pos;
+                if (trace_d_tok) trace_d_tok[i * T + t] = a < b ? a : b;
+            }
+            st[1] -= r * lo;
+            st[0] = hi == 0x100000000ull ? st[0] - r * lo : r * (hi - lo);
+            while (st[0] <= XP_RANGE_LOW) {
+                st[0] <<= 1;
+                st[1] = (st[1] << 1) | xp_next_bit(st, (uint64_t)N);
+            }
+            seq[i * T + t] = (int32_t)tok;
+            n = t + 1;
+            p = tok;
+            if (tok == eos) break;
+        }
+        if (len) len[i] = (int32_t)n;
+        if (status) status[i] = rc;
+    }
+    free(cells);
+    ws_free(&w);
+    return ORC_OK;
+}
+
+int orc_version(void) { return 2; }

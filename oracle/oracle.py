@@ -57,6 +57,11 @@ def lib():
         _lib.orc_lattice_codes_variant.restype = ctypes.c_int
         _lib.orc_ngram_diversity.argtypes = [P, P, L, L, L, P, P, P]
         _lib.orc_reward_mean.argtypes = [P, P, L, L, L, P, L, P, P]
+        _lib.orc_xp_lattice_state.argtypes = [L, D, L, L, L, P]
+        _lib.orc_xp_row_cells.argtypes = [P, ctypes.c_int, L, D, L, D, P]
+        _lib.orc_xp_decode_bigram.argtypes = [P, ctypes.c_int, L, L, P, P, L, L, L, L, D, L, D, P, P, P, P, P, L, L]
+        for f in (_lib.orc_xp_lattice_state, _lib.orc_xp_row_cells, _lib.orc_xp_decode_bigram):
+            f.restype = ctypes.c_int
         for f in (_lib.orc_lattice_codes, _lib.orc_step, _lib.orc_decode_bigram_codes,
                   _lib.orc_decode_bigram, _lib.orc_encode_bigram, _lib.orc_ngram_diversity,
                   _lib.orc_reward_mean, _lib.orc_version):
@@ -266,3 +271,62 @@ def reward_mean(seq: np.ndarray, length: np.ndarray, N: int, r: np.ndarray):
     if rc != OK:
         raise ValueError("orc_reward_mean returned %d" % rc)
     return lane_reward, mean
+
+
+# ----------------------------------------------------------------------------- extended-precision codes
+def xp_lattice_state(N: int, u: float, S: int = 1, j0: int = 0, count: Optional[int] = None) -> np.ndarray:
+    """uint64 [S*count, 4]: decoder state of the lattice codes (j + floor(u 2^53)/2^53)/N for
+    j = j0 .. j0+count-1 (default: all N), one copy per start token."""
+    count = N - j0 if count is None else count
+    out = np.zeros((max(S, 0) * max(count, 0), 4), dtype=np.uint64)
+    rc = lib().orc_xp_lattice_state(N, u, j0, count, S, _ptr(out))
+    if rc != OK:
+        raise ValueError("orc_xp_lattice_state: invalid argument")
+    return out
+
+
+def xp_row_cells(row: np.ndarray, dtype: int, temp: float = 1.0, top_k: int = 0, top_p: float = 1.0) -> np.ndarray:
+    """uint64 [V+1]: the 2^32-cell boundaries F(P_j) of one row's modified distribution."""
+    row = np.ascontiguousarray(row)
+    V = row.shape[0]
+    cells = np.zeros(V + 1, dtype=np.uint64)
+    rc = lib().orc_xp_row_cells(_ptr(row), dtype, V, temp, top_k, top_p, _ptr(cells))
+    if rc != OK:
+        raise ValueError("orc_xp_row_cells returned %d" % rc)
+    return cells
+
+
+@dataclass
+class XpDecodeOut:
+    seq: np.ndarray
+    len: np.ndarray
+    status: np.ndarray
+    state: np.ndarray
+    trace_pos: Optional[np.ndarray] = None
+    trace_d_tok: Optional[np.ndarray] = None
+
+
+def xp_decode_bigram(table: np.ndarray, dtype: int, prev: np.ndarray, state: np.ndarray, N: int, T: int, eos: int,
+                     temp: float = 1.0, top_k: int = 0, top_p: float = 1.0, V: Optional[int] = None,
+                     trace: bool = False, threads: int = 1) -> XpDecodeOut:
+    """Algorithm 1's loop with extended-precision codes; `state` [lanes, 4] uint64 is not modified
+    (the updated copy is returned)."""
+    table = _check_logits(table, dtype)
+    ld = table.shape[1]
+    V = ld if V is None else V
+    prev = np.ascontiguousarray(prev, dtype=np.int32)
+    state = np.array(state, dtype=np.uint64, copy=True)
+    lanes = prev.shape[0]
+    if state.shape != (lanes, 4):
+        raise ValueError("state must be [lanes, 4] uint64")
+    o = XpDecodeOut(np.empty((lanes, T), np.int32), np.empty(lanes, np.int32), np.empty(lanes, np.int32), state)
+    if trace:
+        o.trace_pos = np.empty((lanes, T), np.float64)
+        o.trace_d_tok = np.empty((lanes, T), np.float64)
+
+    def run(a, b):
+        return lib().orc_xp_decode_bigram(_ptr(table), dtype, V, ld, _ptr(prev), _ptr(state), lanes, N, T, eos, temp,
+                                          top_k, top_p, _ptr(o.seq), _ptr(o.len), _ptr(o.status),
+                                          _ptr(o.trace_pos), _ptr(o.trace_d_tok), a, b)
+    _run_ranges(run, lanes, threads)
+    return o

@@ -39,7 +39,7 @@ TUNE_DEBUG_NO_COPY = 8
 
 EXPORTS = ["as_lattice_codes", "as_lattice_codes_variant", "as_step", "as_step_lattice", "as_step_host", "as_step_host_work_bytes", "as_step_host_static",
            "as_decode_bigram",
-           "as_decode_bigram_codes", "as_encode_bigram", "as_ngram_diversity", "as_reward_mean", "as_tune",
+           "as_decode_bigram_codes", "as_xp_lattice_state", "as_decode_bigram_xp", "as_encode_bigram", "as_ngram_diversity", "as_reward_mean", "as_tune",
            "as_last_error", "as_version"]
 
 
@@ -88,10 +88,14 @@ def lib():
         L.as_lattice_codes_variant.restype = I
         L.as_ngram_diversity.argtypes = [P, P, I, I, I, P, P, P, P]
         L.as_reward_mean.argtypes = [P, P, I, I, I, P, I, P, P, P, P]
+        L.as_xp_lattice_state.argtypes = [I, D, I, I, I, P, P]
+        L.as_xp_lattice_state.restype = I
+        L.as_decode_bigram_xp.argtypes = [P, I, I, LL, P, P, I, I, I, I, D, I, D, P, P, P, P]
+        L.as_decode_bigram_xp.restype = I
         L.as_tune.argtypes = [I, I]
         L.as_last_error.restype = ctypes.c_char_p
         for n in ("as_lattice_codes", "as_step", "as_step_host", "as_decode_bigram",
-                  "as_decode_bigram_codes", "as_encode_bigram", "as_ngram_diversity", "as_reward_mean", "as_tune",
+                  "as_decode_bigram_codes", "as_xp_lattice_state", "as_decode_bigram_xp", "as_encode_bigram", "as_ngram_diversity", "as_reward_mean", "as_tune",
                   "as_version"):
             getattr(L, n).restype = I
         _lib = L
@@ -277,6 +281,40 @@ def as_decode_bigram_codes(table: torch.Tensor, prev: torch.Tensor, codes_in: to
     _check(lib().as_decode_bigram_codes(_ptr(table), _logits_dtype(table), V, ld, _ptr(prev), _ptr(codes_in),
                                         lanes, T, eos, temp, top_k, top_p, _ptr(seq), _ptr(length),
                                         _ptr(codes_final), _ptr(lane_status), _stream(stream)))
+    return seq, length
+
+
+def as_xp_lattice_state(N: int, u: float, j0: int = 0, count: Optional[int] = None, S: int = 1,
+                        out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """int64 [S*count, 4] (the bits of four unsigned 64-bit words per lane): decoder state of the
+    lattice codes (j + u)/N, j = j0 .. j0+count-1, one copy per start token."""
+    count = N - j0 if count is None else count
+    if out is None:
+        out = torch.empty((max(S, 0) * max(count, 0), 4), dtype=torch.int64, device="cuda")
+    _check(lib().as_xp_lattice_state(N, u, j0, count, S, _ptr(out), _stream(stream)))
+    return out
+
+
+def as_decode_bigram_xp(table: torch.Tensor, prev: torch.Tensor, state: torch.Tensor, N: int, T: int, eos: int,
+                        temp: float = 1.0, top_k: int = 0, top_p: float = 1.0, V: Optional[int] = None,
+                        lane_status: Optional[torch.Tensor] = None, seq: Optional[torch.Tensor] = None,
+                        length: Optional[torch.Tensor] = None, stream=None):
+    """Algorithm 1's loop with extended-precision codes; `state` [lanes, 4] int64 is updated in place."""
+    rows, width, ld = _logits_layout(table)
+    V = width if V is None else V
+    if rows < V:
+        raise ValueError("bigram table needs at least V rows")
+    lanes = prev.numel()
+    if state.dtype != torch.int64 or state.numel() != 4 * lanes or not state.is_contiguous():
+        raise ValueError("state must be a contiguous [lanes, 4] int64 tensor")
+    dev = table.device
+    if seq is None:
+        seq = torch.empty((lanes, T), dtype=torch.int32, device=dev)
+    if length is None:
+        length = torch.empty(lanes, dtype=torch.int32, device=dev)
+    _check(lib().as_decode_bigram_xp(_ptr(table), _logits_dtype(table), V, ld, _ptr(prev), _ptr(state), lanes, N, T,
+                                     eos, temp, top_k, top_p, _ptr(seq), _ptr(length), _ptr(lane_status),
+                                     _stream(stream)))
     return seq, length
 
 

@@ -1,6 +1,7 @@
 // C-ABI entry points (see include/arith_sampling.h) and the kernels behind them.
 #include "../../include/arith_sampling.h"
 #include "as_stream.cuh"
+#include "as_nocut.cuh"
 #include "as_metrics.cuh"
 
 #include <atomic>
@@ -187,6 +188,45 @@ static int launch_staged_cs(int cs, const StepArgs& a, size_t smem, int sms, int
     }
 }
 
+// Lanes without a cut on 16-byte aligned rows of up to 96 KB: groups of 256 threads, each with a
+// row buffer in shared memory (as_nocut.cuh).  AS_ERR_UNSUPPORTED (no message): not for that kernel.
+template <int DT, int MODE>
+static int launch_nocut_dm(NocutArgs& a, double temp, int sms, cudaStream_t st) {
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    auto kern = nocut_kernel<DT, MODE>;
+    cudaError_t e;
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_OPTIN_MAX - 1024));
+        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(max dynamic shared memory)");
+        attr_set[dev] = true;
+    }
+    const size_t row_stride = (((size_t)a.V * Traits<DT>::BYTES) + 127) & ~(size_t)127;
+    int groups = (int)((SMEM_OPTIN_MAX - 1024 - nc_fixed_bytes()) / row_stride);
+    if (groups > NC_MAXG) groups = NC_MAXG;
+    if (groups < 1) return AS_ERR_UNSUPPORTED;
+    a.use_table = (DT == DT_BF16 && temp >= NC_MIN_TEMP) ? 1 : 0;
+    a.wait_cycles = wait_cycles_now();
+    a.debug_no_copy = g_tune_no_copy;
+    long long grid = ((long long)a.lanes + groups - 1) / groups;
+    if (grid > sms) grid = sms;
+    const size_t smem = nc_fixed_bytes() + (size_t)groups * row_stride;
+    kern<<<(unsigned)grid, groups * NC_GT, smem, st>>>(a, groups, (int)row_stride);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "no-cut kernel launch");
+    return AS_OK;
+}
+
+template <int MODE>
+static int launch_nocut(NocutArgs& a, int dtype, double temp, int sms, cudaStream_t st) {
+    const size_t esz = dtype == AS_F32 ? 4 : 2;
+    if (g_tune_path != 0) return AS_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(a.data) & 15) != 0 || (((size_t)a.ld * esz) & 15) != 0) return AS_ERR_UNSUPPORTED;
+    if ((size_t)a.V * esz > (size_t)NC_MAXROW) return AS_ERR_UNSUPPORTED;
+    return dtype == AS_F32 ? launch_nocut_dm<DT_F32, MODE>(a, temp, sms, st) : launch_nocut_dm<DT_BF16, MODE>(a, temp, sms, st);
+}
+
 // ---------------------------------------------------------------------------
 // kernels
 // ---------------------------------------------------------------------------
@@ -324,6 +364,64 @@ encode_generic_kernel(const void* __restrict__ table, int V, long long ld, const
         if (threadIdx.x == 0) {
             lo_out[ln] = lo + comp;
             width_out[ln] = width;
+            if (lane_status) lane_status[ln] = status;
+        }
+    }
+}
+
+// Extended-precision codes: decoder state of the lattice codes (j + u)/N, j = j0 .. j0 + count - 1,
+// one copy per start token.  U = floor(u 2^53); A = j 2^53 + U; the first 53 binary digits of the
+// code are A div N, all further ones come from the long division of A mod N by N.
+__global__ void xp_state_kernel(int N, unsigned long long U, int j0, int count, int S, unsigned long long* __restrict__ state) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= count) return;
+    const unsigned __int128 A = ((unsigned __int128)(unsigned long long)(j0 + i) << 53) + U;
+    XpState s;
+    s.range = XP_RANGE_TOP;
+    s.code = 0;
+    s.q = (unsigned long long)(A / (unsigned long long)N);
+    s.packed = (53ull << 32) | (unsigned long long)(A % (unsigned long long)N);
+    s.code = xp_next_bits(s, 32, (unsigned)N);
+    s.code = (s.code << 31) | xp_next_bits(s, 31, (unsigned)N);
+    for (int g = 0; g < S; ++g) {
+        unsigned long long* o = state + ((size_t)g * count + i) * 4;
+        o[0] = s.range; o[1] = s.code; o[2] = s.q; o[3] = s.packed;
+    }
+}
+
+// Algorithm 1's loop with extended-precision codes, one CTA per lane, any cut (general routine).
+template <int DT>
+__global__ void __launch_bounds__(GEN_NT)
+decode_xp_generic_kernel(const void* __restrict__ table, int V, long long ld, const int* __restrict__ prev_in,
+                         unsigned long long* __restrict__ state, int lanes, int N, int T, int eos, double inv_tau,
+                         int top_k, double top_p, int* __restrict__ seq, int* __restrict__ len,
+                         int* __restrict__ lane_status) {
+    __shared__ GenericSmem<GEN_NT> sm;
+    for (int ln = blockIdx.x; ln < lanes; ln += gridDim.x) {
+        XpState xs;
+        xs.range = state[(size_t)ln * 4]; xs.code = state[(size_t)ln * 4 + 1];
+        xs.q = state[(size_t)ln * 4 + 2]; xs.packed = state[(size_t)ln * 4 + 3];
+        int prev = prev_in[ln];
+        int n = 0, status = ST_OK;
+        for (int t = 0; t < T; ++t) {
+            if (prev < 0 || prev >= V || !xp_state_ok(xs)) { status = ST_NUMERIC; break; }
+            const char* row = reinterpret_cast<const char*>(table) + (size_t)prev * (size_t)ld * Traits<DT>::BYTES;
+            const bool vec_ok = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
+            GenericLane<DT, GEN_NT> g(sm, row, V, vec_ok);
+            const LaneResult r = g.run_xp(xp_target(xs), inv_tau, top_k, top_p);
+            if (r.status != ST_OK) { status = r.status; break; }
+            xp_advance(xs, r.xp_lo, r.xp_hi, (unsigned)N);
+            if (threadIdx.x == 0) seq[(size_t)ln * T + t] = r.token;
+            n = t + 1;
+            prev = r.token;
+            if (r.token == eos) break;
+        }
+        for (int t = n + (int)threadIdx.x; t < T; t += GEN_NT) seq[(size_t)ln * T + t] = -1;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            len[ln] = n;
+            state[(size_t)ln * 4] = xs.range; state[(size_t)ln * 4 + 1] = xs.code;
+            state[(size_t)ln * 4 + 2] = xs.q; state[(size_t)ln * 4 + 3] = xs.packed;
             if (lane_status) lane_status[ln] = status;
         }
     }
@@ -552,6 +650,14 @@ static int step_common(const void* d_logits, int dtype, int lanes, int V, long l
         rc = launch_streaming(a, dtype, unaligned, di->sms, st);
         if (rc != AS_ERR_UNSUPPORTED) return rc;
     }
+    if (top_k == 0 && !(top_p < 1.0)) {
+        NocutArgs n = {};
+        n.data = d_logits; n.ld = ld; n.V = V; n.lanes = lanes; n.inv_tau = inv_tau;
+        n.codes = d_codes; n.lat_N = lat_N; n.lat_j0 = lat_j0; n.lat_u = lat_u;
+        n.tokens = d_tokens; n.codes_out = d_codes_out; n.diag = dp;
+        rc = launch_nocut<NC_STEP>(n, dtype, temp, di->sms, st);
+        if (rc != AS_ERR_UNSUPPORTED) return rc;
+    }
     if (g_tune_path == 2) {
         // cluster kernel: the row split over CS CTAs' shared memory
         int cs = g_tune_cluster;
@@ -755,6 +861,14 @@ static int decode_common(const void* d_table, int dtype, int V, long long ld, co
             return AS_OK;
         }
     }
+    if (top_k == 0 && !(top_p < 1.0)) {
+        NocutArgs n = {};
+        n.data = d_table; n.ld = ld; n.V = V; n.lanes = lanes; n.inv_tau = inv_tau;
+        n.tok_in = d_tok; n.codes_in = d_codes_in; n.N = N; n.u = u; n.T = T; n.eos = eos;
+        n.seq = d_seq; n.len = d_len; n.codes_final = d_codes_final; n.lane_status = d_lane_status;
+        rc = launch_nocut<NC_DECODE>(n, dtype, temp, di->sms, st);
+        if (rc != AS_ERR_UNSUPPORTED) return rc;
+    }
     const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
     if (dtype == AS_F32)
         decode_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_table, V, ld, d_tok, d_codes_in, lanes, N, u, T, eos, inv_tau, top_k, top_p, d_seq, d_len, d_codes_final, d_lane_status);
@@ -805,8 +919,16 @@ int as_encode_bigram(const void* d_table, int dtype, int V, long long ld, const 
     if (top_k < 0 || top_k >= V) top_k = 0;
     if (!(top_p > 0.0 && top_p < 1.0)) top_p = 1.0;
     const double inv_tau = 1.0 / temp;
-    const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
     cudaStream_t st = (cudaStream_t)stream;
+    if (top_k == 0 && !(top_p < 1.0)) {
+        NocutArgs n = {};
+        n.data = d_table; n.ld = ld; n.V = V; n.lanes = lanes; n.inv_tau = inv_tau;
+        n.tok_in = d_prev; n.seq_in = d_seq; n.len_in = d_len; n.T = T;
+        n.lo_out = d_lo; n.width_out = d_width; n.lane_status = d_lane_status;
+        rc = launch_nocut<NC_ENCODE>(n, dtype, temp, di->sms, st);
+        if (rc != AS_ERR_UNSUPPORTED) return rc;
+    }
+    const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
     if (dtype == AS_F32)
         encode_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_table, V, ld, d_prev, d_seq, d_len, lanes, T, inv_tau, top_k, top_p, d_lo, d_width, d_lane_status);
     else
@@ -869,6 +991,63 @@ int as_reward_mean(const int32_t* d_seq, const int32_t* d_len, int S, int N, int
         d_seq, d_len, S, N, T, d_r, V, d_lane_reward, d_mean, d_group_status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "reward mean kernel launch");
+    return AS_OK;
+}
+
+int as_xp_lattice_state(int N, double u, int j0, int count, int S, uint64_t* d_state, void* stream) {
+    if (N < 1) return set_err(AS_ERR_INVALID_ARG, "N = %d must be >= 1", N);
+    if (!(u >= 0.0 && u < 1.0)) return set_err(AS_ERR_INVALID_ARG, "shift u must lie in [0,1)");
+    if (j0 < 0 || count < 0 || (long long)j0 + count > N)
+        return set_err(AS_ERR_INVALID_ARG, "codes j0 .. j0+count-1 must lie in [0, N = %d)", N);
+    if (S < 0) return set_err(AS_ERR_INVALID_ARG, "S = %d must be >= 0", S);
+    if (count == 0 || S == 0) return AS_OK;
+    if (!d_state) return set_err(AS_ERR_INVALID_ARG, "d_state is NULL");
+    const DeviceInfo* di;
+    int rc = device_info(&di);
+    if (rc != AS_OK) return rc;
+    const unsigned long long U = (unsigned long long)std::floor(u * 9007199254740992.0);   // floor(u 2^53), exact
+    xp_state_kernel<<<(count + 127) / 128, 128, 0, (cudaStream_t)stream>>>(N, U, j0, count, S,
+                                                                            reinterpret_cast<unsigned long long*>(d_state));
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "extended-precision state kernel launch");
+    return AS_OK;
+}
+
+int as_decode_bigram_xp(const void* d_table, int dtype, int V, long long ld, const int32_t* d_prev,
+                        uint64_t* d_state, int lanes, int N, int T, int eos, double temp, int top_k,
+                        double top_p, int32_t* d_seq, int32_t* d_len, int32_t* d_lane_status, void* stream) {
+    if (lanes < 0) return set_err(AS_ERR_INVALID_ARG, "lanes = %d must be >= 0", lanes);
+    if (N < 1) return set_err(AS_ERR_INVALID_ARG, "N = %d must be >= 1", N);
+    if (T < 0) return set_err(AS_ERR_INVALID_ARG, "T = %d must be >= 0", T);
+    int rc = check_scalars(dtype, V, ld, temp, top_p);
+    if (rc != AS_OK) return rc;
+    if (lanes == 0) return AS_OK;
+    if ((rc = check_data(d_table, dtype)) != AS_OK) return rc;
+    if (!d_prev || !d_state || !d_len || (!d_seq && T > 0))
+        return set_err(AS_ERR_INVALID_ARG, "d_prev, d_state, d_seq or d_len is NULL");
+    const DeviceInfo* di;
+    rc = device_info(&di);
+    if (rc != AS_OK) return rc;
+    if (top_k < 0 || top_k >= V) top_k = 0;
+    if (!(top_p > 0.0 && top_p < 1.0)) top_p = 1.0;
+    const double inv_tau = 1.0 / temp;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned long long* state = reinterpret_cast<unsigned long long*>(d_state);
+    if (top_k == 0 && !(top_p < 1.0)) {
+        NocutArgs n = {};
+        n.data = d_table; n.ld = ld; n.V = V; n.lanes = lanes; n.inv_tau = inv_tau;
+        n.tok_in = d_prev; n.N = N; n.T = T; n.eos = eos;
+        n.seq = d_seq; n.len = d_len; n.lane_status = d_lane_status; n.xp_state = state;
+        rc = launch_nocut<NC_DECODE_XP>(n, dtype, temp, di->sms, st);
+        if (rc != AS_ERR_UNSUPPORTED) return rc;
+    }
+    const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
+    if (dtype == AS_F32)
+        decode_xp_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_table, V, ld, d_prev, state, lanes, N, T, eos, inv_tau, top_k, top_p, d_seq, d_len, d_lane_status);
+    else
+        decode_xp_generic_kernel<DT_BF16><<<grid, GEN_NT, 0, st>>>(d_table, V, ld, d_prev, state, lanes, N, T, eos, inv_tau, top_k, top_p, d_seq, d_len, d_lane_status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "extended-precision decode kernel launch");
     return AS_OK;
 }
 

@@ -94,8 +94,8 @@ __device__ __forceinline__ void load_vec_keys(const void* row, int V, int vi, bo
 // exp(y) = 2^n * 2^(j/64) * exp(f), exp(f) by a degree-5 polynomial
 // (truncation ~3e-17).  tbl[j] = 2^(j/64).  Arguments below -700 return 0.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ double exp_nonpos(double y, const double* __restrict__ tbl) {
-    if (!(y >= -700.0)) return 0.0;
+// exp(y) for |y| <= 700 or so (no range check: the result's exponent is formed by integer addition)
+__device__ __forceinline__ double exp_core(double y, const double* __restrict__ tbl) {
     const double MAGIC = 6755399441055744.0;          // 1.5 * 2^52: rounds to integer
     double r = fma(y, 0x1.71547652b82fep+6, MAGIC);    // y * 64/ln2
     const int k = __double2loint(r);
@@ -108,8 +108,12 @@ __device__ __forceinline__ double exp_nonpos(double y, const double* __restrict_
     p = fma(p, f, 1.0);
     p = fma(p, f, 1.0);
     const double v = tbl[k & 63] * p;
-    const int n = k >> 6;                              // floor((64n+j)/64), n in [-1010, 0]
+    const int n = k >> 6;                              // floor((64n+j)/64)
     return __hiloint2double(__double2hiint(v) + (n << 20), __double2loint(v));
+}
+__device__ __forceinline__ double exp_nonpos(double y, const double* __restrict__ tbl) {
+    if (!(y >= -700.0)) return 0.0;
+    return exp_core(y, tbl);
 }
 
 // 2^(j/64), j = 0..63, correctly rounded.
@@ -321,6 +325,127 @@ template <> struct Pass<DT_F32> {
     }
 };
 
+// ---------------------------------------------------------------------------
+// Extended-precision codes: Algorithm 1's c <- (c - m)/(M - m) in exact arithmetic, as the
+// step of an arithmetic decoder.  A lane's state is four 64-bit words: the current interval
+// has `range` units, in (2^62, 2^63]; `code` < range is the code's offset in it; `q` holds the
+// not yet consumed bits of the code's first 53 binary digits, `packed` = (their number << 32)
+// | the remainder of the long division that yields all further digits of the rational code
+// (j + u)/N.  One step cuts the interval into 2^32 cells of r = range >> 32 units; the cell
+// t = min(code / r, 2^32 - 1) holds the code; token j owns the cells [F(P_j), F(P_{j+1})) with
+// P the prefix sums of the kept masses in index order and F(P) = floor(P * 2^32 / Z), the last
+// token with mass ending at 2^32 (it also takes the range mod 2^32 units left over).
+// ---------------------------------------------------------------------------
+constexpr unsigned long long XP_TOP = 0x100000000ull;           // 2^32 cells
+constexpr unsigned long long XP_RANGE_TOP = 1ull << 63;
+constexpr unsigned long long XP_RANGE_LOW = 1ull << 62;
+
+struct XpState {
+    unsigned long long range, code, q, packed;
+};
+
+__device__ __forceinline__ unsigned long long xp_cell(double P, double K) {
+    const double f = P * K;
+    return f >= 4294967296.0 ? XP_TOP : (unsigned long long)f;
+}
+__device__ __forceinline__ bool xp_state_ok(const XpState& s) {
+    return s.range > XP_RANGE_LOW && s.range <= XP_RANGE_TOP && s.code < s.range;
+}
+__device__ __forceinline__ unsigned long long xp_target(const XpState& s) {
+    const unsigned long long t = s.code / (s.range >> 32);
+    return t > 0xFFFFFFFFull ? 0xFFFFFFFFull : t;
+}
+// the next k <= 32 binary digits of the code, most significant first
+__device__ __forceinline__ unsigned long long xp_next_bits(XpState& s, int k, unsigned N) {
+    unsigned long long out = 0;
+    int nq = (int)(s.packed >> 32);
+    unsigned long long rem = s.packed & 0xFFFFFFFFull;
+    const int take = k < nq ? k : nq;
+    if (take > 0) {
+        nq -= take;
+        out = (s.q >> nq) & ((1ull << take) - 1ull);
+        s.q &= nq ? ((1ull << nq) - 1ull) : 0ull;
+        k -= take;
+    }
+    if (k > 0) {
+        const unsigned long long x = rem << k;            // rem < N < 2^31, k <= 32
+        out = (out << k) | (x / N);
+        rem = x % N;
+    }
+    s.packed = ((unsigned long long)nq << 32) | rem;
+    return out;
+}
+// the chosen token owns the cells [lo, hi): narrow the interval to it and shift digits in
+__device__ __forceinline__ void xp_advance(XpState& s, unsigned long long lo, unsigned long long hi, unsigned N) {
+    const unsigned long long r = s.range >> 32;
+    s.code -= r * lo;
+    s.range = hi == XP_TOP ? s.range - r * lo : r * (hi - lo);
+    int shift = __clzll((long long)(s.range - 1)) - 1;    // range -> (2^62, 2^63]
+    while (shift > 0) {
+        const int k = shift < 32 ? shift : 32;
+        s.code = (s.code << k) | xp_next_bits(s, k, N);
+        s.range <<= k;
+        shift -= k;
+    }
+}
+
+// One sub-row of the chunk that holds the code's cell: lane l has the masses ev[0..E) of E
+// consecutive tokens, lanes in index order.  `run` is the fp64 prefix before the sub-row,
+// `carry` the cell where it starts (both uniform, both advanced here).  The cell where a lane's
+// last token with mass ends is computed once and handed on, so that neighbouring tokens always
+// meet in the same cell whatever the rounding of the sums; the chunk's last token with mass
+// (in the sub-row flagged is_last) ends at Fend.  Returns the lane that holds the token (its
+// element pk, cells [plo, phi), mass pe) or -1; uniform.
+template <int E>
+__device__ __forceinline__ int xp_subrow(const double (&ev)[E], int lane, double K, unsigned long long tcell,
+                                         bool is_last, unsigned long long Fend, double& run,
+                                         unsigned long long& carry, int& pk, unsigned long long& plo,
+                                         unsigned long long& phi, double& pe) {
+    double local = 0.0;
+    int klast = -1;
+#pragma unroll
+    for (int k = 0; k < E; ++k) { local += ev[k]; if (ev[k] > 0.0) klast = k; }
+    const double incl = warp_incl_scan_d(local, lane);
+    double excl = __shfl_up_sync(FULL, incl, 1);
+    if (lane == 0) excl = 0.0;
+    const unsigned massive = __ballot_sync(FULL, local > 0.0);
+    const double run_next = run + __shfl_sync(FULL, incl, 31);
+    if (!massive) { run = run_next; return -1; }
+    const int Llast = 31 - __clz(massive);
+    const unsigned long long endc = (is_last && lane == Llast) ? Fend : xp_cell(run + incl, K);
+    const unsigned before = massive & ((1u << lane) - 1u);
+    const unsigned long long prev_end = __shfl_sync(FULL, endc, before ? 31 - __clz(before) : 0);
+    unsigned long long lo = before ? prev_end : carry;
+    int pick = -1;
+    unsigned long long mylo = 0, myhi = 0;
+    double mye = 1.0;
+    double S = run + excl;
+#pragma unroll
+    for (int k = 0; k < E; ++k) {
+        if (ev[k] > 0.0) {
+            unsigned long long hi;
+            if (k == klast) {
+                hi = endc;
+            } else {
+                S += ev[k];
+                hi = xp_cell(S, K);
+            }
+            if (pick < 0 && hi > tcell) { pick = k; mylo = lo; myhi = hi; mye = ev[k]; }
+            lo = hi;
+        }
+    }
+    carry = __shfl_sync(FULL, endc, Llast);
+    run = run_next;
+    const unsigned bal = __ballot_sync(FULL, pick >= 0);
+    if (!bal) return -1;
+    const int L = __ffs(bal) - 1;
+    pk = __shfl_sync(FULL, pick, L);
+    plo = __shfl_sync(FULL, mylo, L);
+    phi = __shfl_sync(FULL, myhi, L);
+    pe = __shfl_sync(FULL, mye, L);
+    return L;
+}
+
 // Result of one decode step for one lane, identical in every thread of the CTA.
 struct LaneResult {
     int token;
@@ -329,6 +454,7 @@ struct LaneResult {
     double code_out;
     double p_tok;
     double cdf_lo;
+    unsigned long long xp_lo, xp_hi;      // extended-precision steps: the token's cells [xp_lo, xp_hi)
 };
 
 }  // namespace asx

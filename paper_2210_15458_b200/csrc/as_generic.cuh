@@ -689,6 +689,83 @@ struct GenericLane {
         return out;
     }
 
+    // One step with an extended-precision code: the token that owns cell `tcell` of the 2^32 cells
+    // of this step's CDF over the kept set (any cut), with its cells in the result's xp_lo / xp_hi.
+    __device__ __noinline__ LaneResult run_xp(unsigned long long tcell, double inv_tau_, int top_k, double top_p) {
+        inv_tau = inv_tau_;
+        fill_exp_table(sm.exp_tbl, tid);
+        Pred p;
+        int n_kept;
+        if (prepare(top_k, top_p, p, n_kept) != ST_OK) return fail(0.0, ST_NUMERIC);
+        if (warp == 0) {
+            const double Z = sm.chunk_sum[nchunks];
+            const double K = 4294967296.0 / Z;
+            int last_c = -1;
+            for (int ci = lane; ci < nchunks; ci += 32)
+                if (sm.chunk_sum[ci + 1] > sm.chunk_sum[ci]) last_c = ci;
+            last_c = (int)warp_max_u((unsigned)(last_c + 1)) - 1;
+            int tok = -1;
+            unsigned long long plo = 0, phi = 0;
+            double pe = 1.0;
+            if (last_c >= 0) {
+                int first = INT_MAX;
+                for (int ci = lane; ci <= last_c; ci += 32) {
+                    const unsigned long long fe = ci == last_c ? XP_TOP : xp_cell(sm.chunk_sum[ci + 1], K);
+                    if (fe > tcell && sm.chunk_sum[ci + 1] > sm.chunk_sum[ci]) first = min(first, ci);
+                }
+                const int cstar = (int)warp_min_u((unsigned)first);
+                const unsigned long long Fend = cstar == last_c ? XP_TOP : xp_cell(sm.chunk_sum[cstar + 1], K);
+                // masses of sub-row r of the chunk (kept elements only)
+                auto sub_masses = [&](int r, int& tie_run, double (&ev)[E], int& base) {
+                    uint32_t k[E];
+                    chunk_keys(cstar, r, k, base);
+                    const int rank0 = lane_rank0(k, p, tie_run);
+                    const unsigned bits = kept_bits(k, p, rank0);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) ev[e] = (bits & (1u << e)) ? mass(k[e]) : 0.0;
+                };
+                // the last sub-row of the chunk that holds mass
+                int r_last = 0;
+                {
+                    int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[cstar] : 0;
+                    for (int r = 0; r < R; ++r) {
+                        double ev[E];
+                        int base;
+                        sub_masses(r, tie_run, ev, base);
+                        double local = 0.0;
+#pragma unroll
+                        for (int e = 0; e < E; ++e) local += ev[e];
+                        if (__ballot_sync(FULL, local > 0.0)) r_last = r;
+                    }
+                }
+                double run = sm.chunk_sum[cstar];
+                unsigned long long carry = xp_cell(run, K);
+                int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[cstar] : 0;
+                for (int r = 0; r <= r_last && tok < 0; ++r) {
+                    double ev[E];
+                    int base;
+                    sub_masses(r, tie_run, ev, base);
+                    int pk = 0;
+                    const int L = xp_subrow<E>(ev, lane, K, tcell, r == r_last, Fend, run, carry, pk, plo, phi, pe);
+                    if (L >= 0) tok = __shfl_sync(FULL, base, L) + pk;
+                }
+            }
+            if (lane == 0) {
+                LaneResult r;
+                r.token = tok; r.status = tok < 0 ? ST_NUMERIC : ST_OK; r.n_kept = n_kept;
+                r.code_out = 0.0;
+                r.p_tok = pe / sm.chunk_sum[nchunks];
+                r.cdf_lo = (double)plo * (1.0 / 4294967296.0);
+                r.xp_lo = plo; r.xp_hi = phi;
+                sm.res = r;
+            }
+        }
+        Sync::sync();
+        const LaneResult out = sm.res;
+        Sync::sync();
+        return out;
+    }
+
     // interval_of for lanes without top-k / nucleus on 16-byte aligned rows: a packed max pass,
     // then one pass that sums every mass and, separately, the masses below the token.
     __device__ __noinline__ LaneResult interval_nocut(int tok, double inv_tau_) {

@@ -732,3 +732,37 @@ def test_a_wait_that_runs_out_reports_timeout_and_the_next_call_is_fine(B, orc, 
         check(B, orc, arr, BF16, codes, 0.8, 20, 1.0, what="after a time-out")
     finally:
         B.as_tune(B.TUNE_STEP_PATH, 0)
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_step_without_a_cut_every_evaluation_mode(B, orc, dtype):
+    # temperature only (Algorithm 1 as stated): rows in shared memory, masses from the bf16 table
+    # or from the fp64 exponential.  Covered: ragged row ends, rows of one piece and of several,
+    # masked tokens, zeros of both signs and subnormals (outside the table: evaluated directly),
+    # magnitudes >= 64 (the row is redone relative to its maximum), temperatures below the
+    # table's range, NaN / +inf / all-masked rows, codes 0 and 1.
+    rng = np.random.default_rng(4242)
+    for V, ld in [(8, 8), (64, 64), (4099, 4104), (9000, 9000), (32128, 32128), (49152, 49152), (40003, 40008)]:
+        lanes = 23
+        x = rng.normal(0, 2.5, (lanes, ld)).astype(np.float32)
+        x[:, V:] = 70.0                                        # padding between rows must not count
+        x[1, : V // 2] = -np.inf
+        x[2, rng.choice(V, max(1, V // 7), replace=False)] = 0.0
+        x[2, rng.choice(V, max(1, V // 9), replace=False)] = -0.0
+        x[3, rng.choice(V, max(1, V // 5), replace=False)] = 1e-39    # subnormal in fp32, zero in bf16
+        x[4, rng.integers(0, V)] = 77.0                        # outside the table: robust pass
+        x[5, :] -= 300.0                                       # everything far below zero
+        x[6, rng.integers(0, V)] = np.nan
+        x[7, rng.integers(0, V)] = np.inf
+        x[8, :] = -np.inf
+        x[9, :] = -np.inf
+        x[9, V - 1] = -5.0                                     # a single live token, the last one
+        x[10, :] = 3.0                                         # flat row
+        arr = _store(x, dtype)
+        codes = rng.random(lanes)
+        codes[0], codes[11], codes[12] = 0.0, 1.0, 1.0 - 2.0 ** -53
+        codes[13] = 1.5
+        for temp in (0.8, 1.0, 0.05, 3.0):
+            r = check(B, orc, arr, dtype, codes, temp, 0, 1.0, V=V, what="no cut V=%d dt=%d temp=%g" % (V, dtype, temp))
+            # (at temperature 3 a long row is nearly flat: most tokens are narrower than the boundary band)
+            assert r["compared"] >= (8 if temp < 2.0 or V < 4000 else 3)
