@@ -143,6 +143,22 @@ int as_step(const void *d_logits, int dtype, int lanes, int V, long long ld,
             void *stream);
 
 /*
+ * as_step with the locally typical cut in place of the nucleus (Sec. 2 names typical decoding
+ * among the logit modifiers the method composes with; the rule is that of locally typical
+ * sampling): after temperature and the optional top-k, with p the softmax over the survivors and
+ * H its entropy, the tokens are ordered by |-ln p_j - H| ascending (lower index first among
+ * equals) and the smallest prefix with mass >= typical_p is kept, then renormalised.
+ *   typical_p  mass of the typical set; <= 0 or >= 1 disables (the call is then as_step
+ *              without a nucleus).  Everything else as as_step.
+ * Served by the general full-row routine (d_path reports AS_PATH_GENERAL).
+ * Errors: as as_step, plus AS_ERR_INVALID_ARG for a NaN typical_p.
+ */
+int as_step_typical(const void *d_logits, int dtype, int lanes, int V, long long ld,
+                    const double *d_codes, double temp, int top_k, double typical_p,
+                    int32_t *d_tokens, double *d_codes_out, const as_step_diag *diag,
+                    void *stream);
+
+/*
  * The first step of a decode (Algorithm 1 entered with the codes of the
  * Definition "Arithmetic sampling", Sec. 4.2): as_step with lane i taking the
  * lattice code c = (j0 + i + u)/N mod 1 formed in the kernel -- bit-identical to

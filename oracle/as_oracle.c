@@ -116,7 +116,7 @@ typedef struct {
  * (NaN / +inf logit, no finite logit); fills n_kept, d_topp, tie_topk of `out`.
  */
 static int kept_masses(const void *row, int dtype, long V, double temp, long top_k, double top_p,
-                       double *l, double *e, char *keep, ranked *rk, double *Z_out,
+                       double typical_p, double *l, double *e, char *keep, ranked *rk, double *Z_out,
                        step_result *out)
 {
     long j, nK = 0;
@@ -150,6 +150,47 @@ static int kept_masses(const void *row, int dtype, long V, double temp, long top
         else e[j] = 0.0;
     }
     double Z1 = nsum_val(&z1);
+
+    /* 4b: locally typical set (Sec. 2 names typical decoding among the compatible logit modifiers;
+     * rule of Meister et al.): with H the entropy of the distribution over the survivors, order
+     * them by |-ln p_j - H| ascending (index ascending among equals) and keep the smallest prefix
+     * with mass >= typical_p.  It takes the nucleus's place: a step has one or the other.
+     * d_topp reports how far the cut is from being ambiguous: the normalised distance of the two
+     * straddling prefix masses from the target, or 0 when the last kept and the first dropped
+     * token are nearer than 1e-9 in |-ln p - H| (their order then hangs on rounding). */
+    if (typical_p > 0.0 && typical_p < 1.0) {
+        long n = 0, r, cut;
+        double lnZ = log(Z1);
+        nsum h = {0.0, 0.0};
+        for (j = 0; j < V; ++j)
+            if (keep[j] && e[j] > 0.0) nsum_add(&h, -(e[j] / Z1) * ((l[j] / temp - m) - lnZ));
+        double H = nsum_val(&h);
+        for (j = 0; j < V; ++j)
+            if (keep[j]) { rk[n].key = -fabs(-((l[j] / temp - m) - lnZ) - H); rk[n].idx = j; ++n; }
+        qsort(rk, (size_t)n, sizeof(ranked), cmp_key_desc_idx_asc);     /* -distance descending */
+        double target = typical_p * Z1, before = 0.0, after = 0.0;
+        nsum run = {0.0, 0.0};
+        cut = n;
+        for (r = 0; r < n; ++r) {
+            before = nsum_val(&run);
+            nsum_add(&run, e[rk[r].idx]);
+            after = nsum_val(&run);
+            if (after >= target) { cut = r + 1; break; }
+        }
+        for (r = cut; r < n; ++r) { keep[rk[r].idx] = 0; e[rk[r].idx] = 0.0; }
+        if (cut < n || after >= target) {
+            double a = fabs(target - before), b = fabs(after - target);
+            out->d_topp = (a < b ? a : b) / Z1;
+        }
+        if (cut < n && rk[cut - 1].key - rk[cut].key < 1e-9 &&
+            l[rk[cut - 1].idx] != l[rk[cut].idx])
+            out->d_topp = 0.0;
+        nK = cut;
+        /* renormalised total for whatever follows */
+        nsum z2 = {0.0, 0.0};
+        for (j = 0; j < V; ++j) if (keep[j]) nsum_add(&z2, e[j]);
+        Z1 = nsum_val(&z2);
+    }
 
     /* 5: nucleus: smallest (prob desc, index asc) prefix with mass >= top_p */
     if (top_p > 0.0 && top_p < 1.0) {
@@ -185,9 +226,9 @@ static int kept_masses(const void *row, int dtype, long V, double temp, long top
  * One step for one lane (Algorithm 1, loop body).  row points at V stored
  * logits.  Work arrays as for kept_masses.
  */
-static void step_lane(const void *row, int dtype, long V, double c, double temp,
-                      long top_k, double top_p, double *l, double *e, char *keep,
-                      ranked *rk, step_result *out)
+static void step_lane_t(const void *row, int dtype, long V, double c, double temp,
+                        long top_k, double top_p, double typical_p, double *l, double *e, char *keep,
+                        ranked *rk, step_result *out)
 {
     long j;
     double Z;
@@ -198,7 +239,7 @@ static void step_lane(const void *row, int dtype, long V, double c, double temp,
     if (!(c >= 0.0 && c <= 1.0)) return;          /* also rejects NaN */
     if (c == 1.0) c = ORC_ONE_BELOW;              /* code domain is [0,1) */
 
-    if (kept_masses(row, dtype, V, temp, top_k, top_p, l, e, keep, rk, &Z, out) != ORC_OK) {
+    if (kept_masses(row, dtype, V, temp, top_k, top_p, typical_p, l, e, keep, rk, &Z, out) != ORC_OK) {
         out->n_kept = 0; out->d_topp = INFINITY; out->tie_topk = 0;
         return;
     }
@@ -231,6 +272,13 @@ static void step_lane(const void *row, int dtype, long V, double c, double temp,
     out->cdf_lo = lo;
     out->d_tok = da < db ? da : db;
     out->status = ORC_OK;
+}
+
+static void step_lane(const void *row, int dtype, long V, double c, double temp,
+                      long top_k, double top_p, double *l, double *e, char *keep,
+                      ranked *rk, step_result *out)
+{
+    step_lane_t(row, dtype, V, c, temp, top_k, top_p, 1.0, l, e, keep, rk, out);
 }
 
 typedef struct { double *l, *e; char *keep; ranked *rk; } workspace;
@@ -298,8 +346,8 @@ int orc_lattice_codes_variant(long N, double b, long variant, double *codes)
     return ORC_OK;
 }
 
-int orc_step(const void *logits, int dtype, long lanes, long V, long ld,
-             const double *codes, double temp, long top_k, double top_p,
+static int step_all(const void *logits, int dtype, long lanes, long V, long ld,
+             const double *codes, double temp, long top_k, double top_p, double typical_p,
              int32_t *tokens, double *codes_out, double *p_tok, double *cdf_lo,
              int32_t *n_kept, double *d_tok, double *d_topp, int32_t *tie_topk,
              int32_t *status, long lane_begin, long lane_end)
@@ -315,7 +363,7 @@ int orc_step(const void *logits, int dtype, long lanes, long V, long ld,
     for (i = lane_begin; i < lane_end; ++i) {
         step_result r;
         const char *row = (const char *)logits + (size_t)i * (size_t)ld * esz;
-        step_lane(row, dtype, V, codes[i], temp, top_k, top_p, w.l, w.e, w.keep, w.rk, &r);
+        step_lane_t(row, dtype, V, codes[i], temp, top_k, top_p, typical_p, w.l, w.e, w.keep, w.rk, &r);
         if (tokens) tokens[i] = r.token;
         if (codes_out) codes_out[i] = r.code_out;
         if (p_tok) p_tok[i] = r.p_tok;
@@ -328,6 +376,28 @@ int orc_step(const void *logits, int dtype, long lanes, long V, long ld,
     }
     ws_free(&w);
     return ORC_OK;
+}
+
+int orc_step(const void *logits, int dtype, long lanes, long V, long ld,
+             const double *codes, double temp, long top_k, double top_p,
+             int32_t *tokens, double *codes_out, double *p_tok, double *cdf_lo,
+             int32_t *n_kept, double *d_tok, double *d_topp, int32_t *tie_topk,
+             int32_t *status, long lane_begin, long lane_end)
+{
+    return step_all(logits, dtype, lanes, V, ld, codes, temp, top_k, top_p, 1.0, tokens, codes_out, p_tok,
+                    cdf_lo, n_kept, d_tok, d_topp, tie_topk, status, lane_begin, lane_end);
+}
+
+/* orc_step with the locally typical cut of mass typical_p in place of the nucleus */
+int orc_step_typical(const void *logits, int dtype, long lanes, long V, long ld,
+                     const double *codes, double temp, long top_k, double typical_p,
+                     int32_t *tokens, double *codes_out, double *p_tok, double *cdf_lo,
+                     int32_t *n_kept, double *d_tok, double *d_topp, int32_t *tie_topk,
+                     int32_t *status, long lane_begin, long lane_end)
+{
+    if (isnan(typical_p)) return ORC_ERR_INVALID_ARG;
+    return step_all(logits, dtype, lanes, V, ld, codes, temp, top_k, 1.0, typical_p, tokens, codes_out, p_tok,
+                    cdf_lo, n_kept, d_tok, d_topp, tie_topk, status, lane_begin, lane_end);
 }
 
 /*
@@ -632,7 +702,7 @@ static int xp_row_cells(const void *row, int dtype, long V, double temp, long to
 {
     long j, last = -1;
     double Z;
-    int rc = kept_masses(row, dtype, V, temp, top_k, top_p, w->l, w->e, w->keep, w->rk, &Z, info);
+    int rc = kept_masses(row, dtype, V, temp, top_k, top_p, 1.0, w->l, w->e, w->keep, w->rk, &Z, info);
     if (rc != ORC_OK) return rc;
     const double K = XP_CELLS / Z;
     nsum run = {0.0, 0.0};

@@ -49,6 +49,8 @@ def lib():
         P = ctypes.c_void_p
         _lib.orc_lattice_codes.argtypes = [L, D, P]
         _lib.orc_step.argtypes = [P, ctypes.c_int, L, L, L, P, D, L, D] + [P] * 9 + [L, L]
+        _lib.orc_step_typical.argtypes = [P, ctypes.c_int, L, L, L, P, D, L, D] + [P] * 9 + [L, L]
+        _lib.orc_step_typical.restype = ctypes.c_int
         _lib.orc_decode_bigram_codes.argtypes = ([P, ctypes.c_int, L, L, P, P, L, L, L, D, L, D]
                                                  + [P] * 8 + [L, L])
         _lib.orc_decode_bigram.argtypes = [P, ctypes.c_int, L, L, P, L, L, D, L, L, D, L, D, P, P, P, P]
@@ -131,7 +133,13 @@ class StepOut:
 
 
 def step(logits: np.ndarray, dtype: int, codes: np.ndarray, temp: float = 1.0, top_k: int = 0,
-         top_p: float = 1.0, V: Optional[int] = None, threads: int = 1) -> StepOut:
+         top_p: float = 1.0, V: Optional[int] = None, threads: int = 1, typical_p: float = 1.0) -> StepOut:
+    """One decode step per lane.  typical_p in (0,1): the locally typical cut instead of the nucleus."""
+    typical = 0.0 < typical_p < 1.0
+    if typical and 0.0 < top_p < 1.0:
+        raise ValueError("a step takes a nucleus or a typical cut, not both")
+    fn = lib().orc_step_typical if typical else lib().orc_step
+    cutp = typical_p if typical else top_p
     logits = _check_logits(logits, dtype)
     lanes, ld = logits.shape
     V = ld if V is None else V
@@ -143,7 +151,7 @@ def step(logits: np.ndarray, dtype: int, codes: np.ndarray, temp: float = 1.0, t
                 np.empty(lanes, np.float64), np.empty(lanes, np.int32), np.empty(lanes, np.int32))
 
     def run(a, b):
-        return lib().orc_step(_ptr(logits), dtype, lanes, V, ld, _ptr(codes), temp, top_k, top_p,
+        return fn(_ptr(logits), dtype, lanes, V, ld, _ptr(codes), temp, top_k, cutp,
                               _ptr(o.tokens), _ptr(o.codes), _ptr(o.p_tok), _ptr(o.cdf_lo),
                               _ptr(o.n_kept), _ptr(o.d_tok), _ptr(o.d_topp), _ptr(o.tie_topk),
                               _ptr(o.status), a, b)

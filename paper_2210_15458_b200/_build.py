@@ -7,6 +7,8 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libarith_sampling.so")
+# the same sources with every shared-memory index checked (-DAS_BOUNDS_CHECK): for the tests
+LIB_CHECKED = os.path.join(_HERE, "libarith_sampling_check.so")
 SOURCES = ["as_api.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
@@ -28,18 +30,20 @@ def _newest_source_mtime() -> float:
     return m
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile csrc/*.cu into libarith_sampling.so if it is missing or stale."""
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source_mtime():
-        return LIB
-    tmp = LIB + ".tmp.%d" % os.getpid()
-    cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Compile csrc/*.cu into libarith_sampling.so (checked: libarith_sampling_check.so, with
+    -DAS_BOUNDS_CHECK) if it is missing or stale."""
+    lib = LIB_CHECKED if checked else LIB
+    if not force and os.path.exists(lib) and os.path.getmtime(lib) >= _newest_source_mtime():
+        return lib
+    tmp = lib + ".tmp.%d" % os.getpid()
+    cmd = [_nvcc()] + NVCC_FLAGS + (["-DAS_BOUNDS_CHECK"] if checked else []) + (["-Xptxas", "-v"] if verbose else []) + \
           ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
     import sys
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

@@ -37,7 +37,7 @@ TUNE_SERIAL_LAUNCH = 6
 TUNE_WAIT_KCYCLES = 7
 TUNE_DEBUG_NO_COPY = 8
 
-EXPORTS = ["as_lattice_codes", "as_lattice_codes_variant", "as_step", "as_step_lattice", "as_step_host", "as_step_host_work_bytes", "as_step_host_static",
+EXPORTS = ["as_lattice_codes", "as_lattice_codes_variant", "as_step", "as_step_typical", "as_step_lattice", "as_step_host", "as_step_host_work_bytes", "as_step_host_static",
            "as_decode_bigram",
            "as_decode_bigram_codes", "as_xp_lattice_state", "as_decode_bigram_xp", "as_encode_bigram", "as_ngram_diversity", "as_reward_mean", "as_tune",
            "as_last_error", "as_version"]
@@ -62,11 +62,30 @@ def library_path() -> str:
     return _build.LIB
 
 
+_path = None
+
+
+def use_library(path: Optional[str]) -> None:
+    """Switch to another build of the library (the bounds-checked one, in tests); None = the default."""
+    global _lib, _path
+    _lib, _path = None, path
+
+
+def as_debug_bounds(reset: bool = True):
+    """Checked builds only: (failures, first site, its index, its bound) since the last reset."""
+    out = (ctypes.c_int * 4)()
+    fn = lib().as_debug_bounds
+    fn.argtypes = [ctypes.c_void_p, ctypes.c_int]
+    fn.restype = ctypes.c_int
+    _check(fn(ctypes.cast(out, ctypes.c_void_p), 1 if reset else 0))
+    return tuple(out)
+
+
 def lib():
     """Load the CUDA library (never builds or falls back silently)."""
     global _lib
     if _lib is None:
-        path = library_path()
+        path = _path or library_path()
         if not os.path.exists(path):
             raise RuntimeError("CUDA library %s not found: run `python -c 'import __graft_entry__ as g; "
                                "g.build()'` (nvcc, sm_100a) first" % path)
@@ -74,6 +93,8 @@ def lib():
         P, I, D, LL = ctypes.c_void_p, ctypes.c_int, ctypes.c_double, ctypes.c_longlong
         L.as_lattice_codes.argtypes = [I, D, P, P]
         L.as_step.argtypes = [P, I, I, I, LL, P, D, I, D, P, P, ctypes.POINTER(as_step_diag), P]
+        L.as_step_typical.argtypes = [P, I, I, I, LL, P, D, I, D, P, P, ctypes.POINTER(as_step_diag), P]
+        L.as_step_typical.restype = I
         L.as_step_host.argtypes = [P, I, I, I, LL, P, D, I, D, P, P, P, P, ctypes.c_size_t, P]
         L.as_step_host_static.argtypes = [P, I, I, I, LL, P, D, I, D, P, P, P, P]
         L.as_step_host_static.restype = I
@@ -161,9 +182,10 @@ def as_lattice_codes_variant(N: int, b: float, variant: int, out: Optional[torch
 def as_step(logits: torch.Tensor, codes: torch.Tensor, temp: float = 1.0, top_k: int = 0,
             top_p: float = 1.0, tokens: Optional[torch.Tensor] = None,
             codes_out: Optional[torch.Tensor] = None, diag: Optional[dict] = None, V: Optional[int] = None,
-            stream=None):
+            stream=None, typical_p: Optional[float] = None):
     """tokens, codes' = one decode step.  `diag`, if a dict, receives the tensors p_tok,
-    cdf_lo, n_kept, lane_status, path (allocated here unless already present)."""
+    cdf_lo, n_kept, lane_status, path (allocated here unless already present).  With typical_p
+    the call goes to as_step_typical (the typical cut in place of the nucleus)."""
     lanes, width, ld = _logits_layout(logits)
     V = width if V is None else V
     dev = logits.device
@@ -182,6 +204,13 @@ def as_step(logits: torch.Tensor, codes: torch.Tensor, temp: float = 1.0, top_k:
         diag.setdefault("path", torch.empty(lanes, dtype=torch.int32, device=dev))
         dg = as_step_diag(_ptr(diag["p_tok"]), _ptr(diag["cdf_lo"]), _ptr(diag["n_kept"]),
                           _ptr(diag["lane_status"]), _ptr(diag["path"]))
+    if typical_p is not None:
+        if 0.0 < top_p < 1.0:
+            raise ValueError("a step takes top_p or typical_p, not both")
+        _check(lib().as_step_typical(_ptr(logits), _logits_dtype(logits), lanes, V, ld, _ptr(codes), temp, top_k,
+                                     typical_p, _ptr(tokens), _ptr(codes_out),
+                                     ctypes.byref(dg) if dg is not None else None, _stream(stream)))
+        return tokens, codes_out
     _check(lib().as_step(_ptr(logits), _logits_dtype(logits), lanes, V, ld, _ptr(codes), temp, top_k, top_p,
                          _ptr(tokens), _ptr(codes_out), ctypes.byref(dg) if dg is not None else None,
                          _stream(stream)))

@@ -260,7 +260,7 @@ template <int DT>
 __global__ void __launch_bounds__(GEN_NT)
 step_generic_kernel(const void* __restrict__ logits, int lanes, int V, long long ld,
                     const double* codes, int lat_N, int lat_j0, double lat_u, double inv_tau, int top_k,
-                    double top_p, int* __restrict__ tokens, double* codes_out, DiagPtrs diag) {
+                    double top_p, double typical_p, int* __restrict__ tokens, double* codes_out, DiagPtrs diag) {
     __shared__ GenericSmem<GEN_NT> sm;
     for (int ln = blockIdx.x; ln < lanes; ln += gridDim.x) {
         const char* row = reinterpret_cast<const char*>(logits) + (size_t)ln * (size_t)ld * Traits<DT>::BYTES;
@@ -273,7 +273,7 @@ step_generic_kernel(const void* __restrict__ logits, int lanes, int V, long long
             c = codes[ln];
         }
         GenericLane<DT, GEN_NT> g(sm, row, V, vec_ok);
-        const LaneResult r = g.run(c, inv_tau, top_k, top_p);
+        const LaneResult r = g.run(c, inv_tau, top_k, top_p, typical_p);
         if (threadIdx.x == 0) {
             tokens[ln] = r.token;
             codes_out[ln] = r.code_out;
@@ -410,7 +410,7 @@ decode_xp_generic_kernel(const void* __restrict__ table, int V, long long ld, co
             GenericLane<DT, GEN_NT> g(sm, row, V, vec_ok);
             const LaneResult r = g.run_xp(xp_target(xs), inv_tau, top_k, top_p);
             if (r.status != ST_OK) { status = r.status; break; }
-            xp_advance(xs, r.xp_lo, r.xp_hi, (unsigned)N);
+            xp_advance(xs, sm.xp_lo, sm.xp_hi, (unsigned)N);
             if (threadIdx.x == 0) seq[(size_t)ln * T + t] = r.token;
             n = t + 1;
             prev = r.token;
@@ -511,6 +511,17 @@ int as_debug_cta(unsigned long long* h_out) {
 }
 int as_debug_counts(unsigned long long* h_out) {
     return cudaMemcpyFromSymbol(h_out, g_asx_counts, sizeof(unsigned long long) * 16) == cudaSuccess ? AS_OK : AS_ERR_CUDA;
+}
+#endif
+
+#ifdef AS_BOUNDS_CHECK
+// checked builds only: the record of out-of-range indices (failures, first site, its index, its
+// bound) since the last reset
+int as_debug_bounds(int* h_out4, int reset) {
+    int zero[4] = {0, 0, 0, 0};
+    if (h_out4 && cudaMemcpyFromSymbol(h_out4, g_asx_bounds, sizeof(zero)) != cudaSuccess) return AS_ERR_CUDA;
+    if (reset && cudaMemcpyToSymbol(g_asx_bounds, zero, sizeof(zero)) != cudaSuccess) return AS_ERR_CUDA;
+    return AS_OK;
 }
 #endif
 
@@ -618,7 +629,8 @@ static int launch_streaming(StepArgs& a, int dtype, bool unaligned, int sms, cud
 // as_step and as_step_lattice: lat_N = 0 reads d_codes, lat_N > 0 forms the lattice codes in the kernel
 static int step_common(const void* d_logits, int dtype, int lanes, int V, long long ld, const double* d_codes,
                        int lat_N, int lat_j0, double lat_u, double temp, int top_k, double top_p,
-                       int32_t* d_tokens, double* d_codes_out, const as_step_diag* diag, void* stream) {
+                       int32_t* d_tokens, double* d_codes_out, const as_step_diag* diag, void* stream,
+                       double typical_p = 1.0) {
     if (lanes < 0) return set_err(AS_ERR_INVALID_ARG, "lanes = %d must be >= 0", lanes);
     int rc = check_scalars(dtype, V, ld, temp, top_p);
     if (rc != AS_OK) return rc;
@@ -632,6 +644,10 @@ static int step_common(const void* d_logits, int dtype, int lanes, int V, long l
     if (diag) dp = {diag->d_p_tok, diag->d_cdf_lo, diag->d_n_kept, diag->d_lane_status, diag->d_path};
     if (top_k < 0 || top_k >= V) top_k = 0;
     if (!(top_p > 0.0 && top_p < 1.0)) top_p = 1.0;
+    if (std::isnan(typical_p)) return set_err(AS_ERR_INVALID_ARG, "typical_p is NaN");
+    const bool typical = typical_p > 0.0 && typical_p < 1.0;
+    if (!typical) typical_p = 1.0;
+    if (typical && top_p < 1.0) return set_err(AS_ERR_INVALID_ARG, "a step takes a nucleus (top_p) or a typical cut (typical_p), not both");
     const double inv_tau = 1.0 / temp;
     cudaStream_t st = (cudaStream_t)stream;
     StepArgs a;
@@ -646,11 +662,11 @@ static int step_common(const void* d_logits, int dtype, int lanes, int V, long l
     // some row starts off a 16-byte boundary: it is read from the boundary below, up to E-1 elements longer
     const bool unaligned = (reinterpret_cast<uintptr_t>(d_logits) & 15) != 0 || (((size_t)ld * esz) & 15) != 0;
     const size_t row_bytes = (size_t)((V + (unaligned && g_tune_path == 0 ? E - 1 : 0) + E - 1) / E) * 16;
-    if (g_tune_path == 0) {
+    if (g_tune_path == 0 && !typical) {
         rc = launch_streaming(a, dtype, unaligned, di->sms, st);
         if (rc != AS_ERR_UNSUPPORTED) return rc;
     }
-    if (top_k == 0 && !(top_p < 1.0)) {
+    if (top_k == 0 && !(top_p < 1.0) && !typical) {
         NocutArgs n = {};
         n.data = d_logits; n.ld = ld; n.V = V; n.lanes = lanes; n.inv_tau = inv_tau;
         n.codes = d_codes; n.lat_N = lat_N; n.lat_j0 = lat_j0; n.lat_u = lat_u;
@@ -658,7 +674,7 @@ static int step_common(const void* d_logits, int dtype, int lanes, int V, long l
         rc = launch_nocut<NC_STEP>(n, dtype, temp, di->sms, st);
         if (rc != AS_ERR_UNSUPPORTED) return rc;
     }
-    if (g_tune_path == 2) {
+    if (g_tune_path == 2 && !typical) {
         // cluster kernel: the row split over CS CTAs' shared memory
         int cs = g_tune_cluster;
         if (cs == 0) cs = row_bytes <= 80 * 1024 ? 1 : row_bytes <= 160 * 1024 ? 2 : row_bytes <= 320 * 1024 ? 4 : 8;
@@ -672,9 +688,9 @@ static int step_common(const void* d_logits, int dtype, int lanes, int V, long l
     }
     const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
     if (dtype == AS_F32)
-        step_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, lat_N, lat_j0, lat_u, inv_tau, top_k, top_p, d_tokens, d_codes_out, dp);
+        step_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, lat_N, lat_j0, lat_u, inv_tau, top_k, top_p, typical_p, d_tokens, d_codes_out, dp);
     else
-        step_generic_kernel<DT_BF16><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, lat_N, lat_j0, lat_u, inv_tau, top_k, top_p, d_tokens, d_codes_out, dp);
+        step_generic_kernel<DT_BF16><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, lat_N, lat_j0, lat_u, inv_tau, top_k, top_p, typical_p, d_tokens, d_codes_out, dp);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "step kernel launch");
     return AS_OK;
@@ -687,6 +703,13 @@ int as_step(const void* d_logits, int dtype, int lanes, int V, long long ld, con
             const as_step_diag* diag, void* stream) {
     return step_common(d_logits, dtype, lanes, V, ld, d_codes, 0, 0, 0.0, temp, top_k, top_p, d_tokens,
                        d_codes_out, diag, stream);
+}
+
+int as_step_typical(const void* d_logits, int dtype, int lanes, int V, long long ld, const double* d_codes,
+                    double temp, int top_k, double typical_p, int32_t* d_tokens, double* d_codes_out,
+                    const as_step_diag* diag, void* stream) {
+    return step_common(d_logits, dtype, lanes, V, ld, d_codes, 0, 0, 0.0, temp, top_k, 1.0, d_tokens,
+                       d_codes_out, diag, stream, typical_p);
 }
 
 int as_step_lattice(const void* d_logits, int dtype, int lanes, int V, long long ld, int N, double u, int j0,

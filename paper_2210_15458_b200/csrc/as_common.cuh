@@ -13,6 +13,27 @@ constexpr int ST_OK = 0;
 constexpr int ST_TIMEOUT = -4;
 constexpr int ST_NUMERIC = -5;
 
+// Checked builds (-DAS_BOUNDS_CHECK): every index into a ring stage, a hit or candidate list, a
+// rank array, a histogram, a chunk array, the mass table or a row buffer goes through ASX_AT.  An
+// index outside [0, n) is recorded (the count of failures and the first one's site, index and
+// bound) and replaced by 0, so that the access stays in bounds: nothing traps, and the host reads
+// the record after the launch.  In ordinary builds ASX_AT(i, n, site) is just i.
+#ifdef AS_BOUNDS_CHECK
+__device__ int g_asx_bounds[4];
+__device__ __forceinline__ bool asx_in(long long i, long long n, int site) {
+    if (i >= 0 && i < n) return true;
+    if (atomicAdd(&g_asx_bounds[0], 1) == 0) {
+        g_asx_bounds[1] = site;
+        g_asx_bounds[2] = (int)i;
+        g_asx_bounds[3] = (int)n;
+    }
+    return false;
+}
+#define ASX_AT(i, n, site) (asx_in((long long)(i), (long long)(n), (site)) ? (i) : 0)
+#else
+#define ASX_AT(i, n, site) (i)
+#endif
+
 // Largest double below 1: rescaled codes are clamped into [0, ONE_BELOW].
 #define ASX_ONE_BELOW 0x1.fffffffffffffp-1
 
@@ -454,7 +475,6 @@ struct LaneResult {
     double code_out;
     double p_tok;
     double cdf_lo;
-    unsigned long long xp_lo, xp_hi;      // extended-precision steps: the token's cells [xp_lo, xp_hi)
 };
 
 }  // namespace asx

@@ -31,10 +31,23 @@ struct Pred {
     int eq_mode;
 };
 
+// Locally typical cut: kept(j) also needs tkey(j) > T, or tkey(j) == T and: eq_mode 1 -> always;
+// eq_mode 2 -> only the first `need` such kept elements in index order.  tkey orders the tokens
+// by |y_j - mu| ascending (y the scaled logit, mu its mean under the distribution = ln Z - H).
+struct TypPred {
+    int on;
+    double mu;
+    unsigned long long T;
+    int need;
+    int eq_mode;
+};
+
 template <int NT>
 struct GenericSmem {
     double chunk_sum[MAXCH + 1];
     int chunk_eq[MAXCH + 1];
+    int chunk_eq2[MAXCH + 1];             // typical cut: ties at its threshold, per chunk
+    unsigned chunk_has[MAXCH / 32];       // bit ci: chunk ci holds mass (set with chunk_sum, before its scan)
     double hist_mass[256 * HIST_REP];     // bin d, replica r at [d * HIST_REP + r]: lanes spread over
     int hist_cnt[256 * HIST_REP];         // the replicas, so that a crowded bin is hit by fewer threads
     double red_d[NT / 32];
@@ -46,6 +59,7 @@ struct GenericSmem {
     int b_i[4];
     unsigned b_u[2];
     LaneResult res;
+    unsigned long long xp_lo, xp_hi;      // extended-precision steps: the chosen token's cells
 };
 
 // Barrier over the NT threads that run a lane: the whole CTA, or (in kernels with a
@@ -73,9 +87,11 @@ struct GenericLane {
     int nvec, R, nchunks;
     int tid, lane, warp;
     double lmax, inv_tau;
+    TypPred tp;
 
     __device__ GenericLane(GenericSmem<NT>& s, const void* row_, int V_, bool vec_ok_)
         : sm(s), row(row_), V(V_), vec_ok(vec_ok_) {
+        tp.on = 0; tp.mu = 0.0; tp.T = 0; tp.need = 0; tp.eq_mode = 0;
         tid = threadIdx.x;
         lane = tid & 31;
         warp = tid >> 5;
@@ -126,6 +142,56 @@ struct GenericLane {
         return exp_nonpos(((double)Tr::value_f(key) - lmax) * inv_tau, sm.exp_tbl);
     }
 
+    // Does chunk ci hold mass?  (Not to be read off the scanned sums: the scan adds lane totals in
+    // another order than the running sums inside a lane, so sum[ci+1] > sum[ci] can hold by an ulp
+    // for an empty chunk at a lane boundary.)
+    __device__ __forceinline__ bool has_mass(int ci) const { return (sm.chunk_has[ci >> 5] >> (ci & 31)) & 1u; }
+    __device__ __forceinline__ void clear_has() {
+        for (int i = tid; i < MAXCH / 32; i += NT) sm.chunk_has[i] = 0u;
+        Sync::sync();
+    }
+    __device__ __forceinline__ void put_chunk(int ci, double local) {      // lane 0 of the chunk's warp
+        sm.chunk_sum[ASX_AT(ci, MAXCH + 1, 82)] = local;
+        if (local > 0.0) atomicOr(&sm.chunk_has[ci >> 5], 1u << (ci & 31));
+    }
+
+    // typical cut: order key of a token, larger = nearer the mean scaled logit
+    __device__ __forceinline__ unsigned long long tkey(uint32_t key) const {
+        const double y = ((double)Tr::value_f(key) - lmax) * inv_tau;
+        return ~(unsigned long long)__double_as_longlong(fabs(y - tp.mu));
+    }
+    // kept elements of this lane's vector under the top-k / nucleus predicate and, if on, the
+    // typical cut; tie_run / tie_run2 carry the index-order ranks of the two kinds of ties
+    __device__ __forceinline__ unsigned kept_all(const uint32_t (&k)[E], const Pred& p, int& tie_run, int& tie_run2) const {
+        const int rank0 = lane_rank0(k, p, tie_run);
+        unsigned bits = kept_bits(k, p, rank0);
+        if (!tp.on) return bits;
+        unsigned gt = 0, eqm = 0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            if (bits & (1u << e)) {
+                const unsigned long long t = tkey(k[e]);
+                if (t > tp.T) gt |= 1u << e;
+                else if (t == tp.T) eqm |= 1u << e;
+            }
+        }
+        if (tp.eq_mode == 1) return gt | eqm;
+        if (tp.eq_mode == 2) {
+            const int cnt = __popc(eqm);
+            const int incl = warp_incl_scan_i(cnt, lane);
+            int rank = tie_run2 + incl - cnt;
+            tie_run2 += __shfl_sync(FULL, incl, 31);
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                if (eqm & (1u << e)) {
+                    if (rank < tp.need) gt |= 1u << e;
+                    ++rank;
+                }
+            }
+        }
+        return gt;
+    }
+
     // exclusive scan of a[0..n), n >= 1, in place by warp 0; a[n] receives the total
     template <typename T>
     __device__ void scan_exclusive(T* a, int n) {
@@ -166,7 +232,7 @@ struct GenericLane {
                 for (int e = 0; e < E; ++e) cnt += (k[e] == T);
             }
             cnt = warp_sum_i(cnt);
-            if (lane == 0) sm.chunk_eq[ci] = cnt;
+            if (lane == 0) sm.chunk_eq[ASX_AT(ci, MAXCH + 1, 83)] = cnt;
         }
         Sync::sync();
         scan_exclusive(sm.chunk_eq, nchunks);
@@ -174,21 +240,22 @@ struct GenericLane {
 
     // chunk_sum[ci] <- mass of the kept elements of chunk ci
     __device__ void sum_pass(const Pred& p) {
+        clear_has();
         for (int ci = warp; ci < nchunks; ci += NW) {
             int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[ci] : 0;
+            int tie_run2 = (tp.on && tp.eq_mode == 2) ? sm.chunk_eq2[ci] : 0;
             double local = 0.0;
             for (int r = 0; r < R; ++r) {
                 uint32_t k[E];
                 int base;
                 chunk_keys(ci, r, k, base);
-                const int rank0 = lane_rank0(k, p, tie_run);
-                const unsigned bits = kept_bits(k, p, rank0);
+                const unsigned bits = kept_all(k, p, tie_run, tie_run2);
 #pragma unroll
                 for (int e = 0; e < E; ++e)
                     if (bits & (1u << e)) local += mass(k[e]);
             }
             local = warp_sum_d(local);
-            if (lane == 0) sm.chunk_sum[ci] = local;
+            if (lane == 0) put_chunk(ci, local);
         }
         Sync::sync();
     }
@@ -224,8 +291,8 @@ struct GenericLane {
                         const int d = (k[e] >> shift) & 255;
                         if (d != cur_d) {
                             if (cur_n) {
-                                atomicAdd(&sm.hist_cnt[cur_d * HIST_REP + rep], cur_n);
-                                if (MASS) atomicAdd(&sm.hist_mass[cur_d * HIST_REP + rep], cur_m);
+                                atomicAdd(&sm.hist_cnt[ASX_AT(cur_d * HIST_REP + rep, 256 * HIST_REP, 80)], cur_n);
+                                if (MASS) atomicAdd(&sm.hist_mass[ASX_AT(cur_d * HIST_REP + rep, 256 * HIST_REP, 81)], cur_m);
                             }
                             cur_d = d; cur_n = 0; cur_m = 0.0;
                         }
@@ -236,8 +303,8 @@ struct GenericLane {
             }
         }
         if (cur_n) {
-            atomicAdd(&sm.hist_cnt[cur_d * HIST_REP + rep], cur_n);
-            if (MASS) atomicAdd(&sm.hist_mass[cur_d * HIST_REP + rep], cur_m);
+            atomicAdd(&sm.hist_cnt[ASX_AT(cur_d * HIST_REP + rep, 256 * HIST_REP, 80)], cur_n);
+            if (MASS) atomicAdd(&sm.hist_mass[ASX_AT(cur_d * HIST_REP + rep, 256 * HIST_REP, 81)], cur_m);
         }
         Sync::sync();
     }
@@ -271,9 +338,9 @@ struct GenericLane {
             double above_m = __shfl_down_sync(FULL, suf_m, 1);
             if (lane == 31) { above_c = 0; above_m = 0.0; }
             int best = -1, best_above_c = 0, best_c = 0;
-            double best_above_m = 0.0;
+            double best_above_m = 0.0, best_m = 0.0;
             int low = -1, low_above_c = 0, low_c = 0;
-            double low_above_m = 0.0;
+            double low_above_m = 0.0, low_m = 0.0;
             int run_c = above_c;
             double run_m = above_m;
 #pragma unroll
@@ -282,9 +349,9 @@ struct GenericLane {
                     const bool ok = MASS ? (acc_mass + (run_m + m[e]) >= m_target)
                                          : (acc_cnt + run_c + c[e] >= k_target);
                     if (ok && best < 0) {
-                        best = lane * 8 + e; best_above_c = run_c; best_above_m = run_m; best_c = c[e];
+                        best = lane * 8 + e; best_above_c = run_c; best_above_m = run_m; best_c = c[e]; best_m = m[e];
                     }
-                    low = lane * 8 + e; low_above_c = run_c; low_above_m = run_m; low_c = c[e];
+                    low = lane * 8 + e; low_above_c = run_c; low_above_m = run_m; low_c = c[e]; low_m = m[e];
                 }
                 run_c += c[e];
                 run_m += m[e];
@@ -296,8 +363,9 @@ struct GenericLane {
             } else {
                 const unsigned bal2 = __ballot_sync(FULL, low >= 0);
                 src = bal2 ? (__ffs(bal2) - 1) : 0;
-                best = low; best_above_c = low_above_c; best_above_m = low_above_m; best_c = low_c;
+                best = low; best_above_c = low_above_c; best_above_m = low_above_m; best_c = low_c; best_m = low_m;
             }
+            best_m = __shfl_sync(FULL, best_m, src);
             best = __shfl_sync(FULL, best, src);
             best_above_c = __shfl_sync(FULL, best_above_c, src);
             best_above_m = __shfl_sync(FULL, best_above_m, src);
@@ -307,6 +375,7 @@ struct GenericLane {
                 sm.b_i[1] = acc_cnt + best_above_c;
                 sm.b_i[2] = best_c;
                 sm.b_d[0] = acc_mass + best_above_m;
+                sm.b_d[1] = best_m;
             }
         }
         Sync::sync();
@@ -376,6 +445,7 @@ struct GenericLane {
         // logit of every step goes through.
         const bool plain = kmin > Tr::KEY_NINF && fma((double)Tr::value_f(kmin), s64, c64) >= -64000.0;
         // ---- 2. per-chunk masses in index order
+        clear_has();
         int nfin = 0;
         for (int ci = warp; ci < nchunks; ci += NW) {
             double local = 0.0;
@@ -395,7 +465,7 @@ struct GenericLane {
                 }
             }
             local = warp_sum_d(local);
-            if (lane == 0) sm.chunk_sum[ci] = local;
+            if (lane == 0) put_chunk(ci, local);
         }
         nfin = warp_sum_i(nfin);
         if (lane == 0) atomicAdd(&sm.b_i[2], nfin);
@@ -408,10 +478,9 @@ struct GenericLane {
         if (tid == 0) { sm.b_i[0] = INT_MAX; sm.b_i[1] = -1; }
         Sync::sync();
         for (int ci = tid; ci < nchunks; ci += NT) {
-            const double excl = sm.chunk_sum[ci], incl = sm.chunk_sum[ci + 1];
-            if (incl > excl) {
+            if (has_mass(ci)) {
                 atomicMax(&sm.b_i[1], ci);
-                if (t < incl) atomicMin(&sm.b_i[0], ci);
+                if (t < sm.chunk_sum[ci + 1]) atomicMin(&sm.b_i[0], ci);
             }
         }
         Sync::sync();
@@ -485,10 +554,125 @@ struct GenericLane {
         return out;
     }
 
+    // The typical cut among the elements kept by `p` (whose masses' scan is in chunk_sum): sets tp.
+    __device__ void typical_cut(const Pred& p, double typical_p, int& n_kept) {
+        const double Z1 = sm.chunk_sum[nchunks];
+        Sync::sync();
+        // mean scaled logit under the distribution: mu = sum e_j y_j / Z1  (= ln Z1 - H)
+        double acc = 0.0;
+        for (int ci = warp; ci < nchunks; ci += NW) {
+            int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[ci] : 0, unused = 0;
+            for (int r = 0; r < R; ++r) {
+                uint32_t k[E];
+                int base;
+                chunk_keys(ci, r, k, base);
+                const unsigned bits = kept_all(k, p, tie_run, unused);
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    if (bits & (1u << e)) {
+                        const double y = ((double)Tr::value_f(k[e]) - lmax) * inv_tau;
+                        const double m = exp_nonpos(y, sm.exp_tbl);
+                        if (m > 0.0) acc += m * y;
+                    }
+                }
+            }
+        }
+        acc = warp_sum_d(acc);
+        if (lane == 0) sm.red_d[warp] = acc;
+        Sync::sync();
+        double tot = 0.0;
+        for (int w = 0; w < NW; ++w) tot += sm.red_d[w];
+        Sync::sync();
+        tp.mu = tot / Z1;
+        // mass-weighted radix select on the 64-bit order key, 8 bits at a time
+        const double target = typical_p * Z1;
+        unsigned long long prefix = 0, mask = 0;
+        int acc_c = 0, eq = 0;
+        double acc_m = 0.0, eq_m = 0.0;
+        const int rep = lane & (HIST_REP - 1);
+        for (int shift = 56; shift >= 0; shift -= 8) {
+            for (int i = tid; i < 256 * HIST_REP; i += NT) { sm.hist_cnt[i] = 0; sm.hist_mass[i] = 0.0; }
+            Sync::sync();
+            int cur_d = -1, cur_n = 0;
+            double cur_m = 0.0;
+            for (int ci = warp; ci < nchunks; ci += NW) {
+                int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[ci] : 0, unused = 0;
+                for (int r = 0; r < R; ++r) {
+                    uint32_t k[E];
+                    int base;
+                    chunk_keys(ci, r, k, base);
+                    const unsigned bits = kept_all(k, p, tie_run, unused);
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        if (bits & (1u << e)) {
+                            const unsigned long long t = tkey(k[e]);
+                            if ((t & mask) == prefix) {
+                                const int d = (int)((t >> shift) & 255ull);
+                                if (d != cur_d) {
+                                    if (cur_n) {
+                                        atomicAdd(&sm.hist_cnt[ASX_AT(cur_d * HIST_REP + rep, 256 * HIST_REP, 80)], cur_n);
+                                        atomicAdd(&sm.hist_mass[ASX_AT(cur_d * HIST_REP + rep, 256 * HIST_REP, 81)], cur_m);
+                                    }
+                                    cur_d = d; cur_n = 0; cur_m = 0.0;
+                                }
+                                ++cur_n;
+                                cur_m += mass(k[e]);
+                            }
+                        }
+                    }
+                }
+            }
+            if (cur_n) {
+                atomicAdd(&sm.hist_cnt[ASX_AT(cur_d * HIST_REP + rep, 256 * HIST_REP, 80)], cur_n);
+                atomicAdd(&sm.hist_mass[ASX_AT(cur_d * HIST_REP + rep, 256 * HIST_REP, 81)], cur_m);
+            }
+            Sync::sync();
+            choose_digit<true>(acc_c, acc_m, 0, target);
+            prefix |= (unsigned long long)sm.b_i[0] << shift;
+            mask |= 0xFFull << shift;
+            acc_c = sm.b_i[1];
+            eq = sm.b_i[2];
+            acc_m = sm.b_d[0];
+            eq_m = sm.b_d[1];
+            Sync::sync();
+        }
+        // `eq` kept elements share the threshold key (equal logits: equal masses): take the fewest
+        // of them, lowest indices first, that bring the mass to the target
+        const double e_P = eq_m / (double)eq;
+        long long r = (long long)ceil((target - acc_m) / e_P);
+        if (r < 1) r = 1;
+        if (r > eq) r = eq;
+        while (r > 1 && acc_m + (double)(r - 1) * e_P >= target) --r;
+        while (r < eq && acc_m + (double)r * e_P < target) ++r;
+        // ties at the threshold, per chunk, among the elements kept so far
+        for (int ci = warp; ci < nchunks; ci += NW) {
+            int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[ci] : 0, unused = 0;
+            int cnt = 0;
+            for (int rr = 0; rr < R; ++rr) {
+                uint32_t k[E];
+                int base;
+                chunk_keys(ci, rr, k, base);
+                const unsigned bits = kept_all(k, p, tie_run, unused);
+#pragma unroll
+                for (int e = 0; e < E; ++e)
+                    if ((bits & (1u << e)) && tkey(k[e]) == prefix) ++cnt;
+            }
+            cnt = warp_sum_i(cnt);
+            if (lane == 0) sm.chunk_eq2[ci] = cnt;
+        }
+        Sync::sync();
+        scan_exclusive(sm.chunk_eq2, nchunks);
+        tp.T = prefix;
+        tp.need = (int)r;
+        tp.eq_mode = ((int)r < eq) ? 2 : 1;
+        tp.on = 1;
+        n_kept = acc_c + (int)r;
+    }
+
     // Steps 1-4 of the general routine: the kept set as a predicate `p`, its size, and in
     // chunk_sum the exclusive scan of the kept masses per chunk (chunk_sum[nchunks] = Z).
     // Needs inv_tau set and the exp table filled; returns ST_OK or ST_NUMERIC.
-    __device__ __forceinline__ int prepare(int top_k, double top_p, Pred& p, int& n_kept) {
+    __device__ __forceinline__ int prepare(int top_k, double top_p, Pred& p, int& n_kept, double typical_p = 1.0) {
         // ---- 1. extremes and finite count
         unsigned kmax = 0, kmin = 0xFFFFFFFFu;
         int nfin = 0;
@@ -544,6 +728,15 @@ struct GenericLane {
         sum_pass(p);
         scan_exclusive(sm.chunk_sum, nchunks);
 
+        // ---- 3b. locally typical cut on the distribution over the survivors (it takes the
+        //          nucleus's place): tokens ordered by |y - mu| ascending, mu = sum p_j y_j
+        if (typical_p > 0.0 && typical_p < 1.0) {
+            typical_cut(p, typical_p, n_kept);
+            sum_pass(p);
+            scan_exclusive(sm.chunk_sum, nchunks);
+            return ST_OK;
+        }
+
         // ---- 4. nucleus on the distribution renormalised over the survivors
         if (top_p > 0.0 && top_p < 1.0) {
             const double target = top_p * sm.chunk_sum[nchunks];
@@ -589,8 +782,9 @@ struct GenericLane {
         return ST_OK;
     }
 
-    __device__ __noinline__ LaneResult run(double c_in, double inv_tau_, int top_k, double top_p) {
-        if (top_k <= 0 && !(top_p > 0.0 && top_p < 1.0) && vec_ok) return run_nocut(c_in, inv_tau_);
+    __device__ __noinline__ LaneResult run(double c_in, double inv_tau_, int top_k, double top_p, double typical_p = 1.0) {
+        const bool typical = typical_p > 0.0 && typical_p < 1.0;
+        if (top_k <= 0 && !(top_p > 0.0 && top_p < 1.0) && !typical && vec_ok) return run_nocut(c_in, inv_tau_);
         inv_tau = inv_tau_;
         fill_exp_table(sm.exp_tbl, tid);
         double c = c_in;
@@ -598,7 +792,7 @@ struct GenericLane {
         if (c == 1.0) c = ASX_ONE_BELOW;
         Pred p;
         int n_kept;
-        if (prepare(top_k, top_p, p, n_kept) != ST_OK || code_bad) return fail(c_in, ST_NUMERIC);
+        if (prepare(top_k, top_p, p, n_kept, typical_p) != ST_OK || code_bad) return fail(c_in, ST_NUMERIC);
 
         // ---- 5/6. locate the chunk, then the element
         const double Z = sm.chunk_sum[nchunks];
@@ -606,10 +800,9 @@ struct GenericLane {
         if (tid == 0) { sm.b_i[0] = INT_MAX; sm.b_i[1] = -1; }
         Sync::sync();
         for (int ci = tid; ci < nchunks; ci += NT) {
-            const double excl = sm.chunk_sum[ci], incl = sm.chunk_sum[ci + 1];
-            if (incl > excl) {
+            if (has_mass(ci)) {
                 atomicMax(&sm.b_i[1], ci);
-                if (t < incl) atomicMin(&sm.b_i[0], ci);
+                if (t < sm.chunk_sum[ci + 1]) atomicMin(&sm.b_i[0], ci);
             }
         }
         Sync::sync();
@@ -617,8 +810,9 @@ struct GenericLane {
         const int cstar = force_last ? sm.b_i[1] : sm.b_i[0];
 
         if (warp == 0) {
-            double run = sm.chunk_sum[cstar];
+            double run = sm.chunk_sum[ASX_AT(cstar, MAXCH + 1, 84)];
             int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[cstar] : 0;
+            int tie_run2 = (tp.on && tp.eq_mode == 2) ? sm.chunk_eq2[cstar] : 0;
             int last_idx = -1;
             double last_S = 0.0, last_e = 1.0;
             int tok = -1;
@@ -627,8 +821,7 @@ struct GenericLane {
                 uint32_t k[E];
                 int base;
                 chunk_keys(cstar, r, k, base);
-                const int rank0 = lane_rank0(k, p, tie_run);
-                const unsigned bits = kept_bits(k, p, rank0);
+                const unsigned bits = kept_all(k, p, tie_run, tie_run2);
                 double ev[E];
                 double local = 0.0;
 #pragma unroll
@@ -690,7 +883,7 @@ struct GenericLane {
     }
 
     // One step with an extended-precision code: the token that owns cell `tcell` of the 2^32 cells
-    // of this step's CDF over the kept set (any cut), with its cells in the result's xp_lo / xp_hi.
+    // of this step's CDF over the kept set (any cut), with its cells in sm.xp_lo / sm.xp_hi.
     __device__ __noinline__ LaneResult run_xp(unsigned long long tcell, double inv_tau_, int top_k, double top_p) {
         inv_tau = inv_tau_;
         fill_exp_table(sm.exp_tbl, tid);
@@ -702,7 +895,7 @@ struct GenericLane {
             const double K = 4294967296.0 / Z;
             int last_c = -1;
             for (int ci = lane; ci < nchunks; ci += 32)
-                if (sm.chunk_sum[ci + 1] > sm.chunk_sum[ci]) last_c = ci;
+                if (has_mass(ci)) last_c = ci;
             last_c = (int)warp_max_u((unsigned)(last_c + 1)) - 1;
             int tok = -1;
             unsigned long long plo = 0, phi = 0;
@@ -711,7 +904,7 @@ struct GenericLane {
                 int first = INT_MAX;
                 for (int ci = lane; ci <= last_c; ci += 32) {
                     const unsigned long long fe = ci == last_c ? XP_TOP : xp_cell(sm.chunk_sum[ci + 1], K);
-                    if (fe > tcell && sm.chunk_sum[ci + 1] > sm.chunk_sum[ci]) first = min(first, ci);
+                    if (fe > tcell && has_mass(ci)) first = min(first, ci);
                 }
                 const int cstar = (int)warp_min_u((unsigned)first);
                 const unsigned long long Fend = cstar == last_c ? XP_TOP : xp_cell(sm.chunk_sum[cstar + 1], K);
@@ -739,7 +932,12 @@ struct GenericLane {
                     }
                 }
                 double run = sm.chunk_sum[cstar];
-                unsigned long long carry = xp_cell(run, K);
+                // the chunk starts in the cell where the chunk with mass before it ended
+                int prev_c = -1;
+                for (int ci = lane; ci < cstar; ci += 32)
+                    if (has_mass(ci)) prev_c = ci;
+                prev_c = (int)warp_max_u((unsigned)(prev_c + 1)) - 1;
+                unsigned long long carry = prev_c < 0 ? 0ull : xp_cell(sm.chunk_sum[prev_c + 1], K);
                 int tie_run = (p.eq_mode == 2) ? sm.chunk_eq[cstar] : 0;
                 for (int r = 0; r <= r_last && tok < 0; ++r) {
                     double ev[E];
@@ -756,7 +954,7 @@ struct GenericLane {
                 r.code_out = 0.0;
                 r.p_tok = pe / sm.chunk_sum[nchunks];
                 r.cdf_lo = (double)plo * (1.0 / 4294967296.0);
-                r.xp_lo = plo; r.xp_hi = phi;
+                sm.xp_lo = plo; sm.xp_hi = phi;
                 sm.res = r;
             }
         }

@@ -35,7 +35,8 @@ constexpr int NC_MAXG = 3;                        // groups per CTA
 constexpr int NC_PIECE_BYTES = 16384;
 constexpr int NC_MAXPIECE = 6;
 constexpr int NC_MAXROW = NC_MAXPIECE * NC_PIECE_BYTES;        // rows up to 96 KB
-constexpr int NC_MAXCH = NC_MAXROW / 16 / 32;                  // 192 chunks
+constexpr int NC_R = 4;                           // sub-rows of 32 vectors per chunk
+constexpr int NC_MAXCH = NC_MAXROW / 16 / 32 / NC_R;           // 48 chunks
 constexpr int NC_EXP_LO = 119;                    // biased exponent of 2^-8
 constexpr int NC_BINADES = 14;                    // [2^-8, 2^6)
 constexpr int NC_ENT = NC_BINADES * 128;          // table entries per sign
@@ -89,7 +90,10 @@ struct NcGroupSmem {
     int flags;
     int masked;          // table mode: -inf elements (padding included); robust mode: finite elements
     int poisoned;
+    unsigned long long has;      // bit c: chunk c holds mass (not to be read off the scanned sums, whose
+                                 // lane totals are added in another order than the sums inside a lane)
     LaneResult res;
+    unsigned long long xp_lo, xp_hi;     // extended-precision steps: the chosen token's cells [xp_lo, xp_hi)
 };
 
 // shared memory in front of the row buffers: mass table, 2^(j/64) table, the groups' control blocks
@@ -127,9 +131,13 @@ struct NcRow {
         if (!mbar_wait_bounded(smem_u32(&g.full[p]), parity, wait_cycles)) *(volatile int*)&g.poisoned = 1;
     }
 
+    __device__ __forceinline__ static uint4 ninf_vec() {
+        const uint32_t w = DT == DT_BF16 ? 0xFF80FF80u : 0xFF800000u;
+        return make_uint4(w, w, w, w);
+    }
     // vector v of the row; elements at or past V read as -inf
     __device__ __forceinline__ uint4 load_vec(int v) const {
-        if (v < bulk_vec) return rowv[v];
+        if (v < bulk_vec) return rowv[ASX_AT(v, NC_MAXROW / 16, 70)];
         uint32_t w[4];
         const int base = v * E;
         if (DT == DT_BF16) {
@@ -174,7 +182,7 @@ struct NcRow {
             bad |= (ok0 ? 0u : 1u) << (2 * i) | (ok1 ? 0u : 1u) << (2 * i + 1);
         }
 #pragma unroll
-        for (int k = 0; k < 8; ++k) e[k] = tbl[idx[k]];
+        for (int k = 0; k < 8; ++k) e[k] = tbl[ASX_AT(idx[k], NC_TBL_DOUBLES, 71)];
         if (bad) {
 #pragma unroll
             for (int k = 0; k < 8; ++k)
@@ -198,22 +206,33 @@ struct NcRow {
     }
 
     // ---- per-chunk sums in index order.  g.flags / g.masked must be zero on entry (group-wide).
+    //      A chunk is NC_R sub-rows of 32 vectors; a warp takes the NC_R vectors of a lane at once,
+    //      so that their table loads are in flight together and one reduction serves them all.
     template <bool TBL>
     __device__ void sum_pass() {
         int flags = 0, count = 0, cur = -1;
         for (int c = warp; c < nch; c += NC_GW) {
-            const int piece = (c * 512) / NC_PIECE_BYTES;
+            const int piece = (c * NC_R * 512) / NC_PIECE_BYTES;
             if (piece != cur && piece < npiece) { wait_piece(piece); cur = piece; }
-            const int v = c * 32 + lane;
+            uint4 q[NC_R];
+#pragma unroll
+            for (int r = 0; r < NC_R; ++r) {
+                const int v = (c * NC_R + r) * 32 + lane;
+                q[r] = v < nvec ? load_vec(v) : ninf_vec();
+            }
             double s = 0.0;
-            if (v < nvec) {
+#pragma unroll
+            for (int r = 0; r < NC_R; ++r) {
                 double e[E];
-                masses<TBL>(load_vec(v), e, flags, count);
-                if constexpr (E == 8) s = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
-                else s = (e[0] + e[1]) + (e[2] + e[3]);
+                masses<TBL>(q[r], e, flags, count);
+                if constexpr (E == 8) s += ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+                else s += (e[0] + e[1]) + (e[2] + e[3]);
             }
             s = warp_sum_d(s);
-            if (lane == 0) g.chunk_sum[c] = s;
+            if (lane == 0) {
+                g.chunk_sum[ASX_AT(c, NC_MAXCH + 1, 72)] = s;
+                if (s > 0.0) atomicOr(&g.has, 1ull << c);
+            }
         }
         flags = __reduce_or_sync(FULL, flags);
         count = __reduce_add_sync(FULL, count);
@@ -259,6 +278,15 @@ struct NcRow {
         __syncwarp();
     }
 
+    // masses of sub-row r of chunk c for this lane (zeros past the row)
+    template <bool TBL>
+    __device__ __forceinline__ int sub_masses(int c, int r, double (&ev)[E]) const {
+        const int v = (c * NC_R + r) * 32 + lane;
+        int f = 0, cnt = 0;
+        masses<TBL>(v < nvec ? load_vec(v) : ninf_vec(), ev, f, cnt);
+        return v * E;
+    }
+
     // ---- warp 0: the token whose interval holds c * Z, and the rescaled code
     template <bool TBL>
     __device__ void locate(double c, double c_in, int n_kept) {
@@ -267,10 +295,9 @@ struct NcRow {
         const double t = c * Z;
         int first = INT_MAX, last_c = -1;
         for (int ci = lane; ci < nch; ci += 32) {
-            const double excl = g.chunk_sum[ci], incl = g.chunk_sum[ci + 1];
-            if (incl > excl) {
+            if ((g.has >> ci) & 1ull) {
                 last_c = ci;
-                if (t < incl) first = min(first, ci);
+                if (t < g.chunk_sum[ci + 1]) first = min(first, ci);
             }
         }
         first = (int)warp_min_u((unsigned)first);
@@ -280,39 +307,41 @@ struct NcRow {
         int tok = -1;
         double tok_S = 0.0, tok_e = 1.0;
         if (cstar >= 0) {
-            const double run = g.chunk_sum[cstar];
-            const int v = cstar * 32 + lane;
-            double ev[E];
+            double run = g.chunk_sum[ASX_AT(cstar, NC_MAXCH + 1, 73)];
+            int last_idx = -1;
+            double last_S = 0.0, last_e = 1.0;
+            for (int r = 0; r < NC_R && tok < 0; ++r) {
+                double ev[E];
+                const int base = sub_masses<TBL>(cstar, r, ev);
+                double local = 0.0;
 #pragma unroll
-            for (int k = 0; k < E; ++k) ev[k] = 0.0;
-            int f = 0, cnt = 0;
-            if (v < nvec) masses<TBL>(load_vec(v), ev, f, cnt);
-            double local = 0.0;
+                for (int k = 0; k < E; ++k) local += ev[k];
+                const double incl = warp_incl_scan_d(local, lane);
+                double excl = __shfl_up_sync(FULL, incl, 1);
+                if (lane == 0) excl = 0.0;
+                int pick = -1;
+                double pick_S = 0.0, pick_e = 1.0;
+                double S = run + excl;
 #pragma unroll
-            for (int k = 0; k < E; ++k) local += ev[k];
-            const double incl = warp_incl_scan_d(local, lane);
-            double excl = __shfl_up_sync(FULL, incl, 1);
-            if (lane == 0) excl = 0.0;
-            int pick = -1, last_idx = -1;
-            double pick_S = 0.0, pick_e = 1.0, last_S = 0.0, last_e = 1.0;
-            double S = run + excl;
-#pragma unroll
-            for (int k = 0; k < E; ++k) {
-                if (ev[k] > 0.0) {
-                    if (pick < 0 && t < S + ev[k]) { pick = v * E + k; pick_S = S; pick_e = ev[k]; }
-                    last_idx = v * E + k; last_S = S; last_e = ev[k];
-                    S += ev[k];
+                for (int k = 0; k < E; ++k) {
+                    if (ev[k] > 0.0) {
+                        if (pick < 0 && t < S + ev[k]) { pick = base + k; pick_S = S; pick_e = ev[k]; }
+                        last_idx = base + k; last_S = S; last_e = ev[k];
+                        S += ev[k];
+                    }
                 }
+                const bool cross = !force_last && local > 0.0 && (t < run + incl);
+                const unsigned bal = __ballot_sync(FULL, cross);
+                if (bal) {
+                    const int L = __ffs(bal) - 1;
+                    if (pick < 0) { pick = last_idx; pick_S = last_S; pick_e = last_e; }
+                    tok = __shfl_sync(FULL, pick, L);
+                    tok_S = __shfl_sync(FULL, pick_S, L);
+                    tok_e = __shfl_sync(FULL, pick_e, L);
+                }
+                run += __shfl_sync(FULL, incl, 31);
             }
-            const bool cross = !force_last && local > 0.0 && (t < run + incl);
-            const unsigned bal = __ballot_sync(FULL, cross);
-            if (bal) {
-                const int L = __ffs(bal) - 1;
-                if (pick < 0) { pick = last_idx; pick_S = last_S; pick_e = last_e; }
-                tok = __shfl_sync(FULL, pick, L);
-                tok_S = __shfl_sync(FULL, pick_S, L);
-                tok_e = __shfl_sync(FULL, pick_e, L);
-            } else {   // rounding at the top end: the last token with mass in the chunk
+            if (tok < 0) {   // rounding at the top end: the last token with mass in the chunk
                 const unsigned best = warp_max_u((unsigned)(last_idx + 1));
                 const unsigned bal2 = __ballot_sync(FULL, (unsigned)(last_idx + 1) == best);
                 const int L = __ffs(bal2) - 1;
@@ -335,7 +364,7 @@ struct NcRow {
     }
 
     // ---- warp 0: the token that owns the cell `tcell` of the 2^32 cells of this step's CDF
-    //      (extended-precision codes); the result carries the token's cells [xp_lo, xp_hi)
+    //      (extended-precision codes); the token's cells go to g.xp_lo / g.xp_hi
     template <bool TBL>
     __device__ void locate_xp(unsigned long long tcell, int n_kept) {
         scan_chunks();
@@ -343,7 +372,7 @@ struct NcRow {
         const double K = 4294967296.0 / Z;
         int last_c = -1;
         for (int ci = lane; ci < nch; ci += 32)
-            if (g.chunk_sum[ci + 1] > g.chunk_sum[ci]) last_c = ci;
+            if ((g.has >> ci) & 1ull) last_c = ci;
         last_c = (int)warp_max_u((unsigned)(last_c + 1)) - 1;
         int tok = -1;
         unsigned long long plo = 0, phi = 0;
@@ -353,21 +382,32 @@ struct NcRow {
             int first = INT_MAX;
             for (int ci = lane; ci <= last_c; ci += 32) {
                 const unsigned long long fe = ci == last_c ? XP_TOP : xp_cell(g.chunk_sum[ci + 1], K);
-                if (fe > tcell && g.chunk_sum[ci + 1] > g.chunk_sum[ci]) first = min(first, ci);
+                if (fe > tcell && ((g.has >> ci) & 1ull)) first = min(first, ci);
             }
             const int cstar = (int)warp_min_u((unsigned)first);
             const unsigned long long Fend = cstar == last_c ? XP_TOP : xp_cell(g.chunk_sum[cstar + 1], K);
-            double run = g.chunk_sum[cstar];
-            unsigned long long carry = xp_cell(run, K);
-            const int v = cstar * 32 + lane;
-            double ev[E];
+            // the last sub-row of the chunk that holds mass
+            int r_last = 0;
+            for (int r = 0; r < NC_R; ++r) {
+                double ev[E];
+                sub_masses<TBL>(cstar, r, ev);
+                double local = 0.0;
 #pragma unroll
-            for (int k = 0; k < E; ++k) ev[k] = 0.0;
-            int f = 0, cnt = 0;
-            if (v < nvec) masses<TBL>(load_vec(v), ev, f, cnt);
-            int pk = 0;
-            const int L = xp_subrow<E>(ev, lane, K, tcell, true, Fend, run, carry, pk, plo, phi, pe);
-            if (L >= 0) tok = (cstar * 32 + L) * E + pk;
+                for (int k = 0; k < E; ++k) local += ev[k];
+                if (__ballot_sync(FULL, local > 0.0)) r_last = r;
+            }
+            double run = g.chunk_sum[cstar];
+            // the chunk starts in the cell where the chunk with mass before it ended
+            const unsigned long long before = g.has & ((1ull << cstar) - 1ull);
+            const unsigned long long carry0 = before ? xp_cell(g.chunk_sum[64 - __clzll((long long)before)], K) : 0ull;
+            unsigned long long carry = carry0;
+            for (int r = 0; r <= r_last && tok < 0; ++r) {
+                double ev[E];
+                const int base = sub_masses<TBL>(cstar, r, ev);
+                int pk = 0;
+                const int L = xp_subrow<E>(ev, lane, K, tcell, r == r_last, Fend, run, carry, pk, plo, phi, pe);
+                if (L >= 0) tok = __shfl_sync(FULL, base, L) + pk;
+            }
         }
         if (lane == 0) {
             LaneResult r;
@@ -375,7 +415,7 @@ struct NcRow {
             r.code_out = 0.0;
             r.p_tok = pe / Z;
             r.cdf_lo = (double)plo * (1.0 / 4294967296.0);
-            r.xp_lo = plo; r.xp_hi = phi;
+            g.xp_lo = plo; g.xp_hi = phi;
             g.res = r;
         }
     }
@@ -385,18 +425,17 @@ struct NcRow {
     __device__ void interval(int tok, int n_kept) {
         scan_chunks();
         const double Z = g.chunk_sum[nch];
-        const int cstar = (tok / E) >> 5;
-        const int v = cstar * 32 + lane;
-        double ev[E];
-#pragma unroll
-        for (int k = 0; k < E; ++k) ev[k] = 0.0;
-        int f = 0, cnt = 0;
-        if (v < nvec) masses<TBL>(load_vec(v), ev, f, cnt);
+        const int cstar = (tok / E) / (32 * NC_R);
         double below = 0.0, e_tok = 0.0;
+        for (int r = 0; r < NC_R; ++r) {
+            if ((cstar * NC_R + r) * 32 * E > tok) break;      // warp-uniform: sub-rows past the token
+            double ev[E];
+            const int base = sub_masses<TBL>(cstar, r, ev);
 #pragma unroll
-        for (int k = 0; k < E; ++k) {
-            if (v * E + k < tok) below += ev[k];
-            if (v * E + k == tok) e_tok = ev[k];
+            for (int k = 0; k < E; ++k) {
+                if (base + k < tok) below += ev[k];
+                if (base + k == tok) e_tok = ev[k];
+            }
         }
         below = warp_sum_d(below);
         e_tok = warp_sum_d(e_tok);                 // one lane holds it, the others add zero
@@ -409,7 +448,7 @@ struct NcRow {
             r.token = kept ? tok : -1; r.status = kept ? ST_OK : ST_NUMERIC; r.n_kept = n_kept;
             r.code_out = 0.0;
             r.p_tok = e_tok / Z;
-            r.cdf_lo = (g.chunk_sum[cstar] + below) / Z;
+            r.cdf_lo = (g.chunk_sum[ASX_AT(cstar, NC_MAXCH + 1, 74)] + below) / Z;
             g.res = r;
         }
     }
@@ -429,7 +468,7 @@ struct NcRow {
             if (flags & NCF_BAD) failed = true;
             else if (flags & NCF_BIG) robust = true;
             if (!failed && !robust && warp == 0 && !g.poisoned) {
-                const int n_kept = nvec * E - g.masked;
+                const int n_kept = nch * NC_R * 32 * E - g.masked;       // (padding counts as masked)
                 if (n_kept <= 0) { if (lane == 0) g.res = failed_lane(c_in, ST_NUMERIC); }
                 else if (xp) locate_xp<true>(tcell, n_kept);
                 else if (tok_given < 0) locate<true>(c, c_in, n_kept);
@@ -437,7 +476,7 @@ struct NcRow {
             }
             if (robust) {                                        // (the counters start again)
                 nc_bar<NC_GT>(gi);
-                if (gtid == 0) { g.flags = 0; g.masked = 0; }
+                if (gtid == 0) { g.flags = 0; g.masked = 0; g.has = 0ull; }
                 nc_bar<NC_GT>(gi);
             }
         }
@@ -463,7 +502,7 @@ struct NcRow {
         }
         nc_bar<NC_GT>(gi);
         const LaneResult out = g.res;
-        if (gtid == 0) { g.flags = 0; g.masked = 0; }
+        if (gtid == 0) { g.flags = 0; g.masked = 0; g.has = 0ull; }
         nc_bar<NC_GT>(gi);          // the buffer and the result slot are free again
         return out;
     }
@@ -484,7 +523,7 @@ __global__ void __launch_bounds__(NC_MAXG * NC_GT, 1) nocut_kernel(const NocutAr
     fill_exp_table(exp_tbl, tid);
     if (gtid == 0) {
         for (int p = 0; p < NC_MAXPIECE; ++p) mbar_init(smem_u32(&g.full[p]), 1);
-        g.flags = 0; g.masked = 0; g.poisoned = 0;
+        g.flags = 0; g.masked = 0; g.poisoned = 0; g.has = 0ull;
     }
     if (tid == 0) fence_mbar_init();
     __syncthreads();
@@ -505,7 +544,7 @@ __global__ void __launch_bounds__(NC_MAXG * NC_GT, 1) nocut_kernel(const NocutAr
     R.nvec = (V + Tr::E - 1) / Tr::E;
     const int bulk_bytes = (V * Tr::BYTES) & ~15;
     R.bulk_vec = bulk_bytes >> 4;
-    R.nch = (R.nvec + 31) / 32;
+    R.nch = (R.nvec + 32 * NC_R - 1) / (32 * NC_R);
     R.npiece = (bulk_bytes + NC_PIECE_BYTES - 1) / NC_PIECE_BYTES;
     R.gi = gi; R.gtid = gtid; R.lane = gtid & 31; R.warp = gtid >> 5;
     R.inv_tau = a.inv_tau; R.s64 = 0.0; R.c64 = 0.0;
@@ -608,7 +647,7 @@ __global__ void __launch_bounds__(NC_MAXG * NC_GT, 1) nocut_kernel(const NocutAr
                     const LaneResult r = R.run(0.0, -1, a.use_table != 0, true, xp_target(xs));
                     row_done();
                     if (r.status != ST_OK) { status = r.status; break; }
-                    xp_advance(xs, r.xp_lo, r.xp_hi, (unsigned)a.N);
+                    xp_advance(xs, g.xp_lo, g.xp_hi, (unsigned)a.N);
                     if (gtid == 0) a.seq[(size_t)ln * a.T + t] = r.token;
                     n = t + 1;
                     prev = r.token;

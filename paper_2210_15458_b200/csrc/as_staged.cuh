@@ -263,7 +263,7 @@ __device__ bool epilogue(StagedSmem<NT>& sm, int C, double c, double c_in, doubl
         const unsigned long long ci = sm.cand[i];
         int r = 0;
         for (int j = 0; j < C; ++j) r += (sm.cand[j] > ci);
-        ep.order[r] = (unsigned short)i;
+        ep.order[ASX_AT(r, ST_CAP, 91)] = (unsigned short)i;
     }
     __syncthreads();
     ASX_MARK(8);
@@ -310,8 +310,8 @@ __device__ bool epilogue(StagedSmem<NT>& sm, int C, double c, double c_in, doubl
         const uint32_t idx = ~(uint32_t)sm.cand[ep.order[r]];
         int ir = 0;
         for (int q = 0; q < n_final; ++q) ir += (~(uint32_t)sm.cand[ep.order[q]] < idx);
-        ep.e_idx[ir] = ep.e[r];
-        ep.tok_idx[ir] = (int)idx;
+        ep.e_idx[ASX_AT(ir, ST_CAP, 92)] = ep.e[r];
+        ep.tok_idx[ASX_AT(ir, ST_CAP, 93)] = (int)idx;
     }
     __syncthreads();
     ASX_MARK(11);
@@ -542,7 +542,7 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
         const float lmaxf = Tr::value_f(gmax);
         float tail = 0.f;
         for (int v = tid; v < my_nvec; v += NT) {
-            const uint4 q = rowv[v];
+            const uint4 q = rowv[ASX_AT(v, ST_MAXCHUNK * ST_CHUNK_VEC, 94)];
             if (!want_tail) {
                 if (P::vmax(q) >= t0f) {
                     float x[E];
@@ -553,7 +553,7 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
                         if (x[e] >= t0f && key >= gt0 && key > Tr::KEY_NINF) {
                             const int slot = atomicAdd(&lead->cand_count, 1);
                             if (slot < ST_CAP)
-                                lead->cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)((v0 + v) * E + e);
+                                lead->cand[ASX_AT(slot, ST_CAP, 90)] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)((v0 + v) * E + e);
                         }
                     }
                 }
@@ -570,7 +570,7 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
                             pushed = true;
                             const int slot = atomicAdd(&lead->cand_count, 1);
                             if (slot < ST_CAP)
-                                lead->cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)((v0 + v) * E + e);
+                                lead->cand[ASX_AT(slot, ST_CAP, 90)] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)((v0 + v) * E + e);
                         }
                     }
                     tail += pushed ? 0.f : ev;

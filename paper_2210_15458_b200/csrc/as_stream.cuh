@@ -164,9 +164,9 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
             if (valid) {
                 // with a top-k alone nothing past rank kmax is looked at again: zeros there, which
                 // the index loop below relies on
-                if (sub == 0) dst[r] = (topk_only && r >= kmax) ? 0ull : ci;
+                if (sub == 0) dst[ASX_AT(r, SK_CAP + 4, 10)] = (topk_only && r >= kmax) ? 0ull : ci;
                 if (sub == (G > 1 ? 1 : 0))
-                    e[r] = exp_nonpos(((double)Tr::value_f((uint32_t)(ci >> 32)) - lmax) * inv_tau, sm.exp_tbl);
+                    e[ASX_AT(r, SK_CAP, 11)] = exp_nonpos(((double)Tr::value_f((uint32_t)(ci >> 32)) - lmax) * inv_tau, sm.exp_tbl);
             }
         }
     }
@@ -196,7 +196,7 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
             } else {
                 nf = below + 1;
             }
-            if (okw && (uint32_t)(dst[nf - 1] >> 32) < depth_key) okw = 0;   // cut below the exact depth
+            if (okw && (uint32_t)(dst[ASX_AT(nf - 1, SK_CAP + 4, 12)] >> 32) < depth_key) okw = 0;   // cut below the exact depth
             __syncwarp();
             if (lane == 0) {
                 sm.b_i[0] = nf; sm.b_i[1] = okw;
@@ -211,7 +211,7 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
         // top-k only: the answer follows from kmax alone, every thread sees it; the entries past
         // the kept ranks were stored as zeros
         n_final = kmax;
-        ok = ((uint32_t)(dst[kmax - 1] >> 32) >= depth_key) ? 1 : 0;
+        ok = ((uint32_t)(dst[ASX_AT(kmax - 1, SK_CAP + 4, 13)] >> 32) >= depth_key) ? 1 : 0;
     }
     ASX_MARK(7);
     if (ok) {
@@ -228,7 +228,7 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
                 ir += (~(uint32_t)dst[q] < idx) + (~(uint32_t)dst[q + 1] < idx) +
                       (~(uint32_t)dst[q + 2] < idx) + (~(uint32_t)dst[q + 3] < idx);
             for (int o = G >> 1; o > 0; o >>= 1) ir += __shfl_xor_sync(FULL, ir, o);
-            if (valid && sub == 0) src[ir] = ((unsigned long long)idx << 32) | (uint32_t)r;
+            if (valid && sub == 0) src[ASX_AT(ir, SK_CAP + 4, 14)] = ((unsigned long long)idx << 32) | (uint32_t)r;
         }
         Sync::sync();
         ASX_MARK(8);
@@ -241,9 +241,9 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
             if (per <= 4) {
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
-                    if (b + k < en) { ev4[k] = e[(uint32_t)src[b + k]]; s += ev4[k]; }
+                    if (b + k < en) { ev4[k] = e[ASX_AT((uint32_t)src[b + k], SK_CAP, 15)]; s += ev4[k]; }
             } else {
-                for (int i = b; i < en; ++i) s += e[(uint32_t)src[i]];
+                for (int i = b; i < en; ++i) s += e[ASX_AT((uint32_t)src[i], SK_CAP, 16)];
             }
             const double incl = warp_incl_scan_d(s, lane);
             double run = __shfl_up_sync(FULL, incl, 1);
@@ -291,7 +291,7 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
                 if (!(cn >= 0.0)) cn = 0.0;
                 if (cn > ASX_ONE_BELOW) cn = ASX_ONE_BELOW;
                 LaneResult r;
-                r.token = (int)(src[pick] >> 32); r.status = ST_OK; r.n_kept = n_final; r.code_out = cn;
+                r.token = (int)(src[ASX_AT(pick, SK_CAP + 4, 17)] >> 32); r.status = ST_OK; r.n_kept = n_final; r.code_out = cn;
                 r.p_tok = p_tok; r.cdf_lo = cdf_lo;
                 out = r;
             }
@@ -325,7 +325,7 @@ __device__ __forceinline__ void reread_row(uint4* staging, const char* row, int 
     int slot = 0;
     for (int v = tid; v < nvec_full; v += SK_NT) {
         asm volatile("cp.async.wait_group %0;" ::"n"(D - 1) : "memory");
-        const uint4 q = mine[slot * SK_NT];
+        const uint4 q = mine[ASX_AT(slot, D, 60) * SK_NT];
         f(q, v);
         copy(slot, v + D * SK_NT);                 // after f: the slot's value has been consumed
         slot = slot + 1 == D ? 0 : slot + 1;
@@ -385,8 +385,8 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2,
             const float d = (y0 - y) * DP_BINS_PER_UNIT;
             if (d < (float)DP_NB) {
                 const int bin = (int)d;
-                atomicAdd(&hcnt[bin], 1);
-                atomicAdd(&hmass[bin], ex2_approx(y));
+                atomicAdd(&hcnt[ASX_AT(bin, DP_NB, 20)], 1);
+                atomicAdd(&hmass[ASX_AT(bin, DP_NB, 21)], ex2_approx(y));
             }
         }
     });
@@ -436,7 +436,7 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2,
             const uint32_t key = P::key_of_f(x);
             if (key > Tr::KEY_NINF) {
                 const int slot = atomicAdd(&sm.cand_count, 1);
-                if (slot < SK_CAP) sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)j;
+                if (slot < SK_CAP) sm.u.ep.cand[ASX_AT(slot, SK_CAP + 4, 30)] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)j;
                 if (x < t0f) joined += ex2_approx((x - lmaxf) * scale2);
             }
         }
@@ -476,7 +476,7 @@ __device__ __noinline__ float recollect_row(StreamSmem& sm, int V, const char* r
             if (key >= t0key && key > Tr::KEY_NINF) {
                 hit = true;
                 const int slot = atomicAdd(&sm.cand_count, 1);
-                if (slot < SK_CAP) sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)j;
+                if (slot < SK_CAP) sm.u.ep.cand[ASX_AT(slot, SK_CAP + 4, 30)] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)j;
             }
         }
         if (!hit) tail += ex2_approx((x - ref) * scale2);
@@ -705,8 +705,8 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                 if ((hm >> j) & 1u) {
                     const int slot = base + __popc(bal[j] & ((1u << lane) - 1u));
                     if (slot < SK_CAPV) {
-                        sm.u.ep.v.cvec[slot] = q[j];
-                        sm.u.ep.cidx[slot] = vec0 + j * NT;
+                        sm.u.ep.v.cvec[ASX_AT(slot, SK_CAPV, 40)] = q[j];
+                        sm.u.ep.cidx[ASX_AT(slot, SK_CAPV, 41)] = vec0 + j * NT;
                     }
                 }
                 base += __popc(bal[j]);
@@ -737,7 +737,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                 const uint32_t key = P::key_of_f(xe);
                 if (key >= t0key && key > Tr::KEY_NINF) {
                     const int slot = atomicAdd(&sm.cand_count, 1);
-                    if (slot < SK_CAP) sm.u.ep.cand[slot] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)(base + e);
+                    if (slot < SK_CAP) sm.u.ep.cand[ASX_AT(slot, SK_CAP + 4, 31)] = ((unsigned long long)key << 32) | (uint32_t)~(uint32_t)(base + e);
                 }
             }
             return;
@@ -759,7 +759,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             for (int e = 0; e < E; ++e) {
                 if ((em >> e) & 1u) {
                     if (slot < SK_CAP)
-                        sm.u.ep.cand[slot] = ((unsigned long long)P::key_of_f(x[e]) << 32) | (uint32_t)~(uint32_t)(base + e);
+                        sm.u.ep.cand[ASX_AT(slot, SK_CAP + 4, 32)] = ((unsigned long long)P::key_of_f(x[e]) << 32) | (uint32_t)~(uint32_t)(base + e);
                     ++slot;
                 }
             }
@@ -841,7 +841,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                 const int v = j * NT + tid;
                 const bool ok = v < nv;
                 valid |= (ok ? 1u : 0u) << j;
-                q[j] = ok ? sv[v] : make_uint4(ninf_word, ninf_word, ninf_word, ninf_word);
+                q[j] = ok ? sv[ASX_AT(v, SK_STAGE_VEC, 51)] : make_uint4(ninf_word, ninf_word, ninf_word, ninf_word);
             }
             return valid;
         };
@@ -923,7 +923,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                         const int i = __ffs(hm) - 1;
                         hm &= hm - 1;
                         const int s = i / SK_VPT, v = (i % SK_VPT) * NT + tid;
-                        const uint4 q = ringv[(size_t)stage_of(s) * SK_STAGE_VEC + v];
+                        const uint4 q = ringv[ASX_AT((size_t)stage_of(s) * SK_STAGE_VEC + v, (size_t)S * SK_STAGE_VEC, 50)];
                         float unused = 0.f;
                         push_vec(q, (s * SK_STAGE_VEC + v) * E - lead, t0f, t0key, false, ref, unused);
                     }
@@ -996,7 +996,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         bool list_ok = !decided && !general_row && nvh <= SK_CAPV;
         if (list_ok) {
             for (int i = tid; i < nvh; i += NT) {
-                const uint4 q = sm.u.ep.v.cvec[i];
+                const uint4 q = sm.u.ep.v.cvec[ASX_AT(i, SK_CAPV, 42)];
                 // most listed vectors came in under an earlier, lower threshold
                 if (!want_tail && !(P::part_max(P::reduce(q)) >= t0f)) continue;
                 push_vec(q, sm.u.ep.cidx[i] * E - lead, t0f, t0key, want_tail, ref, tail);

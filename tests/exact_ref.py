@@ -24,7 +24,7 @@ def D(x) -> Decimal:
 
 
 def conditional(logits: Sequence[float], temp: float = 1.0, top_k: int = 0,
-                top_p: float = 1.0) -> List[Decimal]:
+                top_p: float = 1.0, typical_p: float = 1.0) -> List[Decimal]:
     """Modified next-token distribution, membership defined by counting."""
     V = len(logits)
     neg_inf = float("-inf")
@@ -40,6 +40,21 @@ def conditional(logits: Sequence[float], temp: float = 1.0, top_k: int = 0,
     xs = [D(logits[j]) / tau if alive[j] else None for j in range(V)]
     m = max(x for x in xs if x is not None)
     w = [(x - m).exp() if x is not None else Decimal(0) for x in xs]
+    if 0.0 < typical_p < 1.0:
+        # locally typical set by counting: token j stays iff the mass of the tokens whose
+        # |-ln p - H| is smaller (or equal, with a lower index) has not reached the target
+        total = sum(w)
+        pr = [x / total for x in w]
+        H = -sum(q * q.ln() for q in pr if q > 0)
+        dist = [abs(-q.ln() - H) if q > 0 else None for q in pr]
+
+        def closer(i, j):
+            return dist[i] < dist[j] or (dist[i] == dist[j] and i < j)
+        target = D(typical_p) * total
+        alive = [alive[j] and dist[j] is not None and
+                 sum(w[i] for i in range(V) if alive[i] and dist[i] is not None and closer(i, j)) < target
+                 for j in range(V)]
+        w = [w[j] if alive[j] else Decimal(0) for j in range(V)]
     if 0.0 < top_p < 1.0:
         total = sum(w)
         target = D(top_p) * total

@@ -766,3 +766,73 @@ def test_step_without_a_cut_every_evaluation_mode(B, orc, dtype):
             r = check(B, orc, arr, dtype, codes, temp, 0, 1.0, V=V, what="no cut V=%d dt=%d temp=%g" % (V, dtype, temp))
             # (at temperature 3 a long row is nearly flat: most tokens are narrower than the boundary band)
             assert r["compared"] >= (8 if temp < 2.0 or V < 4000 else 3)
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_step_typical_cut(B, orc, dtype):
+    # the locally typical set in place of the nucleus (Sec. 2 names typical decoding among the logit
+    # modifiers): small and ragged shapes, tie-heavy rows (equal logits are equally typical: the lower
+    # indices stay), masked tokens, a preceding top-k, and a Zipf-like 32000-token row
+    from paper_2210_15458_b200 import synth
+    rng = np.random.default_rng(2024)
+    cases = []
+    for V in (2, 5, 33, 1000, 4099):
+        x = rng.normal(0, 2.5, (19, V)).astype(np.float32)
+        if V > 8:
+            x[3, rng.choice(V, V // 4, replace=False)] = -np.inf
+            x[4:8] = np.round(x[4:8])
+        cases.append(x)
+    cases.append(np.zeros((6, 3000), np.float32))                          # flat: ties everywhere
+    for x in cases:
+        arr = _store(x, dtype)
+        lanes = arr.shape[0]
+        codes = rng.random(lanes)
+        codes[0], codes[1] = 0.0, 1.0
+        for temp, k, tp in [(1.0, 0, 0.9), (0.7, 0, 0.5), (1.3, 6, 0.8), (1.0, 0, 0.2), (0.9, 40, 0.95)]:
+            ref = orc.step(arr, dtype, codes, temp, k, typical_p=tp, threads=8)
+            d = {}
+            tok, c2 = B.as_step(to_dev(arr, dtype), torch.from_numpy(codes).cuda(), temp, k, diag=d, typical_p=tp)
+            torch.cuda.synchronize()
+            compare_step(ref, tok.cpu().numpy(), c2.cpu().numpy(), d["p_tok"].cpu().numpy(), d["n_kept"].cpu().numpy(),
+                         d["lane_status"].cpu().numpy(), what="typical V=%d %s" % (arr.shape[1], (temp, k, tp)))
+    w = synth.c2()
+    arr = w.logits(48) if dtype == BF16 else synth.bf16_bits_to_f32(w.logits(48))
+    codes = orc.lattice_codes(48, 0.41)
+    for temp, k, tp in [(0.7, 0, 0.9), (1.0, 0, 0.5), (0.7, 200, 0.95)]:
+        ref = orc.step(arr, dtype, codes, temp, k, typical_p=tp, threads=8)
+        d = {}
+        tok, c2 = B.as_step(to_dev(arr, dtype), torch.from_numpy(codes).cuda(), temp, k, diag=d, typical_p=tp)
+        torch.cuda.synchronize()
+        r = compare_step(ref, tok.cpu().numpy(), c2.cpu().numpy(), d["p_tok"].cpu().numpy(), d["n_kept"].cpu().numpy(),
+                         d["lane_status"].cpu().numpy(), what="typical c2 rows %s" % ((temp, k, tp),))
+        assert r["compared"] >= 36
+    with pytest.raises(ValueError):
+        B.as_step(to_dev(arr, dtype), torch.from_numpy(codes).cuda(), 1.0, 0, 0.9, typical_p=0.5)
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_step_codes_at_the_top_end_through_the_general_routine(B, orc, dtype):
+    # a code of 1 (or the largest double below it) selects the last kept token.  With few kept tokens
+    # spread over a long row, most chunks of the row hold no mass; which chunk is the last one with
+    # mass must not be read off rounded prefix sums
+    rng = np.random.default_rng(4711)
+    for V in (9001, 40000, 200003):
+        lanes = 24
+        arr = _store(rng.normal(0, 3, (lanes, V)), dtype)
+        for c in (1.0, 1.0 - 2.0 ** -53, 0.0):
+            codes = np.full(lanes, c)
+            for temp, k, p in [(1.0, 300, 0.5), (1.0, 4, 1.0), (0.9, 0, 0.3), (1.0, 1000, 0.2)]:
+                try:
+                    B.as_tune(B.TUNE_STEP_PATH, 1)
+                    ref = orc.step(arr, dtype, codes, temp, k, p, threads=8)
+                    d = {}
+                    tok, c2 = B.as_step(to_dev(arr, dtype), torch.from_numpy(codes).cuda(), temp, k, p, diag=d)
+                    torch.cuda.synchronize()
+                finally:
+                    B.as_tune(B.TUNE_STEP_PATH, 0)
+                st = d["lane_status"].cpu().numpy()
+                assert (st == 0).all(), "V=%d code %r %s: status %s" % (V, c, (temp, k, p), st)
+                # at the very ends the token is the first / last kept one whatever the rounding
+                sure = ref.d_topp > 1e-6
+                assert np.array_equal(tok.cpu().numpy()[sure], ref.tokens[sure])
+                assert np.array_equal(d["n_kept"].cpu().numpy()[sure], ref.n_kept[sure])

@@ -691,3 +691,54 @@ def test_encode_under_cuts_matches_the_enumerated_codebook(orc, kw):
         n = max(n for n in range(len(s)) if s[:n] in pre)      # longest prefix with positive probability
         assert l == pytest.approx(float(pre[s[:n]][0]), abs=1e-14)
         assert w == pytest.approx(float(pre[s[:n]][1]), rel=1e-12)
+
+
+# --------------------------------------------------------------------------- typical decoding (named in Sec. 2)
+def test_typical_counting_definition(orc):
+    # the locally typical set against its counting definition in 60-digit decimals, with
+    # temperature, a preceding top-k, ties between equal logits (lower index first) and masked tokens
+    rng = np.random.default_rng(321)
+    rows = [rng.normal(0, 2, 12), np.round(rng.normal(0, 1.5, 14)), rng.normal(0, 3, 9)]
+    rows[2][4] = -np.inf
+    checked = 0
+    for row in rows:
+        row = _rows([row])
+        for temp, k, tp in [(1.0, 0, 0.9), (0.7, 0, 0.5), (1.3, 6, 0.8), (1.0, 0, 0.2), (0.9, 3, 0.95)]:
+            p = ex.conditional([float(v) for v in row[0]], temp, k, 1.0, tp)
+            V = len(p)
+            cdf = [Decimal(0)]
+            for x in p:
+                cdf.append(cdf[-1] + x)
+            codes = (np.arange(200) + 0.5) / 200
+            o = orc.step(np.repeat(row, len(codes), 0), F32, codes, temp=temp, top_k=k, typical_p=tp)
+            if o.d_topp[0] < 1e-9:
+                continue                                   # the cut itself hangs on rounding
+            assert o.n_kept[0] == sum(1 for x in p if x > 0)
+            for c, tok, pt, d in zip(codes, o.tokens, o.p_tok, o.d_tok):
+                cd = ex.D(c)
+                want = [j for j in range(V) if cdf[j] <= cd < cdf[j + 1]][0]
+                if min(cd - cdf[want], cdf[want + 1] - cd) < Decimal("1e-12"):
+                    continue
+                checked += 1
+                assert tok == want and pt == pytest.approx(float(p[want]), rel=1e-12)
+    assert checked > 2000
+
+
+def test_typical_special_cases(orc):
+    # a uniform row: every token is equally typical, the lowest indices fill the mass;
+    # typical_p >= 1 keeps everything; a two-point row keeps the token nearer the entropy
+    flat = _rows([[0.0] * 10])
+    o = orc.step(np.repeat(flat, 50, 0), F32, (np.arange(50) + 0.5) / 50, typical_p=0.35)
+    assert (o.n_kept == 4).all() and (o.tokens <= 3).all()
+    o = orc.step(np.repeat(flat, 50, 0), F32, (np.arange(50) + 0.5) / 50, typical_p=1.0)
+    assert (o.n_kept == 10).all()
+    # p = (0.9, 0.1): H = 0.325; -ln p = (0.105, 2.303): token 0 is the typical one
+    two = _rows([np.log([0.9, 0.1])])
+    o = orc.step(np.repeat(two, 20, 0), F32, (np.arange(20) + 0.5) / 20, typical_p=0.5)
+    assert (o.n_kept == 1).all() and (o.tokens == 0).all()
+    # p = (0.6, 0.2, 0.2): H = 0.950; -ln p = (0.511, 1.609, 1.609): distances 0.439, 0.659, 0.659 -> 0, then 1
+    three = _rows([np.log([0.6, 0.2, 0.2])])
+    o = orc.step(np.repeat(three, 20, 0), F32, (np.arange(20) + 0.5) / 20, typical_p=0.7)
+    assert (o.n_kept == 2).all() and set(o.tokens.tolist()) == {0, 1}
+    with pytest.raises(ValueError):
+        orc.step(flat, F32, np.array([0.5]), top_p=0.5, typical_p=0.5)
