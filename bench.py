@@ -487,6 +487,26 @@ def bench_bigram(reps: int, warmup: int, S: int = 64, T: int = 128, eos_variant:
     stats["ms_ngram_diversity"] = timed(lambda: B.as_ngram_diversity(seq, ln, w.N))[0] if fits else None
     stats["ms_reward_mean"] = timed(lambda: B.as_reward_mean(seq, ln, w.N, r))[0]
     out["groups"] = stats
+    # the same decode with extended-precision codes (the lattice steers every token, not only the
+    # first ~50 bits' worth): time, whole-sequence duplicate rates, and the estimator's spread again
+    st0 = B.as_xp_lattice_state(w.N, w.shift(), 0, w.N, w.S)
+    state = st0.clone()
+
+    def run_xp():
+        state.copy_(st0)
+        B.as_decode_bigram_xp(table, prev, state, w.N, w.T, w.eos, w.temp, w.top_k, w.top_p, seq=seq, length=ln)
+    out["lattice_extended_precision"] = decode_entry(run_xp)
+    means, divs = [], []
+    for k in range(K):
+        stk = B.as_xp_lattice_state(w.N, float(shifts[k]), 0, w.N, w.S)
+        B.as_decode_bigram_xp(table, prev, stk, w.N, w.T, w.eos, w.temp, w.top_k, w.top_p, seq=seq, length=ln)
+        means.append(B.as_reward_mean(seq, ln, w.N, r)[1])
+        if fits:
+            divs.append(B.as_ngram_diversity(seq, ln, w.N)[2])
+    means = torch.stack(means)
+    stats["lattice_extended_precision"] = {
+        "estimator_sd_over_%d_runs_mean_over_groups" % K: float(means.std(dim=0).mean().item()),
+        "ngram_diversity_mean": float(torch.stack(divs).mean().item()) if fits else None}
     if eos_variant:
         # SUPPLEMENTARY variant, not the configuration as specified: with a random permutation the
         # EOS column's bias makes P(EOS) ~ 1e-10 and no lane ever stops early; here that column's
@@ -528,6 +548,12 @@ def side_measurements(B, peak, skip_key):
             tmed, tmn, _ = sb.per_launch_us(sb.step_two_calls)
             blocks[key]["fused_first_step_us_median"] = fmed          # as_step_lattice
             blocks[key]["two_calls_us_median"] = tmed                 # as_lattice_codes + as_step
+        if key == "c2":
+            # the typical cut in place of top-k (general routine: no fast path)
+            def step_typical():
+                B.as_step(sb._next(), sb.codes, w.temp, 0, 1.0, tokens=sb.tokens, codes_out=sb.codes_out, typical_p=0.9)
+            ymed, ymn, _ = sb.per_launch_us(step_typical, replays=5)
+            blocks[key]["typical_p_0.9_us_median"] = ymed
         if key == "c5_1024":
             # the row split over a thread-block cluster (4 and 8 CTAs per lane) beside the default
             for cs in (4, 8):

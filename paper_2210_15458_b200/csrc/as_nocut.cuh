@@ -15,8 +15,8 @@
 //              holds c Z, re-evaluates that chunk element by element, picks the token and
 //              rescales the code (Algorithm 1: (m, M), c <- (c - m)/(M - m)).
 // Masses.  bf16 logits take only 65536 values, and e_j = exp(l_j / temp) depends on nothing
-// else: a shared-memory table over the magnitudes [2^-8, 2^6) of both signs (3584 doubles,
-// filled once per CTA with the fp64 exponential) turns every mass into one 8-byte load and
+// else: a shared-memory table over the magnitudes [2^-8, 2^6) of both signs (4096 slots,
+// 3584 in use, filled once per CTA with the fp64 exponential) turns every mass into one 8-byte load and
 // one fp64 add instead of a 13-operation fp64 exponential.  The masses are not divided by
 // exp(max / temp): token choice and rescaled code do not depend on a common factor, and with
 // temp >= 0.1 the table's range stays far inside fp64.  Elements outside the table: tiny
@@ -35,13 +35,13 @@ constexpr int NC_MAXG = 3;                        // groups per CTA
 constexpr int NC_PIECE_BYTES = 16384;
 constexpr int NC_MAXPIECE = 6;
 constexpr int NC_MAXROW = NC_MAXPIECE * NC_PIECE_BYTES;        // rows up to 96 KB
-constexpr int NC_R = 4;                           // sub-rows of 32 vectors per chunk
-constexpr int NC_MAXCH = NC_MAXROW / 16 / 32 / NC_R;           // 48 chunks
+constexpr int NC_R = 4;                           // chunks a warp takes together in the sum pass
+constexpr int NC_MAXCH = NC_MAXROW / 16 / 32;                  // 192 chunks of 32 vectors
 constexpr int NC_EXP_LO = 119;                    // biased exponent of 2^-8
 constexpr int NC_BINADES = 14;                    // [2^-8, 2^6)
 constexpr int NC_ENT = NC_BINADES * 128;          // table entries per sign
 constexpr uint32_t NC_MAG_LO = (uint32_t)NC_EXP_LO << 7;
-constexpr int NC_TBL_DOUBLES = 2 * NC_ENT + 2;    // + one entry that holds 0.0 (+ padding)
+constexpr int NC_TBL_DOUBLES = 4096;              // sign (1) | low four exponent bits | mantissa (7)
 constexpr double NC_MIN_TEMP = 0.1;               // below: exp(64 / temp) leaves fp64's comfortable range
 
 constexpr int NC_STEP = 0, NC_DECODE = 1, NC_ENCODE = 2, NC_DECODE_XP = 3;
@@ -90,7 +90,7 @@ struct NcGroupSmem {
     int flags;
     int masked;          // table mode: -inf elements (padding included); robust mode: finite elements
     int poisoned;
-    unsigned long long has;      // bit c: chunk c holds mass (not to be read off the scanned sums, whose
+    unsigned has[6];             // bit c: chunk c holds mass (not to be read off the scanned sums, whose
                                  // lane totals are added in another order than the sums inside a lane)
     LaneResult res;
     unsigned long long xp_lo, xp_hi;     // extended-precision steps: the chosen token's cells [xp_lo, xp_hi)
@@ -135,6 +135,10 @@ struct NcRow {
         const uint32_t w = DT == DT_BF16 ? 0xFF80FF80u : 0xFF800000u;
         return make_uint4(w, w, w, w);
     }
+    __device__ __forceinline__ static uint4 ones_vec() {           // the value 1.0 in every element
+        const uint32_t w = DT == DT_BF16 ? 0x3F803F80u : 0x3F800000u;
+        return make_uint4(w, w, w, w);
+    }
     // vector v of the row; elements at or past V read as -inf
     __device__ __forceinline__ uint4 load_vec(int v) const {
         if (v < bulk_vec) return rowv[ASX_AT(v, NC_MAXROW / 16, 70)];
@@ -156,37 +160,52 @@ struct NcRow {
         return make_uint4(w[0], w[1], w[2], w[3]);
     }
 
-    // ---- masses of one vector, table mode (bf16).  An element outside the table goes through
-    //      `slow`: rare, kept out of line.
-    __device__ __noinline__ double slow(uint32_t b, int& flags, int& masked) const {
+    // ---- masses of one vector, table mode (bf16).  Table entry of a bf16 pattern h = s|eeeeeeee|mmmmmmm
+    //      with exponent field in [119, 133): index s<<11 | (e & 15)<<7 | m -- the low four exponent
+    //      bits are distinct over those 14 binades, so the byte offset is two shifts and two masks
+    //      of the pattern itself.  A vector with any element outside the table goes, element by
+    //      element, through `slow1` (rare on real rows; kept out of line).
+    __device__ __forceinline__ static uint32_t tbl_off(uint32_t w, bool high) {
+        return high ? (((w >> 13) & 0x3FF8u) | ((w >> 17) & 0x4000u)) : (((w << 3) & 0x3FF8u) | ((w >> 1) & 0x4000u));
+    }
+    // one element outside the fast path (free of `this`, so that the row's state stays in registers):
+    // its mass, or -1 for -inf (a masked token), -2 for NaN / +inf, -3 for a finite magnitude >= 64
+    __device__ __noinline__ static double slow1(uint32_t b, const double* tbl_, const double* exp_tbl_, double inv_tau_) {
         const uint32_t mag = b & 0x7FFFu;
-        if (mag >= 0x7F80u) {
-            if (b == 0xFF80u) { ++masked; return 0.0; }         // -inf: a masked token
-            flags |= NCF_BAD;                                  // NaN or +inf
-            return 0.0;
-        }
-        if (mag >= NC_MAG_LO) { flags |= NCF_BIG; return 0.0; } // >= 64: the row is redone relative to its maximum
-        return exp_core((double)__uint_as_float(b << 16) * inv_tau, exp_tbl);   // |x| < 2^-8 (zeros, subnormals)
+        if (mag >= 0x7F80u) return b == 0xFF80u ? -1.0 : -2.0;
+        if (mag >= NC_MAG_LO + NC_ENT) return -3.0;
+        if (mag >= NC_MAG_LO) return *reinterpret_cast<const double*>(reinterpret_cast<const char*>(tbl_) + tbl_off(b, false));
+        return exp_core((double)__uint_as_float(b << 16) * inv_tau_, exp_tbl_);   // |x| < 2^-8 (zeros, subnormals)
     }
     __device__ __forceinline__ void masses_tbl(const uint4& q, double (&e)[8], int& flags, int& masked) const {
         const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-        uint32_t idx[8];
-        unsigned bad = 0;
+        // every magnitude in [NC_MAG_LO, NC_MAG_LO + NC_ENT)?  Packed per 16-bit half: t = |h| - NC_MAG_LO
+        // must stay below NC_ENT = 0x700, i.e. neither t nor t + 0x100 may reach bit 11.  (A borrow out
+        // of the low half only occurs when that half is already out of range.)
+        uint32_t bad = 0;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const uint32_t u0 = w[i] - NC_MAG_LO, u1 = (w[i] >> 16) - NC_MAG_LO;
-            const uint32_t m0 = u0 & 0x7FFFu, m1 = u1 & 0x7FFFu;
-            const bool ok0 = m0 < (uint32_t)NC_ENT, ok1 = m1 < (uint32_t)NC_ENT;
-            idx[2 * i] = ok0 ? m0 + ((u0 >> 15) & 1u) * NC_ENT : 2u * NC_ENT;
-            idx[2 * i + 1] = ok1 ? m1 + ((u1 >> 15) & 1u) * NC_ENT : 2u * NC_ENT;
-            bad |= (ok0 ? 0u : 1u) << (2 * i) | (ok1 ? 0u : 1u) << (2 * i + 1);
+            const uint32_t t = (w[i] & 0x7FFF7FFFu) - (NC_MAG_LO | (NC_MAG_LO << 16));
+            bad |= t | (t + 0x01000100u);
         }
+        if (bad & 0xF800F800u) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) e[k] = tbl[ASX_AT(idx[k], NC_TBL_DOUBLES, 71)];
-        if (bad) {
+            for (int k = 0; k < 8; ++k) {
+                double v = slow1((k & 1) ? (w[k >> 1] >> 16) : (w[k >> 1] & 0xFFFFu), tbl, exp_tbl, inv_tau);
+                if (v < 0.0) {
+                    masked += (v == -1.0);
+                    flags |= v == -2.0 ? NCF_BAD : v == -3.0 ? NCF_BIG : 0;
+                    v = 0.0;
+                }
+                e[k] = v;
+            }
+            return;
+        }
+        const char* tb = reinterpret_cast<const char*>(tbl);
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
-                if ((bad >> k) & 1u) e[k] = slow((k & 1) ? (w[k >> 1] >> 16) : (w[k >> 1] & 0xFFFFu), flags, masked);
+        for (int i = 0; i < 4; ++i) {
+            e[2 * i] = *reinterpret_cast<const double*>(tb + ASX_AT(tbl_off(w[i], false), NC_TBL_DOUBLES * 8, 71));
+            e[2 * i + 1] = *reinterpret_cast<const double*>(tb + ASX_AT(tbl_off(w[i], true), NC_TBL_DOUBLES * 8, 71));
         }
     }
     // ---- robust mode: fp64 exponential relative to the row maximum; counts the finite elements
@@ -205,33 +224,55 @@ struct NcRow {
         else masses_dir(q, e, count);
     }
 
-    // ---- per-chunk sums in index order.  g.flags / g.masked must be zero on entry (group-wide).
-    //      A chunk is NC_R sub-rows of 32 vectors; a warp takes the NC_R vectors of a lane at once,
-    //      so that their table loads are in flight together and one reduction serves them all.
+    __device__ __forceinline__ bool chunk_has(int c) const { return (g.has[c >> 5] >> (c & 31)) & 1u; }
+
+    // ---- per-chunk sums in index order (a chunk = 32 consecutive vectors, one per lane).
+    //      g.flags / g.masked / g.has must be zero on entry (group-wide).  A warp takes NC_R
+    //      consecutive chunks at once: their table loads are in flight together and their
+    //      reductions interleave (a lone reduction is a chain of five dependent shuffle-add rounds).
     template <bool TBL>
     __device__ void sum_pass() {
         int flags = 0, count = 0, cur = -1;
-        for (int c = warp; c < nch; c += NC_GW) {
-            const int piece = (c * NC_R * 512) / NC_PIECE_BYTES;
+        const int nsuper = (nch + NC_R - 1) / NC_R;
+        for (int sc = warp; sc < nsuper; sc += NC_GW) {
+            const int piece = (sc * NC_R * 512) / NC_PIECE_BYTES;
             if (piece != cur && piece < npiece) { wait_piece(piece); cur = piece; }
+            // (no branches in here: the four vectors' index arithmetic and table loads interleave.  A
+            //  vector past the row is replaced by a harmless in-table pattern and its sum dropped;
+            //  inside the row's last chunk it counts as masked padding)
             uint4 q[NC_R];
+            bool valid[NC_R];
 #pragma unroll
             for (int r = 0; r < NC_R; ++r) {
-                const int v = (c * NC_R + r) * 32 + lane;
-                q[r] = v < nvec ? load_vec(v) : ninf_vec();
+                const int v = (sc * NC_R + r) * 32 + lane;
+                valid[r] = v < nvec;
+                q[r] = valid[r] ? load_vec(v) : ((TBL && DT == DT_BF16) ? ones_vec() : ninf_vec());
+                count += (!valid[r] && sc * NC_R + r < nch) ? (TBL && DT == DT_BF16 ? E : 0) : 0;
             }
-            double s = 0.0;
+            double s[NC_R];
 #pragma unroll
             for (int r = 0; r < NC_R; ++r) {
                 double e[E];
                 masses<TBL>(q[r], e, flags, count);
-                if constexpr (E == 8) s += ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
-                else s += (e[0] + e[1]) + (e[2] + e[3]);
+                double t;
+                if constexpr (E == 8) t = ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+                else t = (e[0] + e[1]) + (e[2] + e[3]);
+                s[r] = valid[r] ? t : 0.0;
             }
-            s = warp_sum_d(s);
-            if (lane == 0) {
-                g.chunk_sum[ASX_AT(c, NC_MAXCH + 1, 72)] = s;
-                if (s > 0.0) atomicOr(&g.has, 1ull << c);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                for (int r = 0; r < NC_R; ++r) s[r] += __shfl_xor_sync(FULL, s[r], o);
+            }
+            if (lane < NC_R) {
+                double mine = s[0];
+#pragma unroll
+                for (int r = 1; r < NC_R; ++r) mine = lane == r ? s[r] : mine;
+                const int c = sc * NC_R + lane;
+                if (c < nch) {
+                    g.chunk_sum[ASX_AT(c, NC_MAXCH + 1, 72)] = mine;
+                    if (mine > 0.0) atomicOr(&g.has[c >> 5], 1u << (c & 31));
+                }
             }
         }
         flags = __reduce_or_sync(FULL, flags);
@@ -278,13 +319,23 @@ struct NcRow {
         __syncwarp();
     }
 
-    // masses of sub-row r of chunk c for this lane (zeros past the row)
+    // masses of this lane's vector of chunk c (zeros past the row); returns its first token index
     template <bool TBL>
-    __device__ __forceinline__ int sub_masses(int c, int r, double (&ev)[E]) const {
-        const int v = (c * NC_R + r) * 32 + lane;
+    __device__ __forceinline__ int chunk_masses(int c, double (&ev)[E]) const {
+        const int v = c * 32 + lane;
         int f = 0, cnt = 0;
         masses<TBL>(v < nvec ? load_vec(v) : ninf_vec(), ev, f, cnt);
         return v * E;
+    }
+    // three quotients on three lanes (an fp64 division is a long dependent chain): lane 0 returns
+    // n0 / d0, and q1 = n1 / d1, q2 = n2 / d1 come back to it through shuffles
+    __device__ __forceinline__ double div3(double n0, double d0, double n1, double n2, double d1, double& q1, double& q2) const {
+        const double num = lane == 0 ? n0 : lane == 1 ? n1 : n2;
+        const double den = lane == 0 ? d0 : d1;
+        const double quo = num / den;
+        q1 = __shfl_sync(FULL, quo, 1);
+        q2 = __shfl_sync(FULL, quo, 2);
+        return quo;
     }
 
     // ---- warp 0: the token whose interval holds c * Z, and the rescaled code
@@ -295,7 +346,7 @@ struct NcRow {
         const double t = c * Z;
         int first = INT_MAX, last_c = -1;
         for (int ci = lane; ci < nch; ci += 32) {
-            if ((g.has >> ci) & 1ull) {
+            if (chunk_has(ci)) {
                 last_c = ci;
                 if (t < g.chunk_sum[ci + 1]) first = min(first, ci);
             }
@@ -307,41 +358,35 @@ struct NcRow {
         int tok = -1;
         double tok_S = 0.0, tok_e = 1.0;
         if (cstar >= 0) {
-            double run = g.chunk_sum[ASX_AT(cstar, NC_MAXCH + 1, 73)];
-            int last_idx = -1;
-            double last_S = 0.0, last_e = 1.0;
-            for (int r = 0; r < NC_R && tok < 0; ++r) {
-                double ev[E];
-                const int base = sub_masses<TBL>(cstar, r, ev);
-                double local = 0.0;
+            const double run = g.chunk_sum[ASX_AT(cstar, NC_MAXCH + 1, 73)];
+            double ev[E];
+            const int base = chunk_masses<TBL>(cstar, ev);
+            double local = 0.0;
 #pragma unroll
-                for (int k = 0; k < E; ++k) local += ev[k];
-                const double incl = warp_incl_scan_d(local, lane);
-                double excl = __shfl_up_sync(FULL, incl, 1);
-                if (lane == 0) excl = 0.0;
-                int pick = -1;
-                double pick_S = 0.0, pick_e = 1.0;
-                double S = run + excl;
+            for (int k = 0; k < E; ++k) local += ev[k];
+            const double incl = warp_incl_scan_d(local, lane);
+            double excl = __shfl_up_sync(FULL, incl, 1);
+            if (lane == 0) excl = 0.0;
+            int pick = -1, last_idx = -1;
+            double pick_S = 0.0, pick_e = 1.0, last_S = 0.0, last_e = 1.0;
+            double S = run + excl;
 #pragma unroll
-                for (int k = 0; k < E; ++k) {
-                    if (ev[k] > 0.0) {
-                        if (pick < 0 && t < S + ev[k]) { pick = base + k; pick_S = S; pick_e = ev[k]; }
-                        last_idx = base + k; last_S = S; last_e = ev[k];
-                        S += ev[k];
-                    }
+            for (int k = 0; k < E; ++k) {
+                if (ev[k] > 0.0) {
+                    if (pick < 0 && t < S + ev[k]) { pick = base + k; pick_S = S; pick_e = ev[k]; }
+                    last_idx = base + k; last_S = S; last_e = ev[k];
+                    S += ev[k];
                 }
-                const bool cross = !force_last && local > 0.0 && (t < run + incl);
-                const unsigned bal = __ballot_sync(FULL, cross);
-                if (bal) {
-                    const int L = __ffs(bal) - 1;
-                    if (pick < 0) { pick = last_idx; pick_S = last_S; pick_e = last_e; }
-                    tok = __shfl_sync(FULL, pick, L);
-                    tok_S = __shfl_sync(FULL, pick_S, L);
-                    tok_e = __shfl_sync(FULL, pick_e, L);
-                }
-                run += __shfl_sync(FULL, incl, 31);
             }
-            if (tok < 0) {   // rounding at the top end: the last token with mass in the chunk
+            const bool cross = !force_last && local > 0.0 && (t < run + incl);
+            const unsigned bal = __ballot_sync(FULL, cross);
+            if (bal) {
+                const int L = __ffs(bal) - 1;
+                if (pick < 0) { pick = last_idx; pick_S = last_S; pick_e = last_e; }
+                tok = __shfl_sync(FULL, pick, L);
+                tok_S = __shfl_sync(FULL, pick_S, L);
+                tok_e = __shfl_sync(FULL, pick_e, L);
+            } else {   // rounding at the top end: the last token with mass in the chunk
                 const unsigned best = warp_max_u((unsigned)(last_idx + 1));
                 const unsigned bal2 = __ballot_sync(FULL, (unsigned)(last_idx + 1) == best);
                 const int L = __ffs(bal2) - 1;
@@ -350,15 +395,16 @@ struct NcRow {
                 tok_e = __shfl_sync(FULL, last_e, L);
             }
         }
+        double p_tok, cdf_lo;
+        double cn = div3(t - tok_S, tok_e, tok_e, tok_S, Z, p_tok, cdf_lo);
         if (lane == 0) {
-            double cn = (t - tok_S) / tok_e;
             if (!(cn >= 0.0)) cn = 0.0;
             if (cn > ASX_ONE_BELOW) cn = ASX_ONE_BELOW;
             LaneResult r;
             r.token = tok; r.status = tok < 0 ? ST_NUMERIC : ST_OK; r.n_kept = n_kept;
             r.code_out = tok < 0 ? c_in : cn;
-            r.p_tok = tok_e / Z;
-            r.cdf_lo = tok_S / Z;
+            r.p_tok = p_tok;
+            r.cdf_lo = cdf_lo;
             g.res = r;
         }
     }
@@ -372,42 +418,32 @@ struct NcRow {
         const double K = 4294967296.0 / Z;
         int last_c = -1;
         for (int ci = lane; ci < nch; ci += 32)
-            if ((g.has >> ci) & 1ull) last_c = ci;
+            if (chunk_has(ci)) last_c = ci;
         last_c = (int)warp_max_u((unsigned)(last_c + 1)) - 1;
         int tok = -1;
         unsigned long long plo = 0, phi = 0;
         double pe = 1.0;
         if (last_c >= 0) {
-            // the first chunk with mass whose end cell lies beyond the code's cell
+            // the first chunk with mass whose end cell lies beyond the code's cell, and the chunk
+            // with mass before it: a chunk starts in the cell where that one ended
             int first = INT_MAX;
             for (int ci = lane; ci <= last_c; ci += 32) {
                 const unsigned long long fe = ci == last_c ? XP_TOP : xp_cell(g.chunk_sum[ci + 1], K);
-                if (fe > tcell && ((g.has >> ci) & 1ull)) first = min(first, ci);
+                if (fe > tcell && chunk_has(ci)) first = min(first, ci);
             }
             const int cstar = (int)warp_min_u((unsigned)first);
+            int prev_c = -1;
+            for (int ci = lane; ci < cstar; ci += 32)
+                if (chunk_has(ci)) prev_c = ci;
+            prev_c = (int)warp_max_u((unsigned)(prev_c + 1)) - 1;
             const unsigned long long Fend = cstar == last_c ? XP_TOP : xp_cell(g.chunk_sum[cstar + 1], K);
-            // the last sub-row of the chunk that holds mass
-            int r_last = 0;
-            for (int r = 0; r < NC_R; ++r) {
-                double ev[E];
-                sub_masses<TBL>(cstar, r, ev);
-                double local = 0.0;
-#pragma unroll
-                for (int k = 0; k < E; ++k) local += ev[k];
-                if (__ballot_sync(FULL, local > 0.0)) r_last = r;
-            }
             double run = g.chunk_sum[cstar];
-            // the chunk starts in the cell where the chunk with mass before it ended
-            const unsigned long long before = g.has & ((1ull << cstar) - 1ull);
-            const unsigned long long carry0 = before ? xp_cell(g.chunk_sum[64 - __clzll((long long)before)], K) : 0ull;
-            unsigned long long carry = carry0;
-            for (int r = 0; r <= r_last && tok < 0; ++r) {
-                double ev[E];
-                const int base = sub_masses<TBL>(cstar, r, ev);
-                int pk = 0;
-                const int L = xp_subrow<E>(ev, lane, K, tcell, r == r_last, Fend, run, carry, pk, plo, phi, pe);
-                if (L >= 0) tok = __shfl_sync(FULL, base, L) + pk;
-            }
+            unsigned long long carry = prev_c < 0 ? 0ull : xp_cell(g.chunk_sum[prev_c + 1], K);
+            double ev[E];
+            const int base = chunk_masses<TBL>(cstar, ev);
+            int pk = 0;
+            const int L = xp_subrow<E>(ev, lane, K, tcell, true, Fend, run, carry, pk, plo, phi, pe);
+            if (L >= 0) tok = __shfl_sync(FULL, base, L) + pk;
         }
         if (lane == 0) {
             LaneResult r;
@@ -425,20 +461,19 @@ struct NcRow {
     __device__ void interval(int tok, int n_kept) {
         scan_chunks();
         const double Z = g.chunk_sum[nch];
-        const int cstar = (tok / E) / (32 * NC_R);
+        const int cstar = (tok / E) >> 5;
+        double ev[E];
+        const int base = chunk_masses<TBL>(cstar, ev);
         double below = 0.0, e_tok = 0.0;
-        for (int r = 0; r < NC_R; ++r) {
-            if ((cstar * NC_R + r) * 32 * E > tok) break;      // warp-uniform: sub-rows past the token
-            double ev[E];
-            const int base = sub_masses<TBL>(cstar, r, ev);
 #pragma unroll
-            for (int k = 0; k < E; ++k) {
-                if (base + k < tok) below += ev[k];
-                if (base + k == tok) e_tok = ev[k];
-            }
+        for (int k = 0; k < E; ++k) {
+            if (base + k < tok) below += ev[k];
+            if (base + k == tok) e_tok = ev[k];
         }
         below = warp_sum_d(below);
         e_tok = warp_sum_d(e_tok);                 // one lane holds it, the others add zero
+        double p_tok, unused;
+        const double cdf_lo = div3(g.chunk_sum[ASX_AT(cstar, NC_MAXCH + 1, 74)] + below, Z, e_tok, 0.0, Z, p_tok, unused);
         if (lane == 0) {
             // kept = not masked (a finite logit whose mass underflows still has its empty interval)
             bool kept;
@@ -447,8 +482,8 @@ struct NcRow {
             LaneResult r;
             r.token = kept ? tok : -1; r.status = kept ? ST_OK : ST_NUMERIC; r.n_kept = n_kept;
             r.code_out = 0.0;
-            r.p_tok = e_tok / Z;
-            r.cdf_lo = (g.chunk_sum[ASX_AT(cstar, NC_MAXCH + 1, 74)] + below) / Z;
+            r.p_tok = p_tok;
+            r.cdf_lo = cdf_lo;
             g.res = r;
         }
     }
@@ -468,7 +503,7 @@ struct NcRow {
             if (flags & NCF_BAD) failed = true;
             else if (flags & NCF_BIG) robust = true;
             if (!failed && !robust && warp == 0 && !g.poisoned) {
-                const int n_kept = nch * NC_R * 32 * E - g.masked;       // (padding counts as masked)
+                const int n_kept = nch * 32 * E - g.masked;       // (padding counts as masked)
                 if (n_kept <= 0) { if (lane == 0) g.res = failed_lane(c_in, ST_NUMERIC); }
                 else if (xp) locate_xp<true>(tcell, n_kept);
                 else if (tok_given < 0) locate<true>(c, c_in, n_kept);
@@ -476,7 +511,7 @@ struct NcRow {
             }
             if (robust) {                                        // (the counters start again)
                 nc_bar<NC_GT>(gi);
-                if (gtid == 0) { g.flags = 0; g.masked = 0; g.has = 0ull; }
+                if (gtid == 0) { g.flags = 0; g.masked = 0; g.has[0] = g.has[1] = g.has[2] = g.has[3] = g.has[4] = g.has[5] = 0u; }
                 nc_bar<NC_GT>(gi);
             }
         }
@@ -502,7 +537,7 @@ struct NcRow {
         }
         nc_bar<NC_GT>(gi);
         const LaneResult out = g.res;
-        if (gtid == 0) { g.flags = 0; g.masked = 0; g.has = 0ull; }
+        if (gtid == 0) { g.flags = 0; g.masked = 0; g.has[0] = g.has[1] = g.has[2] = g.has[3] = g.has[4] = g.has[5] = 0u; }
         nc_bar<NC_GT>(gi);          // the buffer and the result slot are free again
         return out;
     }
@@ -523,16 +558,18 @@ __global__ void __launch_bounds__(NC_MAXG * NC_GT, 1) nocut_kernel(const NocutAr
     fill_exp_table(exp_tbl, tid);
     if (gtid == 0) {
         for (int p = 0; p < NC_MAXPIECE; ++p) mbar_init(smem_u32(&g.full[p]), 1);
-        g.flags = 0; g.masked = 0; g.poisoned = 0; g.has = 0ull;
+        g.flags = 0; g.masked = 0; g.poisoned = 0; g.has[0] = g.has[1] = g.has[2] = g.has[3] = g.has[4] = g.has[5] = 0u;
     }
     if (tid == 0) fence_mbar_init();
     __syncthreads();
     if (a.use_table && DT == DT_BF16) {
-        for (int i = tid; i < 2 * NC_ENT; i += blockDim.x) {
-            const uint32_t bits = ((uint32_t)(i % NC_ENT) + NC_MAG_LO) | (i >= NC_ENT ? 0x8000u : 0u);
-            tbl[i] = exp_core((double)__uint_as_float(bits << 16) * a.inv_tau, exp_tbl);
+        for (int i = tid; i < NC_TBL_DOUBLES; i += blockDim.x) {
+            const uint32_t e4 = (i >> 7) & 15u;
+            const uint32_t ex = e4 >= (NC_EXP_LO & 15u) ? (NC_EXP_LO & ~15u) + e4 : (NC_EXP_LO & ~15u) + 16u + e4;
+            const uint32_t bits = ((uint32_t)(i >> 11) << 15) | (ex << 7) | (uint32_t)(i & 127);
+            const bool used = ex >= (uint32_t)NC_EXP_LO && ex < (uint32_t)(NC_EXP_LO + NC_BINADES);
+            tbl[i] = used ? exp_core((double)__uint_as_float(bits << 16) * a.inv_tau, exp_tbl) : 0.0;
         }
-        if (tid < 2) tbl[2 * NC_ENT + tid] = 0.0;
     }
     __syncthreads();
 
@@ -544,26 +581,26 @@ __global__ void __launch_bounds__(NC_MAXG * NC_GT, 1) nocut_kernel(const NocutAr
     R.nvec = (V + Tr::E - 1) / Tr::E;
     const int bulk_bytes = (V * Tr::BYTES) & ~15;
     R.bulk_vec = bulk_bytes >> 4;
-    R.nch = (R.nvec + 32 * NC_R - 1) / (32 * NC_R);
+    R.nch = (R.nvec + 31) / 32;
     R.npiece = (bulk_bytes + NC_PIECE_BYTES - 1) / NC_PIECE_BYTES;
     R.gi = gi; R.gtid = gtid; R.lane = gtid & 31; R.warp = gtid >> 5;
     R.inv_tau = a.inv_tau; R.s64 = 0.0; R.c64 = 0.0;
     R.parity = 0;
     R.wait_cycles = a.wait_cycles;
-    bool armed = false;              // thread 0 of the group: copies issued under the current parity
+    bool armed = false;              // copies issued under the current parity (uniform in the group)
 
-    // thread 0 of the group: bring a row into the group's buffer (every reader of the previous
-    // row has passed the group barrier that precedes this call)
+    // bring a row into the group's buffer (every reader of the previous row has passed the group
+    // barrier that precedes this call)
     auto fetch = [&](const char* src) {
         R.grow = src;
-        if (gtid == 0 && !a.debug_no_copy && !*(volatile int*)&g.poisoned) {
-            fence_proxy_async();
-            const uint32_t dst = smem_u32(R.rowv);
-            for (int p = 0; p < R.npiece; ++p) {
+        if (!a.debug_no_copy && !*(volatile int*)&g.poisoned) {
+            if (gtid < R.npiece) {                 // one piece per thread: the issues do not queue behind one another
+                fence_proxy_async();
+                const int p = gtid;
                 const uint32_t bytes = (uint32_t)min(NC_PIECE_BYTES, bulk_bytes - p * NC_PIECE_BYTES);
                 const uint32_t bar = smem_u32(&g.full[p]);
                 mbar_expect_tx(bar, bytes);
-                bulk_g2s(dst + p * NC_PIECE_BYTES, src + (size_t)p * NC_PIECE_BYTES, bytes, bar);
+                bulk_g2s(smem_u32(R.rowv) + p * NC_PIECE_BYTES, src + (size_t)p * NC_PIECE_BYTES, bytes, bar);
             }
             armed = true;
         }
