@@ -496,6 +496,15 @@ def bench_bigram(reps: int, warmup: int, S: int = 64, T: int = 128, eos_variant:
         state.copy_(st0)
         B.as_decode_bigram_xp(table, prev, state, w.N, w.T, w.eos, w.temp, w.top_k, w.top_p, seq=seq, length=ln)
     out["lattice_extended_precision"] = decode_entry(run_xp)
+
+    def run_xp_topk():
+        state.copy_(st0)
+        B.as_decode_bigram_xp(table, prev, state, w.N, w.T, w.eos, w.temp, 10, 1.0, seq=seq, length=ln)
+    med, mn = timed(run_xp_topk)
+    tokens = int(ln.sum().item())
+    out["lattice_extended_precision_top_k_10"] = {"ms_per_decode_median": med, "ms_per_decode_min": mn, "tokens": tokens,
+                                                  "tokens_per_s": tokens / med * 1e3, "launches_per_decode": w.T + 2,
+                                                  "duplicate_prefix_rate": dup_rates(seq)}
     means, divs = [], []
     for k in range(K):
         stk = B.as_xp_lattice_state(w.N, float(shifts[k]), 0, w.N, w.S)

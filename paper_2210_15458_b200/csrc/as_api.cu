@@ -120,13 +120,13 @@ static int launch_staged(const StepArgs& a, size_t smem, int sms, int want_per_s
     return AS_OK;
 }
 
-template <int DT, int CAPV, int MINB, bool UA, bool GATHER = false>
+template <int DT, int CAPV, int MINB, bool UA, bool GATHER = false, bool XP = false>
 static int launch_stream_ua(const StepArgs& a, int stages, int sms, int want_per_sm, cudaStream_t st) {
     static bool attr_set[64] = {false};
     static int per_sm_cache[64][SK_MAXSTAGES + 1] = {{0}};
     int dev = 0;
     cudaGetDevice(&dev);
-    auto kern = step_stream_kernel<DT, CAPV, MINB, UA, GATHER>;
+    auto kern = step_stream_kernel<DT, CAPV, MINB, UA, GATHER, XP>;
     cudaError_t e;
     if (!attr_set[dev]) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(SMEM_OPTIN_MAX - 1024));
@@ -173,6 +173,7 @@ static int launch_stream_ua(const StepArgs& a, int stages, int sms, int want_per
 // copies each row from the boundary below its start
 template <int DT, int CAPV, int MINB>
 static int launch_stream(const StepArgs& a, bool unaligned, int stages, int sms, int want_per_sm, cudaStream_t st) {
+    if (a.row_idx && a.xp_state) return launch_stream_ua<DT, CAPV, MINB, true, true, true>(a, stages, sms, want_per_sm, st);
     if (a.row_idx) return launch_stream_ua<DT, CAPV, MINB, true, true>(a, stages, sms, want_per_sm, st);   // table rows: any alignment
     return unaligned ? launch_stream_ua<DT, CAPV, MINB, true>(a, stages, sms, want_per_sm, st)
                      : launch_stream_ua<DT, CAPV, MINB, false>(a, stages, sms, want_per_sm, st);
@@ -450,7 +451,7 @@ __global__ void decode_setup_kernel(const int* __restrict__ start_or_prev, const
         }
         const bool ok = prev >= 0 && prev < V;
         idx0[ln] = ok ? prev : -1;
-        codes[ln] = c;
+        if (codes) codes[ln] = c;
         if (lane_status) lane_status[ln] = ok ? ST_OK : ST_NUMERIC;
     }
 }
@@ -656,6 +657,7 @@ static int step_common(const void* d_logits, int dtype, int lanes, int V, long l
     a.lanes = lanes; a.V = V; a.top_k = top_k;
     a.lat_N = lat_N; a.lat_j0 = lat_j0; a.lat_u = lat_u;
     a.row_idx = nullptr; a.idx_stride = 1; a.tok_stride = 1; a.eos = -1; a.rows = 0;
+    a.xp_state = nullptr; a.xp_N = 0;
     a.wait_cycles = wait_cycles_now(); a.debug_no_copy = g_tune_no_copy;
     const int E = dtype == AS_F32 ? 4 : 8;
     const size_t esz = dtype == AS_F32 ? 4 : 2;
@@ -854,6 +856,7 @@ static int decode_common(const void* d_table, int dtype, int V, long long ld, co
         a.lanes = lanes; a.V = V; a.top_k = top_k;
         a.lat_N = 0; a.lat_j0 = 0; a.lat_u = 0.0;
         a.rows = V;
+        a.xp_state = nullptr; a.xp_N = 0;
         a.wait_cycles = wait_cycles_now(); a.debug_no_copy = g_tune_no_copy;
         cudaError_t e;
         bool served = true;
@@ -1063,6 +1066,40 @@ int as_decode_bigram_xp(const void* d_table, int dtype, int V, long long ld, con
         n.seq = d_seq; n.len = d_len; n.lane_status = d_lane_status; n.xp_state = state;
         rc = launch_nocut<NC_DECODE_XP>(n, dtype, temp, di->sms, st);
         if (rc != AS_ERR_UNSUPPORTED) return rc;
+    }
+    if ((top_k > 0 || top_p < 1.0) && g_tune_path == 0 && T > 0) {
+        // lanes with a cut: one launch of the streaming kernel per step, rows gathered from the table,
+        // the states advanced in place (as the fp64 loop does with its codes)
+        StepArgs a;
+        a.logits = d_table; a.codes = nullptr; a.codes_out = nullptr;
+        a.diag = {nullptr, nullptr, nullptr, d_lane_status, nullptr};
+        a.ld = ld; a.inv_tau = inv_tau; a.top_p = top_p; a.scale2 = (float)(1.4426950408889634 / temp);
+        a.lanes = lanes; a.V = V; a.top_k = top_k;
+        a.lat_N = 0; a.lat_j0 = 0; a.lat_u = 0.0;
+        a.rows = V;
+        a.xp_state = state; a.xp_N = N;
+        a.wait_cycles = wait_cycles_now(); a.debug_no_copy = g_tune_no_copy;
+        const int E = dtype == AS_F32 ? 4 : 8;
+        const size_t row_bytes = (size_t)((V + E - 1 + E - 1) / E) * 16;
+        const int nsl = (int)((row_bytes + SK_STAGE_BYTES - 1) / SK_STAGE_BYTES);
+        const bool resident = nsl <= SK_RES_STAGES && !(g_tune_stages > 0 && g_tune_stages < nsl);
+        const bool fast = (top_k > 0 && top_k <= (resident ? SK_K0_RESIDENT : SK_K0_STREAMED)) || (top_k == 0 && top_p < 1.0);
+        if (resident || fast) {
+            cudaError_t e;
+            decode_setup_kernel<<<grid_for(lanes, di->sms, 8), 256, 0, st>>>(d_prev, nullptr, lanes, 1, 0.0, V, T, d_len, nullptr, d_seq, d_lane_status);
+            if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "decode set-up kernel launch");
+            for (int t = 0; t < T; ++t) {
+                a.tokens = d_seq + t; a.tok_stride = T;
+                a.row_idx = t == 0 ? d_len : d_seq + (t - 1);
+                a.idx_stride = t == 0 ? 1 : T;
+                a.eos = (t == 0 || eos < 0) ? -1 : eos;
+                rc = launch_streaming(a, dtype, true, di->sms, st);
+                if (rc != AS_OK) return rc == AS_ERR_UNSUPPORTED ? set_err(AS_ERR_CUDA, "streaming kernel refused a decode step") : rc;
+            }
+            decode_wrapup_kernel<<<grid_for(lanes, di->sms, 8), 256, 0, st>>>(d_seq, lanes, T, d_len);
+            if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "decode wrap-up kernel launch");
+            return AS_OK;
+        }
     }
     const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
     if (dtype == AS_F32)

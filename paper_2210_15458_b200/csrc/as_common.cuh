@@ -467,6 +467,60 @@ __device__ __forceinline__ int xp_subrow(const double (&ev)[E], int lane, double
     return L;
 }
 
+// The same selection over one list of tokens in index order, lane l owning the positions [b, en)
+// (masses through ev(i)); the list is the whole kept set: it starts at cell 0 and its last token
+// with mass ends at 2^32.  Returns the owning lane (position pidx, cells [plo, phi), mass pe) or -1;
+// Z receives the total mass.  Uniform.
+template <class F>
+__device__ __forceinline__ int xp_span(int b, int en, F&& ev, int lane, unsigned long long tcell, int& pidx,
+                                       unsigned long long& plo, unsigned long long& phi, double& pe, double& Z) {
+    double local = 0.0;
+    int klast = -1;
+    for (int i = b; i < en; ++i) {
+        const double m = ev(i);
+        local += m;
+        if (m > 0.0) klast = i;
+    }
+    const double incl = warp_incl_scan_d(local, lane);
+    double excl = __shfl_up_sync(FULL, incl, 1);
+    if (lane == 0) excl = 0.0;
+    Z = __shfl_sync(FULL, incl, 31);
+    const unsigned massive = __ballot_sync(FULL, local > 0.0);
+    if (!massive) return -1;
+    const double K = 4294967296.0 / Z;
+    const int Llast = 31 - __clz(massive);
+    const unsigned long long endc = lane == Llast ? XP_TOP : xp_cell(incl, K);
+    const unsigned before = massive & ((1u << lane) - 1u);
+    const unsigned long long prev_end = __shfl_sync(FULL, endc, before ? 31 - __clz(before) : 0);
+    unsigned long long lo = before ? prev_end : 0ull;
+    int pick = -1;
+    unsigned long long mylo = 0, myhi = 0;
+    double mye = 1.0;
+    double S = excl;
+    for (int i = b; i < en; ++i) {
+        const double m = ev(i);
+        if (m > 0.0) {
+            unsigned long long hi;
+            if (i == klast) {
+                hi = endc;
+            } else {
+                S += m;
+                hi = xp_cell(S, K);
+            }
+            if (pick < 0 && hi > tcell) { pick = i; mylo = lo; myhi = hi; mye = m; }
+            lo = hi;
+        }
+    }
+    const unsigned bal = __ballot_sync(FULL, pick >= 0);
+    if (!bal) return -1;
+    const int L = __ffs(bal) - 1;
+    pidx = __shfl_sync(FULL, pick, L);
+    plo = __shfl_sync(FULL, mylo, L);
+    phi = __shfl_sync(FULL, myhi, L);
+    pe = __shfl_sync(FULL, mye, L);
+    return L;
+}
+
 // Result of one decode step for one lane, identical in every thread of the CTA.
 struct LaneResult {
     int token;

@@ -110,6 +110,10 @@ struct StepArgs {
     int tok_stride;
     int eos;
     int rows;
+    // extended-precision decode (builds with XP): the lanes' decoder states [lanes, 4], read and
+    // written in place, and the lattice size that drives their digit source
+    unsigned long long* xp_state;
+    int xp_N;
     // bound on every mbarrier wait, in clock cycles; when it runs out the lane reports ST_TIMEOUT
     long long wait_cycles;
     // test of the time-out path only: the copy-issuing thread issues nothing, so every wait runs out

@@ -74,6 +74,7 @@ struct StreamSmemT {
     int vec_count;
     int cand_count;
     int poisoned;        // a bounded wait ran out: stop issuing / stop waiting
+    unsigned long long xp_lo, xp_hi;   // extended-precision steps: the chosen token's cells
     int prod_done;       // the copy-issuing thread has left; prod_st / prod_round say what it armed
     unsigned prod_st, prod_round;
     int b_i[4];
@@ -134,11 +135,11 @@ __device__ __forceinline__ uint32_t warp_select16(uint32_t a16, uint32_t b16, in
 // entries.  depth_key: every element of the row with key >= depth_key is in the list, so ranks
 // are exact down to that key.  Returns false if the list cannot decide the lane (uniformly in all
 // threads); `out` is set in thread 0 only.
-template <int DT, int NT, class Sync, class StreamSmem>
+template <int DT, int NT, class Sync, class StreamSmem, bool XP = false>
 __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long* src, unsigned long long* dst,
                                              double* e, int C, uint32_t depth_key, double c, double lmax,
                                              double inv_tau, int top_k, double top_p, double tail,
-                                             LaneResult& out) {
+                                             LaneResult& out, unsigned long long tcell = 0) {
     using Tr = Traits<DT>;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // (src[C..C+3] are zero: the caller zero-fills the array before collecting candidates)
@@ -232,7 +233,24 @@ __device__ __noinline__ bool epilogue_ranked(StreamSmem& sm, unsigned long long*
         }
         Sync::sync();
         ASX_MARK(8);
-        if (warp == 0) {
+        if (XP && warp == 0) {
+            // extended-precision step: the token that owns the code's cell among the kept tokens in
+            // index order; its cells go to sm.xp_lo / sm.xp_hi
+            const int per = (n_final + 31) / 32;
+            const int b = min(lane * per, n_final), en = min(b + per, n_final);
+            int pidx = 0;
+            unsigned long long plo = 0, phi = 0;
+            double pe = 1.0, Z = 1.0;
+            const int L = xp_span(b, en, [&](int i) { return e[(uint32_t)src[i]]; }, lane, tcell, pidx, plo, phi, pe, Z);
+            if (lane == 0) {
+                LaneResult r;
+                r.token = L >= 0 ? (int)(src[pidx] >> 32) : -1;
+                r.status = L >= 0 ? ST_OK : ST_NUMERIC; r.n_kept = n_final; r.code_out = 0.0;
+                r.p_tok = pe / Z; r.cdf_lo = (double)plo * (1.0 / 4294967296.0);
+                sm.xp_lo = plo; sm.xp_hi = phi;
+                out = r;
+            }
+        } else if (warp == 0) {
             // lane l owns index-order positions [b, en); up to 4 masses are kept in registers
             const int per = (n_final + 31) / 32;
             const int b = min(lane * per, n_final), en = min(b + per, n_final);
@@ -346,10 +364,10 @@ __device__ __forceinline__ void reread_row(uint4* staging, const char* row, int 
 //      runs again.  Returns false if the window or the list capacity does not suffice.
 constexpr int DP_NB = 1024;
 constexpr float DP_BINS_PER_UNIT = 128.f;
-template <int DT, class StreamSmem>
+template <int DT, class StreamSmem, bool XP = false>
 __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2, double inv_tau, double top_p,
                                             const char* row, uint32_t gmax, float t0f, double tailsum, double c,
-                                            LaneResult& r) {
+                                            LaneResult& r, unsigned long long tcell = 0) {
     using Tr = Traits<DT>;
     using P = Pass<DT>;
     constexpr int E = Tr::E;
@@ -450,8 +468,8 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2,
     if (tsum < 0.0) tsum = 0.0;
     const int C = sm.cand_count;
     if (C <= 0 || C > SK_CAP || !(tsum == tsum) || !(tsum < 1e300)) { ASX_COUNT(3); return false; }
-    const bool ok2 = epilogue_ranked<DT, NT, SyncC, StreamSmem>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, depth_key, c,
-                                                    (double)lmaxf, inv_tau, 0, top_p, tsum, r);
+    const bool ok2 = epilogue_ranked<DT, NT, SyncC, StreamSmem, XP>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, depth_key, c,
+                                                        (double)lmaxf, inv_tau, 0, top_p, tsum, r, tcell);
     if (!ok2) ASX_COUNT(4);
     return ok2;
 }
@@ -513,7 +531,7 @@ __device__ __forceinline__ void mask_lead(uint4& q, int lead) {
     q = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-template <int DT, int CAPV, int MINB, bool UA = false, bool GATHER = false>
+template <int DT, int CAPV, int MINB, bool UA = false, bool GATHER = false, bool XP = false>
 __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const StepArgs a, const int stages) {
     using StreamSmem = StreamSmemT<CAPV>;
     constexpr int SK_CAPV = CAPV;
@@ -770,7 +788,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         if (GATHER && !lane_active(ln)) continue;
         // the code is first looked at just before the epilogue: its 8-byte load queues behind the
         // row copies of the whole grid, and an earlier use would hold up the passes over the row
-        const double c_in = lane_code(a, ln);
+        const double c_in = XP ? 0.5 : lane_code(a, ln);
         const char* row = row_of(ln);
         const int lead = lead_of(ln);
         int bulk_bytes_l = bulk_bytes, bulk_vec_l = bulk_vec, tail_elems_l = tail_elems, nsl_l = nsl;
@@ -1036,6 +1054,13 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         if (blockIdx.x == 0 && tid == 0) { g_asx_marks[20] = nvh; g_asx_marks[21] = C; }
 #endif
         const double c = c_in == 1.0 ? ASX_ONE_BELOW : c_in;
+        XpState xs = {XP_RANGE_TOP, 0ull, 0ull, 0ull};
+        unsigned long long tcell = 0;
+        if (XP) {            // the lane's code comes as the state of an arithmetic decoder
+            xs.range = a.xp_state[(size_t)ln * 4]; xs.code = a.xp_state[(size_t)ln * 4 + 1];
+            if (!xp_state_ok(xs)) { if (!decided) r = failed_lane(c_in, ST_NUMERIC); decided = true; xs.range = XP_RANGE_TOP; xs.code = 0ull; }
+            tcell = xp_target(xs);
+        }
         if (*(volatile int*)&sm.poisoned) {
             r = failed_lane(c_in, ST_TIMEOUT);
             decided = true;
@@ -1043,14 +1068,14 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             r = failed_lane(c_in, ST_NUMERIC);
             decided = true;
         } else if (list_ok && (!want_tail || (tailsum == tailsum && tailsum < 1e300))) {
-            decided = epilogue_ranked<DT, NT, SyncC, StreamSmem>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, t0key, c,
-                                                     lmax, a.inv_tau, a.top_k, a.top_p, tailsum, r);
+            decided = epilogue_ranked<DT, NT, SyncC, StreamSmem, XP>(sm, sm.u.ep.cand, sm.u.ep.v.rk.srt, sm.u.ep.v.rk.e, C, t0key, c,
+                                                         lmax, a.inv_tau, a.top_k, a.top_p, tailsum, r, tcell);
         }
         if (!decided && want_tail && list_ok && !(UA && lead) && !*(volatile int*)&sm.poisoned) {
             // the nucleus reaches below the exact depth of the list: lower the threshold once
             ASX_COUNT(0);
             if (tid == 0) sm.b_i[2] = C;
-            decided = deepen_nucleus<DT, StreamSmem>(sm, V, scale2, a.inv_tau, a.top_p, row, gmax, t0f, tailsum, c, r);
+            decided = deepen_nucleus<DT, StreamSmem, XP>(sm, V, scale2, a.inv_tau, a.top_p, row, gmax, t0f, tailsum, c, r, tcell);
         }
         if (!decided) {
             ASX_COUNT(5);
@@ -1059,14 +1084,27 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             if (!general_row) general_row = row;          // the row again, from global memory (L2)
             SyncC::sync();
             GenericLane<DT, NT, SyncC> gl(sm.u.gen, general_row, V, general_vec_ok);
-            r = gl.run(c_in, a.inv_tau, a.top_k, a.top_p);
+            bool from_gen = false;
+            if (XP) { r = gl.run_xp(tcell, a.inv_tau, a.top_k, a.top_p); from_gen = true; }
+            else r = gl.run(c_in, a.inv_tau, a.top_k, a.top_p);
+            if (XP && tid == 0 && from_gen) { sm.xp_lo = sm.u.gen.xp_lo; sm.xp_hi = sm.u.gen.xp_hi; }
             path = PATH_GENERAL;
             if (general_release)
                 for (int s = 0; s < nsl_l; ++s) release(s);
         }
         if (resident && staged_ok(ln)) advance(nsl_l);
         if (tid == 0) {
-            if (GATHER) {
+            if (XP) {
+                a.tokens[(size_t)ln * a.tok_stride] = r.token;
+                if (r.status == ST_OK) {         // narrow the interval to the token's cells, shift digits in
+                    xs.q = a.xp_state[(size_t)ln * 4 + 2]; xs.packed = a.xp_state[(size_t)ln * 4 + 3];
+                    xp_advance(xs, sm.xp_lo, sm.xp_hi, (unsigned)a.xp_N);
+                    a.xp_state[(size_t)ln * 4] = xs.range; a.xp_state[(size_t)ln * 4 + 1] = xs.code;
+                    a.xp_state[(size_t)ln * 4 + 2] = xs.q; a.xp_state[(size_t)ln * 4 + 3] = xs.packed;
+                } else if (a.diag.lane_status) {
+                    a.diag.lane_status[ln] = r.status;
+                }
+            } else if (GATHER) {
                 a.tokens[(size_t)ln * a.tok_stride] = r.token;
                 a.codes_out[ln] = r.code_out;
                 if (a.diag.lane_status && r.status != ST_OK) a.diag.lane_status[ln] = r.status;
