@@ -47,8 +47,11 @@
  * nucleus keeps the smallest probability-sorted prefix with mass >= top_p;
  * -inf logits are masked; NaN / +inf logits, an all-masked row or a code
  * outside [0,1] give status ORC_ERR_NUMERIC, token -1, code unchanged; pad
- * id is -1.  Parity unpinned by the paper for: modifier order, pad id, the
- * non-finite policy (they are pinned only by these stated readings).
+ * id is -1; the typical cut takes the nucleus's place; the extended-precision
+ * step quantises each step's CDF to 2^32 cells.  Parity unpinned by the paper
+ * for: modifier order (typical decoding's place included), pad id, the
+ * non-finite policy, the choice of 2^32 cells (they are pinned only by these
+ * stated readings; the arithmetic that follows from them is pinned exactly).
  *
  * All sums are Neumaier-compensated so the oracle's own rounding (~1e-16) is
  * far below every tolerance used against it.
