@@ -393,6 +393,11 @@ int as_reward_mean(const int32_t *d_seq, const int32_t *d_len, int S, int N, int
  *                         every wait runs out: exists only so that a test can exercise the
  *                         AS_ERR_TIMEOUT path without any copy in flight; use it with a small
  *                         AS_TUNE_WAIT_KCYCLES
+ *   AS_TUNE_RADIX_NUCLEUS 1 = the general routine of the step calls finds every nucleus by its
+ *                         radix select on mass-weighted keys.  By default a nucleus without a
+ *                         top-k is first looked for through bins of the logit value (two passes
+ *                         over the row for a nucleus of any width), and the radix select takes
+ *                         the rows that the bins cannot settle; the results are the same
  * Returns AS_ERR_INVALID_ARG for an unknown key or value.  The keys are process-wide; a launch
  * reads each once (concurrent calls see the old or the new value).
  */
@@ -404,6 +409,7 @@ int as_reward_mean(const int32_t *d_seq, const int32_t *d_len, int S, int N, int
 #define AS_TUNE_SERIAL_LAUNCH 6
 #define AS_TUNE_WAIT_KCYCLES 7
 #define AS_TUNE_DEBUG_NO_COPY 8
+#define AS_TUNE_RADIX_NUCLEUS 9
 int as_tune(int key, int value);
 
 /* Text of the calling thread's most recent error ("" if none). Never NULL. */

@@ -36,6 +36,7 @@ TUNE_MIN_CTAS = 5
 TUNE_SERIAL_LAUNCH = 6
 TUNE_WAIT_KCYCLES = 7
 TUNE_DEBUG_NO_COPY = 8
+TUNE_RADIX_NUCLEUS = 9
 
 EXPORTS = ["as_lattice_codes", "as_lattice_codes_variant", "as_step", "as_step_typical", "as_step_lattice", "as_step_host", "as_step_host_work_bytes", "as_step_host_static",
            "as_decode_bigram",

@@ -24,7 +24,7 @@ struct Tune {
     void operator=(int x) { v.store(x, std::memory_order_relaxed); }
 };
 static Tune g_tune_path, g_tune_cluster, g_tune_ctas, g_tune_stages, g_tune_minb, g_tune_serial,
-    g_tune_wait_kcycles, g_tune_no_copy;
+    g_tune_wait_kcycles, g_tune_no_copy, g_tune_radix_nucleus;
 
 static long long wait_cycles_now() {
     const int k = g_tune_wait_kcycles;
@@ -166,6 +166,19 @@ static int launch_stream_ua(const StepArgs& a, int stages, int sms, int want_per
     cfg.numAttrs = (!g_tune_serial && grid == a.lanes) ? 1 : 0;
     e = cudaLaunchKernelEx(&cfg, kern, a, stages);
     if (e != cudaSuccess) return cuda_fail(e, "streaming step kernel launch");
+    // the lanes it leaves undecided: the general routine, four CTAs per SM, set up while the
+    // streaming kernel drains
+    cudaLaunchConfig_t cfd = {};
+    long long gd = 4LL * sms;
+    if (gd > a.lanes) gd = a.lanes;
+    cfd.gridDim = dim3((unsigned)gd);
+    cfd.blockDim = dim3(DL_NT);
+    cfd.dynamicSmemBytes = 0;
+    cfd.stream = st;
+    cfd.attrs = attr;
+    cfd.numAttrs = g_tune_serial ? 0 : 1;
+    e = cudaLaunchKernelEx(&cfd, deferred_lanes_kernel<DT, GATHER, XP>, a);
+    if (e != cudaSuccess) return cuda_fail(e, "deferred lanes kernel launch");
     return AS_OK;
 }
 
@@ -261,7 +274,7 @@ template <int DT>
 __global__ void __launch_bounds__(GEN_NT)
 step_generic_kernel(const void* __restrict__ logits, int lanes, int V, long long ld,
                     const double* codes, int lat_N, int lat_j0, double lat_u, double inv_tau, int top_k,
-                    double top_p, double typical_p, int* __restrict__ tokens, double* codes_out, DiagPtrs diag) {
+                    double top_p, double typical_p, int* __restrict__ tokens, double* codes_out, DiagPtrs diag, int radix_nucleus) {
     __shared__ GenericSmem<GEN_NT> sm;
     for (int ln = blockIdx.x; ln < lanes; ln += gridDim.x) {
         const char* row = reinterpret_cast<const char*>(logits) + (size_t)ln * (size_t)ld * Traits<DT>::BYTES;
@@ -274,6 +287,7 @@ step_generic_kernel(const void* __restrict__ logits, int lanes, int V, long long
             c = codes[ln];
         }
         GenericLane<DT, GEN_NT> g(sm, row, V, vec_ok);
+        g.bins = !radix_nucleus;
         const LaneResult r = g.run(c, inv_tau, top_k, top_p, typical_p);
         if (threadIdx.x == 0) {
             tokens[ln] = r.token;
@@ -563,6 +577,10 @@ int as_tune(int key, int value) {
             if (value != 0 && value != 1) return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_DEBUG_NO_COPY takes 0 or 1");
             g_tune_no_copy = value;
             return AS_OK;
+        case AS_TUNE_RADIX_NUCLEUS:
+            if (value != 0 && value != 1) return set_err(AS_ERR_INVALID_ARG, "AS_TUNE_RADIX_NUCLEUS takes 0 or 1");
+            g_tune_radix_nucleus = value;
+            return AS_OK;
         default:
             return set_err(AS_ERR_INVALID_ARG, "unknown tuning key %d", key);
     }
@@ -613,7 +631,7 @@ static int launch_streaming(StepArgs& a, int dtype, bool unaligned, int sms, cud
     // rows of up to SK_RES_STAGES stages stay resident unless a smaller ring is asked for
     const bool resident = nsl <= SK_RES_STAGES && !(g_tune_stages > 0 && g_tune_stages < nsl);
     a.fast = (a.top_k > 0 && a.top_k <= (resident ? SK_K0_RESIDENT : SK_K0_STREAMED)) || (a.top_k == 0 && a.top_p < 1.0);
-    if (!(resident || a.fast)) return AS_ERR_UNSUPPORTED;
+    if (!a.fast) return AS_ERR_UNSUPPORTED;       // (a top-k beyond the candidate list: the general kernels)
     int stages = resident ? (nsl < 1 ? 1 : nsl) : (g_tune_stages > 0 ? g_tune_stages : 3);
     if (!resident && stages >= nsl) stages = nsl - 1;
     if (dtype == AS_F32) {
@@ -658,7 +676,7 @@ static int step_common(const void* d_logits, int dtype, int lanes, int V, long l
     a.lat_N = lat_N; a.lat_j0 = lat_j0; a.lat_u = lat_u;
     a.row_idx = nullptr; a.idx_stride = 1; a.tok_stride = 1; a.eos = -1; a.rows = 0;
     a.xp_state = nullptr; a.xp_N = 0;
-    a.wait_cycles = wait_cycles_now(); a.debug_no_copy = g_tune_no_copy;
+    a.wait_cycles = wait_cycles_now(); a.debug_no_copy = g_tune_no_copy; a.radix_nucleus = g_tune_radix_nucleus;
     const int E = dtype == AS_F32 ? 4 : 8;
     const size_t esz = dtype == AS_F32 ? 4 : 2;
     // some row starts off a 16-byte boundary: it is read from the boundary below, up to E-1 elements longer
@@ -690,9 +708,9 @@ static int step_common(const void* d_logits, int dtype, int lanes, int V, long l
     }
     const int grid = grid_for(lanes, di->sms, g_tune_ctas > 0 ? g_tune_ctas : 4);
     if (dtype == AS_F32)
-        step_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, lat_N, lat_j0, lat_u, inv_tau, top_k, top_p, typical_p, d_tokens, d_codes_out, dp);
+        step_generic_kernel<DT_F32><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, lat_N, lat_j0, lat_u, inv_tau, top_k, top_p, typical_p, d_tokens, d_codes_out, dp, (int)g_tune_radix_nucleus);
     else
-        step_generic_kernel<DT_BF16><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, lat_N, lat_j0, lat_u, inv_tau, top_k, top_p, typical_p, d_tokens, d_codes_out, dp);
+        step_generic_kernel<DT_BF16><<<grid, GEN_NT, 0, st>>>(d_logits, lanes, V, ld, d_codes, lat_N, lat_j0, lat_u, inv_tau, top_k, top_p, typical_p, d_tokens, d_codes_out, dp, (int)g_tune_radix_nucleus);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "step kernel launch");
     return AS_OK;
@@ -857,7 +875,7 @@ static int decode_common(const void* d_table, int dtype, int V, long long ld, co
         a.lat_N = 0; a.lat_j0 = 0; a.lat_u = 0.0;
         a.rows = V;
         a.xp_state = nullptr; a.xp_N = 0;
-        a.wait_cycles = wait_cycles_now(); a.debug_no_copy = g_tune_no_copy;
+        a.wait_cycles = wait_cycles_now(); a.debug_no_copy = g_tune_no_copy; a.radix_nucleus = g_tune_radix_nucleus;
         cudaError_t e;
         bool served = true;
         for (int t = 0; t < T && served; ++t) {
@@ -873,7 +891,7 @@ static int decode_common(const void* d_table, int dtype, int V, long long ld, co
                 const int nsl = (int)((row_bytes + SK_STAGE_BYTES - 1) / SK_STAGE_BYTES);
                 const bool resident = nsl <= SK_RES_STAGES && !(g_tune_stages > 0 && g_tune_stages < nsl);
                 probe.fast = (top_k > 0 && top_k <= (resident ? SK_K0_RESIDENT : SK_K0_STREAMED)) || (top_k == 0 && top_p < 1.0);
-                if (!(resident || probe.fast)) { served = false; break; }
+                if (!probe.fast) { served = false; break; }
                 const int sg = grid_for(lanes, di->sms, 8);
                 decode_setup_kernel<<<sg, 256, 0, st>>>(d_tok, d_codes_in, lanes, N, u, V, T, d_len, d_codes_final, d_seq, d_lane_status);
                 if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "decode set-up kernel launch");
@@ -1078,7 +1096,7 @@ int as_decode_bigram_xp(const void* d_table, int dtype, int V, long long ld, con
         a.lat_N = 0; a.lat_j0 = 0; a.lat_u = 0.0;
         a.rows = V;
         a.xp_state = state; a.xp_N = N;
-        a.wait_cycles = wait_cycles_now(); a.debug_no_copy = g_tune_no_copy;
+        a.wait_cycles = wait_cycles_now(); a.debug_no_copy = g_tune_no_copy; a.radix_nucleus = g_tune_radix_nucleus;
         const int E = dtype == AS_F32 ? 4 : 8;
         const size_t row_bytes = (size_t)((V + E - 1 + E - 1) / E) * 16;
         const int nsl = (int)((row_bytes + SK_STAGE_BYTES - 1) / SK_STAGE_BYTES);

@@ -162,6 +162,27 @@ __device__ __forceinline__ void fill_exp_table(double* tbl, int tid) {
     if (tid < 64) tbl[tid] = ASX_T64[tid];
 }
 
+// Additions to shared memory without a return value, on the shared-space address: through a
+// pointer whose address space the compiler cannot see they would be issued as generic atomics,
+// which take tens of cycles per lane on shared memory.
+__device__ __forceinline__ void red_shared_add(float* p, float v) {
+    asm volatile("red.shared.add.f32 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(p)), "f"(v) : "memory");
+}
+__device__ __forceinline__ void red_shared_add(int* p, int v) {
+    asm volatile("red.shared.add.s32 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ void red_shared_or(unsigned* p, unsigned v) {
+    asm volatile("red.shared.or.b32 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(p)), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned atom_shared_add(unsigned* p, unsigned v) {
+    unsigned old;
+    asm volatile("atom.shared.add.u32 %0, [%1], %2;" : "=r"(old) : "r"((uint32_t)__cvta_generic_to_shared(p)), "r"(v) : "memory");
+    return old;
+}
+__device__ __forceinline__ void red_shared_add(unsigned long long* p, unsigned long long v) {
+    asm volatile("red.shared.add.u64 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(p)), "l"(v) : "memory");
+}
+
 // ---------------------------------------------------------------------------
 // Warp primitives (all 32 lanes active).
 // ---------------------------------------------------------------------------

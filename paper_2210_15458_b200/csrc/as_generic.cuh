@@ -152,7 +152,7 @@ struct GenericLane {
     }
     __device__ __forceinline__ void put_chunk(int ci, double local) {      // lane 0 of the chunk's warp
         sm.chunk_sum[ASX_AT(ci, MAXCH + 1, 82)] = local;
-        if (local > 0.0) atomicOr(&sm.chunk_has[ci >> 5], 1u << (ci & 31));
+        if (local > 0.0) red_shared_or(&sm.chunk_has[ci >> 5], 1u << (ci & 31));
     }
 
     // typical cut: order key of a token, larger = nearer the mean scaled logit
@@ -669,21 +669,578 @@ struct GenericLane {
         n_kept = acc_c + (int)r;
     }
 
-    // Steps 1-4 of the general routine: the kept set as a predicate `p`, its size, and in
-    // chunk_sum the exclusive scan of the kept masses per chunk (chunk_sum[nchunks] = Z).
-    // Needs inv_tau set and the exp table filled; returns ST_OK or ST_NUMERIC.
-    __device__ __forceinline__ int prepare(int top_k, double top_p, Pred& p, int& n_kept, double typical_p = 1.0) {
-        // ---- 1. extremes and finite count
+    // ------------------------------------------------------------------ nucleus through value bins
+    // The nucleus threshold of a row without a top-k, for nuclei of any width, in two passes over
+    // the row instead of the radix select's five with fp64 masses:
+    //   B. counts of the elements in WB bins by depth below the row maximum, d = (l_max - l) / temp
+    //      in octaves, 128 bins per octave over 24 octaves and one bin for the rest (integer
+    //      additions to shared memory are native; fp32 ones are compare-and-swap loops).  The
+    //      binning is a monotone function of the key: every key of a bin is above every key of the
+    //      next.  A bin's count times the masses at its two edges bounds its mass from both sides,
+    //      so the cumulative bounds bracket the bin in which the nucleus ends: bins [b_hi, b_lo].
+    //   C. exact fp64 masses: elements above the bracket are kept (their masses go to the chunk
+    //      sums right away), elements below it only add to Z, the bracket's elements (<= WCAP) are
+    //      listed and ranked exactly (key descending, index ascending).  The first rank at which the
+    //      exact prefix reaches top_p * Z closes the kept set.
+    // Every decision is taken on exact fp64 sums; the bins only say where to look.  Whatever they
+    // cannot settle (a bracket with more than WCAP elements or reaching the last bin, a prefix within
+    // rounding of the target) returns 0 and the radix select decides.
+    static constexpr int WB = 3072;
+    static constexpr int WCAP = 1024;
+    bool bins = true;                          // false: always the radix select
+
+    __device__ __forceinline__ float wdepth(uint32_t key, float lmax_f, float s2) const {
+        return (lmax_f - Tr::value_f(key)) * s2;
+    }
+    // exclusive scan of one value per thread over the block, thread order; `total` to every thread
+    __device__ __forceinline__ double block_excl_scan_d(double v, double& total) {
+        const double incl = warp_incl_scan_d(v, lane);
+        if (lane == 31) sm.red_d[warp] = incl;
+        Sync::sync();
+        double off = 0.0;
+        total = 0.0;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+            if (w < warp) off += sm.red_d[w];
+            total += sm.red_d[w];
+        }
+        Sync::sync();
+        return off + (incl - v);
+    }
+    __device__ __forceinline__ int block_excl_scan_i(int v, int& total) {
+        const int incl = warp_incl_scan_i(v, lane);
+        if (lane == 31) sm.red_i[warp] = incl;
+        Sync::sync();
+        int off = 0;
+        total = 0;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+            if (w < warp) off += sm.red_i[w];
+            total += sm.red_i[w];
+        }
+        Sync::sync();
+        return off + (incl - v);
+    }
+    __device__ __forceinline__ int chunk_of_index(int idx) const { return (idx / E) / (32 * R); }
+
+    // Bins of one counting pass: `nfine` bins of 1 / scale octaves each over depths from d0 down; the
+    // bracket is bins bhi..blo.
+    struct WBracket {
+        float d0, scale;
+        int nfine;
+        int bhi, blo;
+    };
+    // bin of an element at depth d >= d0, or nfine for what lies past the bins
+    __device__ __forceinline__ static int wbin(float d, const WBracket& w) {
+        const float rel = (d - w.d0) * w.scale;
+        return rel < (float)w.nfine ? (int)rel : w.nfine;
+    }
+    // upper edge (smallest depth) of bin b
+    __device__ __forceinline__ static float wedge(int b, const WBracket& w) { return w.d0 + (float)b / w.scale; }
+    // class of an element at depth d: 0 above the bracket (kept), 1 inside it, 2 below it; through the
+    // very expression that filled the bins, so that counts and classes agree element by element
+    __device__ __forceinline__ static int wclass(float d, const WBracket& w) {
+        if (d < w.d0) return 0;
+        const int b = wbin(d, w);
+        return b < w.bhi ? 0 : (b <= w.blo ? 1 : 2);
+    }
+
+    __device__ int nucleus_by_bins(double top_p, int nfin_in, Pred& p, int& n_kept) {
+        int nfin = nfin_in;                          // < 0: not known yet, the first level counts it
+        // This object lives in local memory (its member functions are called out of line), and a store
+        // through a shared-memory pointer may alias it as far as the compiler can tell: members used in
+        // the loops would be loaded again after every such store.  Locals of the same names shadow them
+        // here and stay in registers.
+        GenericSmem<NT>& sm = this->sm;
+        const void* const row = this->row;
+        const int V = this->V, nvec = this->nvec, R = this->R, nchunks = this->nchunks;
+        const bool vec_ok = this->vec_ok;
+        const int tid = this->tid, lane = this->lane, warp = this->warp;
+        const double lmax = this->lmax, inv_tau = this->inv_tau;
+        const double* const exp_tbl = sm.exp_tbl;
+        double* const chunk_sum = sm.chunk_sum;
+        unsigned* const chunk_has = sm.chunk_has;
+        auto mass = [&](uint32_t key) -> double { return exp_nonpos(((double)Tr::value_f(key) - lmax) * inv_tau, exp_tbl); };
+        auto put_chunk = [&](int ci, double local) {
+            chunk_sum[ASX_AT(ci, MAXCH + 1, 82)] = local;
+            if (local > 0.0) red_shared_or(&chunk_has[ci >> 5], 1u << (ci & 31));
+        };
+        auto chunk_of_index = [&](int idx) -> int { return (idx / E) / (32 * R); };
+        int* wbc = reinterpret_cast<int*>(sm.hist_mass);                        // WB counts; later
+        unsigned long long* wcand = reinterpret_cast<unsigned long long*>(sm.hist_mass);   // WCAP composites
+        unsigned long long* acc_hi = reinterpret_cast<unsigned long long*>(sm.hist_cnt);   // MAXCH fixed-point sums
+        unsigned long long* acc_lo = reinterpret_cast<unsigned long long*>(sm.chunk_eq);   // (chunk_eq + chunk_eq2)
+        static_assert(sizeof(sm.hist_mass) + sizeof(sm.hist_cnt) >= WB * 4 && sizeof(sm.hist_mass) >= WCAP * 8,
+                      "bins and list share the histograms' space");
+        static_assert(sizeof(sm.hist_cnt) >= MAXCH * 8 && 2 * sizeof(sm.chunk_eq) >= MAXCH * 8 + 8, "fixed-point sums");
+        const float lmax_f = (float)lmax;
+        const float s2 = (float)(inv_tau * 1.4426950408889634);
+
+        // ---- B. bin counts, at most twice: 128 bins per octave from the maximum down; if the bracket
+        //         that gives holds more elements than the list, its range again with finer bins
+        WBracket wb;
+        wb.d0 = 0.f; wb.scale = 128.f; wb.nfine = WB; wb.bhi = 0; wb.blo = 0;
+        // elements above d0 / past the bins: bounds of their mass, their number
+        double base_lo = 0.0, base_hi = 0.0, Zf = 0.0;
+        int base_c = 0, tail_c = 0;
+        int n_in = 0, n_br = 0;
+        for (int level = 0;; ++level) {
+            for (int i = tid; i < WB; i += NT) wbc[i] = 0;
+            Sync::sync();
+            int deep = 0;                              // past the bins: counted in a register, they are many
+            const int nall = wb.nfine;
+            // fp32 masses in registers, four partial sums: of every element (first level: that is Z to
+            // 4e-5), of the elements above the window (second level)
+            float msum[4] = {0.f, 0.f, 0.f, 0.f};
+            {
+                constexpr int U = 4;                   // loads in flight per thread
+                for (int v0 = tid; v0 < nvec; v0 += U * NT) {
+                    uint32_t k[U][E];
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        const int vi = v0 + u * NT;
+                        if (vi < nvec) {
+                            load_vec_keys<DT>(row, V, vi, vec_ok, k[u]);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < E; ++e) k[u][e] = Tr::KEY_NINF;
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+#pragma unroll
+                        for (int e = 0; e < E; ++e) {
+                            if (k[u][e] > Tr::KEY_NINF) {
+                                const float d = wdepth(k[u][e], lmax_f, s2);
+                                if (level == 0 || d < wb.d0) msum[e & 3] += ex2_approx(-d);
+                                if (d >= wb.d0) {
+                                    const int b = wbin(d, wb);
+                                    if (b < nall) red_shared_add(&wbc[b], 1);
+                                    else ++deep;
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            {
+                double msum_all;
+                (void)block_excl_scan_d(((double)msum[0] + (double)msum[1]) + ((double)msum[2] + (double)msum[3]), msum_all);
+                if (level == 0) {
+                    // (the first level's bins end 24 octaves down; the elements past them are only counted)
+                    int all_deep;
+                    (void)block_excl_scan_i(deep, all_deep);
+                    tail_c = all_deep;
+                    Zf = msum_all;
+                } else {
+                    base_lo = msum_all * (1.0 - 1e-4);
+                    base_hi = msum_all * (1.0 + 1e-4);
+                }
+            }
+            Sync::sync();
+            // Cumulative bounds in bin order, a run of consecutive bins per thread.  An element of
+            // bin b has its mass in (2^-edge(b+1), 2^-edge(b)], edge(b) = d0 + b / scale; the factor
+            // 1e-3 covers the rounding of d.  b_hi: first bin at which the upper bound of the mass so
+            // far reaches the lowest possible target; b_lo: first bin at which the lower bound
+            // reaches the highest possible target.
+            constexpr int PERB = (WB + NT - 1) / NT;
+            const int b0 = min(tid * PERB, nall), b1 = min(b0 + PERB, nall);
+            double s_lo = 0.0, s_hi = 0.0;
+            int s_c = 0;
+            for (int b = b0; b < b1; ++b) {
+                const int c = wbc[b];
+                s_hi += (double)c * (double)ex2_approx(-wedge(b, wb));
+                s_lo += (double)c * (double)ex2_approx(-wedge(b + 1, wb));
+                s_c += c;
+            }
+            double tot_lo, tot_hi;
+            int tot_c;
+            const double run_lo0 = base_lo + block_excl_scan_d(s_lo, tot_lo);
+            const double run_hi0 = base_hi + block_excl_scan_d(s_hi, tot_hi);
+            const int run_c0 = base_c + block_excl_scan_i(s_c, tot_c);
+            const double Z_lo = Zf * (1.0 - 1e-4), Z_hi = Zf * (1.0 + 1e-4);      // (the fp32 sum of every mass)
+            if (nfin < 0) nfin = base_c + tot_c + tail_c;
+            if (base_c + tot_c + tail_c != nfin) return 0;
+            if (tid == 0) { sm.b_i[0] = INT_MAX; sm.b_i[1] = INT_MAX; sm.b_i[2] = -1; sm.b_i[3] = -1; }
+            Sync::sync();
+            const double t_lo = top_p * Z_lo * (1.0 - 1e-3), t_hi = top_p * Z_hi * (1.0 + 1e-3);
+            {
+                double r_lo = run_lo0, r_hi = run_hi0;
+                int first_hi = INT_MAX, first_lo = INT_MAX, last = -1;
+                for (int b = b0; b < b1; ++b) {
+                    const int c = wbc[b];
+                    if (c > 0) {
+                        r_hi += (double)c * (double)ex2_approx(-wedge(b, wb));
+                        r_lo += (double)c * (double)ex2_approx(-wedge(b + 1, wb));
+                        if (first_hi == INT_MAX && r_hi >= t_lo) first_hi = b;
+                        if (first_lo == INT_MAX && r_lo >= t_hi) first_lo = b;
+                        last = b;
+                    }
+                }
+                if (first_hi != INT_MAX) atomicMin(&sm.b_i[0], first_hi);
+                if (first_lo != INT_MAX) atomicMin(&sm.b_i[1], first_lo);
+                if (last >= 0) atomicMax(&sm.b_i[2], last);
+            }
+            Sync::sync();
+            const int bhi = sm.b_i[0];
+            int blo = sm.b_i[1];
+            const int last_bin = sm.b_i[2];
+            Sync::sync();
+            if (bhi == INT_MAX) return 0;               // the nucleus ends past the bins
+            if (blo == INT_MAX) {
+                if (tail_c > 0) return 0;               // ... or may do so
+                blo = last_bin;                         // the target sits at the very end of the mass
+            }
+            // counts at the bracket's two ends
+            {
+                int c_run = run_c0;
+                for (int b = b0; b < b1; ++b) {
+                    if (b == bhi) sm.b_i[2] = c_run;
+                    c_run += wbc[b];
+                    if (b == blo) sm.b_i[3] = c_run;
+                }
+            }
+            Sync::sync();
+            n_in = sm.b_i[2];
+            const int thru_c = sm.b_i[3];
+            n_br = thru_c - n_in;
+            Sync::sync();                               // the bins are dead from here
+            if (thru_c < 0 || blo < bhi || n_br < 1) return 0;
+            wb.bhi = bhi;
+            wb.blo = blo;
+            if (n_br <= WCAP) break;
+            if (level == 1) return 0;
+            // finer bins over the bracket's range: the largest power-of-two scale under which it fits
+            const float w_lo = wedge(bhi, wb), w_hi = wedge(blo + 1, wb);
+            const float width = w_hi - w_lo;
+            float sc = 1.f;
+            while (width * (sc * 2.f) <= (float)WB && sc < 16777216.f) sc *= 2.f;
+            if (sc <= wb.scale) return 0;               // (cannot be refined)
+            tail_c = nfin - thru_c;
+            base_c = n_in;                              // (their mass: summed in the next pass)
+            wb.d0 = w_lo;
+            wb.scale = sc;
+            wb.nfine = (int)ceilf(width * sc);          // exactly the bracket's range
+            wb.bhi = 0; wb.blo = 0;
+        }
+
+        // The classes as key thresholds (the class is a monotone function of the key): K0 the smallest
+        // key above the bracket, K1 the smallest key not below it; two integer compares per element
+        // instead of the depth arithmetic.
+        uint32_t K0, K1;
+        {
+            auto first_key = [&](int cls_max) -> uint32_t {     // smallest key of class <= cls_max
+                if (wclass(wdepth(row_kmax, lmax_f, s2), wb) > cls_max) return row_kmax + 1u;
+                uint32_t lo = Tr::KEY_NINF + 1u, hi = row_kmax;   // class(hi) <= cls_max
+                while (lo < hi) {
+                    const uint32_t mid = lo + ((hi - lo) >> 1);
+                    if (wclass(wdepth(mid, lmax_f, s2), wb) <= cls_max) hi = mid; else lo = mid + 1u;
+                }
+                return hi;
+            };
+            K0 = first_key(0);
+            K1 = first_key(1);
+        }
+
+        // ---- C. exact masses: chunk sums of the elements above the bracket, Z's part below it,
+        //         the bracket's elements listed
+        clear_has();
+        if (tid == 0) sm.b_u[0] = 0u;
+        for (int i = tid; i < MAXCH; i += NT) { acc_hi[i] = 0ull; acc_lo[i] = 0ull; }
+        Sync::sync();
+        float below_f[4] = {0.f, 0.f, 0.f, 0.f};     // four partial sums: a few hundred terms each
+        if (warp < nchunks) {
+            const int nq = ((nchunks - warp + NW - 1) / NW) * R;      // this warp's vectors, chunk by chunk
+            auto vi_of = [&](int q) -> int { return ((warp + (q / R) * NW) * R + q % R) * 32 + lane; };
+            auto fetch = [&](int q, uint4& raw, bool& is_raw) {
+                is_raw = false;
+                if (q < nq) {
+                    const int vi = vi_of(q);
+                    if (vec_ok && (vi + 1) * E <= V) {
+                        raw = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(row) + (size_t)vi * 16);
+                        is_raw = true;
+                    }
+                }
+            };
+            constexpr int G = 4;                          // vectors in flight per lane
+            double local = 0.0;
+            for (int q0 = 0; q0 < nq; q0 += G) {
+                uint4 raw[G];
+                bool is_raw[G];
+#pragma unroll
+                for (int g = 0; g < G; ++g) fetch(q0 + g, raw[g], is_raw[g]);
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const int q = q0 + g;
+                    if (q < nq) {
+                        const int vi = vi_of(q);
+                        uint32_t k[E];
+                        if (is_raw[g]) {
+                            Tr::unpack(raw[g], k);
+                        } else if (vi < nvec) {
+                            load_vec_keys<DT>(row, V, vi, vec_ok, k);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < E; ++e) k[e] = Tr::KEY_NINF;
+                        }
+                        unsigned in_mask = 0;
+#pragma unroll
+                        for (int e = 0; e < E; ++e) {
+                            const uint32_t ke = k[e];
+                            if (ke >= K0) {
+                                in_mask |= 1u << e;
+                            } else if (ke >= K1) {
+                                const unsigned slot = atom_shared_add(&sm.b_u[0], 1u);
+                                if (slot < (unsigned)WCAP)
+                                    wcand[slot] = ((unsigned long long)ke << 32) | (uint32_t)~(uint32_t)(vi * E + e);
+                            } else if (ke > Tr::KEY_NINF) {
+                                below_f[e & 3] += ex2_approx(-wdepth(ke, lmax_f, s2));   // fp32 first: see the decision below
+                            }
+                        }
+                        // fp64 masses of the kept ones, one per round: a lane rarely has more than one in a
+                        // vector, and the warp runs as many rounds as its busiest lane
+                        while (in_mask) {
+                            const int e0 = __ffs(in_mask) - 1;
+                            in_mask &= in_mask - 1;
+                            uint32_t ks = k[0];
+#pragma unroll
+                            for (int e = 1; e < E; ++e) if (e0 == e) ks = k[e];
+                            local += mass(ks);
+                        }
+                        if (q % R == R - 1) {
+                            local = warp_sum_d(local);
+                            if (lane == 0) put_chunk(warp + (q / R) * NW, local);
+                            local = 0.0;
+                        }
+                    }
+                }
+            }
+        }
+        double below = ((double)below_f[0] + (double)below_f[1]) + ((double)below_f[2] + (double)below_f[3]);
+        below = warp_sum_d(below);
+        if (lane == 0) sm.red_d[warp] = below;
+        Sync::sync();
+        if ((int)sm.b_u[0] != n_br) return 0;           // (cannot happen: same function of the same keys)
+        double S_out = 0.0;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) S_out += sm.red_d[w];
+        // S_in by warp 0, lanes over the chunks in a fixed order
+        if (warp == 0) {
+            double s_in = 0.0;
+            for (int ci = lane; ci < nchunks; ci += 32) s_in += sm.chunk_sum[ci];
+            s_in = warp_sum_d(s_in);
+            if (lane == 0) sm.b_d[2] = s_in;
+        }
+        // ---- the bracket's elements in rank order: bitonic sort, descending, padded with zeros
+        int P = 32;
+        while (P < n_br) P <<= 1;
+        for (int i = n_br + tid; i < P; i += NT) wcand[i] = 0ull;
+        Sync::sync();
+        for (int kk = 2; kk <= P; kk <<= 1) {
+            for (int j = kk >> 1; j > 0; j >>= 1) {
+                for (int i = tid; i < P / 2; i += NT) {
+                    const int lo = ((i & ~(j - 1)) << 1) | (i & (j - 1)), hi = lo | j;
+                    const bool desc = (lo & kk) == 0;
+                    const unsigned long long x = wcand[lo], y = wcand[hi];
+                    if ((x < y) == desc) { wcand[lo] = y; wcand[hi] = x; }
+                }
+                Sync::sync();
+            }
+        }
+        const double S_in = sm.b_d[2];
+        // exact prefix masses in rank order: `per` consecutive ranks per thread
+        const int per = (P + NT - 1) / NT;               // 1..4
+        double mloc[4] = {0.0, 0.0, 0.0, 0.0};
+        double lsum = 0.0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int j = tid * per + i;
+            if (i < per && j < n_br) { mloc[i] = mass((uint32_t)(wcand[j] >> 32)); lsum += mloc[i]; }
+        }
+        const double wincl = warp_incl_scan_d(lsum, lane);
+        if (lane == 31) sm.red_d[warp] = wincl;
+        if (tid == 0) { sm.b_i[0] = INT_MAX; sm.b_i[1] = 0; sm.b_i[2] = 0; }
+        Sync::sync();
+        double off = 0.0, S_br = 0.0;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+            if (w < warp) off += sm.red_d[w];
+            S_br += sm.red_d[w];
+        }
+        double before[4];
+        {
+            double run = S_in + (off + (wincl - lsum));  // exact prefix before this thread's ranks
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { before[i] = run; run += mloc[i]; }
+        }
+        // The part of Z below the bracket came from fp32 masses (relative error under 4e-5): good
+        // enough unless a prefix lies that close to the target; then that part is summed again in
+        // fp64 and the decision repeated.  Within rounding of fp64 sums the radix select decides.
+        double out_tol = S_out * 4e-5;
+        int r;
+        double pre_r, incl_r;
+        uint32_t T;
+        for (int attempt = 0;; ++attempt) {
+            const double Z = (S_in + S_br) + S_out;
+            const double target = top_p * Z;
+            const double tol = Z * 1e-13 + top_p * out_tol;
+            Sync::sync();
+            if (tid == 0) sm.b_i[0] = INT_MAX;
+            Sync::sync();
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int j = tid * per + i;
+                if (i < per && j < n_br && before[i] + mloc[i] >= target) atomicMin(&sm.b_i[0], j);
+            }
+            Sync::sync();
+            r = sm.b_i[0];
+            bool again = (r == INT_MAX);         // the sums do not reach the target inside the bracket
+            if (!again) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int j = tid * per + i;
+                    if (i < per && j == r) {
+                        sm.b_d[0] = before[i];
+                        sm.b_d[1] = before[i] + mloc[i];
+                        sm.b_u[1] = (uint32_t)(wcand[j] >> 32);
+                    }
+                }
+                Sync::sync();
+                pre_r = sm.b_d[0]; incl_r = sm.b_d[1]; T = sm.b_u[1];
+                again = incl_r - target < tol || target - pre_r < tol;
+            }
+            if (!again) break;
+            if (attempt == 1 || out_tol == 0.0) return 0;
+            // the masses below the bracket once more, in fp64 (below 2^-40 of the maximum an fp32
+            // mass is exact enough by any count)
+            double ex = 0.0;
+            constexpr int U = 4;
+            for (int v0 = tid; v0 < nvec; v0 += U * NT) {
+                uint32_t k[U][E];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int vi = v0 + u * NT;
+                    if (vi < nvec) {
+                        load_vec_keys<DT>(row, V, vi, vec_ok, k[u]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < E; ++e) k[u][e] = Tr::KEY_NINF;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        if (k[u][e] > Tr::KEY_NINF && k[u][e] < K1) {
+                            const float d = wdepth(k[u][e], lmax_f, s2);
+                            ex += d < 40.f ? mass(k[u][e]) : (double)ex2_approx(-d);
+                        }
+                    }
+                }
+            }
+            ex = warp_sum_d(ex);
+            Sync::sync();
+            if (lane == 0) sm.red_d[warp] = ex;
+            Sync::sync();
+            S_out = 0.0;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) S_out += sm.red_d[w];
+            out_tol = 0.0;
+        }
+        Sync::sync();
+        if (tid == 0) { sm.b_i[1] = 0; sm.b_i[2] = 0; }
+        Sync::sync();
+        {
+            int eq = 0, need = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int j = tid * per + i;
+                if (i < per && j < n_br && (uint32_t)(wcand[j] >> 32) == T) { ++eq; need += (j <= r); }
+            }
+            eq = warp_sum_i(eq);
+            need = warp_sum_i(need);
+            if (lane == 0 && eq) { atomicAdd(&sm.b_i[1], eq); atomicAdd(&sm.b_i[2], need); }
+        }
+        // ---- kept elements of the bracket join their chunks' sums: two 64-bit fixed-point parts per
+        //      chunk, so that the sums do not depend on the order in which the additions arrive
+        const double m_top = mass((uint32_t)(wcand[0] >> 32));
+        const int ex_top = ((int)(__double2hiint(m_top) >> 20) & 0x7FF) - 1023;     // m_top in [2^ex, 2^(ex+1))
+        const double sc = __hiloint2double((1023 + 50 - ex_top) << 20, 0);          // m_top * sc in [2^50, 2^51)
+        const bool sc_ok = m_top > 0.0 && ex_top > -900;
+        if (sc_ok) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int j = tid * per + i;
+                if (i < per && j <= r && j < n_br) {
+                    const double f = mloc[i] * sc;                                   // < 2^51
+                    const unsigned long long hi = (unsigned long long)f;             // (truncates)
+                    const unsigned long long lo = (unsigned long long)((f - (double)hi) * 4503599627370496.0);   // * 2^52
+                    const int ci = chunk_of_index((int)~(uint32_t)wcand[j]);
+                    red_shared_add(&acc_hi[ci], hi);
+                    red_shared_add(&acc_lo[ci], lo);
+                }
+            }
+        }
+        Sync::sync();
+        if (!sc_ok) return 0;
+        const int eq_all = sm.b_i[1], need_all = sm.b_i[2];
+        for (int ci = tid; ci < nchunks; ci += NT) {
+            const unsigned long long hi = acc_hi[ci], lo = acc_lo[ci];
+            if (hi | lo) {
+                const double add = ((double)hi + (double)lo * (1.0 / 4503599627370496.0)) / sc;
+                sm.chunk_sum[ci] += add;
+                if (add > 0.0) red_shared_or(&sm.chunk_has[ci >> 5], 1u << (ci & 31));
+            }
+        }
+        Sync::sync();
+        p.T = T;
+        p.need = need_all;
+        p.eq_mode = need_all < eq_all ? 2 : 1;
+        n_kept = n_in + r + 1;
+        if (p.eq_mode == 2) {
+            // chunk_eq[ci] <- elements equal to T in the chunks before ci: all of them are in the list
+            for (int ci = tid; ci <= nchunks; ci += NT) sm.chunk_eq[ci] = 0;
+            Sync::sync();
+            for (int j = tid; j < n_br; j += NT)
+                if ((uint32_t)(wcand[j] >> 32) == T) atomicAdd(&sm.chunk_eq[chunk_of_index((int)~(uint32_t)wcand[j])], 1);
+            Sync::sync();
+            scan_exclusive(sm.chunk_eq, nchunks);
+        }
+        scan_exclusive(sm.chunk_sum, nchunks);
+        return 1;
+    }
+
+    // pass 1: the row's largest key, whether it is a usable row, its finite count
+    __device__ int extremes(unsigned& kmax_out, int& nfin_out) {
+        GenericSmem<NT>& sm = this->sm;              // (locals: see nucleus_by_bins)
+        const void* const row = this->row;
+        const int V = this->V, nvec = this->nvec, tid = this->tid, lane = this->lane, warp = this->warp;
+        const bool vec_ok = this->vec_ok;
         unsigned kmax = 0, kmin = 0xFFFFFFFFu;
         int nfin = 0;
-        for (int vi = tid; vi < nvec; vi += NT) {
-            uint32_t k[E];
-            load_vec_keys<DT>(row, V, vi, vec_ok, k);
+        {
+            constexpr int U = 4;                       // loads in flight per thread
+            for (int v0 = tid; v0 < nvec; v0 += U * NT) {
+                uint32_t k[U][E];
 #pragma unroll
-            for (int e = 0; e < E; ++e) {
-                kmax = max(kmax, k[e]);
-                kmin = min(kmin, k[e]);
-                nfin += (k[e] > Tr::KEY_NINF);
+                for (int u = 0; u < U; ++u) {
+                    const int vi = v0 + u * NT;
+                    if (vi < nvec) {
+                        load_vec_keys<DT>(row, V, vi, vec_ok, k[u]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < E; ++e) k[u][e] = Tr::KEY_NINF;   // (a masked token: allowed, not counted)
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) {
+                        kmax = max(kmax, k[u][e]);
+                        kmin = min(kmin, k[u][e]);
+                        nfin += (k[u][e] > Tr::KEY_NINF);
+                    }
+                }
             }
         }
         kmax = warp_max_u(kmax);
@@ -698,8 +1255,36 @@ struct GenericLane {
             nfin += sm.red_i[w];
         }
         Sync::sync();
+        kmax_out = kmax;
+        nfin_out = nfin;
         if (kmin < Tr::KEY_NINF || kmax >= Tr::KEY_PINF || kmax == Tr::KEY_NINF) return ST_NUMERIC;
+        return ST_OK;
+    }
+
+    // A caller that has already been over the row (every element finite or masked, not all masked)
+    // hands over its largest key; the nucleus through bins then starts without pass 1.
+    bool have_kmax = false;
+    uint32_t known_kmax = 0;
+    uint32_t row_kmax = 0;                     // the row's largest key, once known
+
+    // Steps 1-4 of the general routine: the kept set as a predicate `p`, its size, and in
+    // chunk_sum the exclusive scan of the kept masses per chunk (chunk_sum[nchunks] = Z).
+    // Needs inv_tau set and the exp table filled; returns ST_OK or ST_NUMERIC.
+    __device__ __forceinline__ int prepare(int top_k, double top_p, Pred& p, int& n_kept, double typical_p = 1.0) {
+        const bool nucleus_only = top_k <= 0 && top_p > 0.0 && top_p < 1.0 && !(typical_p > 0.0 && typical_p < 1.0);
+        unsigned kmax = 0;
+        int nfin = -1;
+        if (bins && nucleus_only && have_kmax) {
+            // ---- nucleus without a top-k, maximum known: the value bins settle most rows in two passes
+            lmax = (double)Tr::value_f(known_kmax);
+            row_kmax = known_kmax;
+            if (nucleus_by_bins(top_p, nfin, p, n_kept)) return ST_OK;
+            Sync::sync();
+        }
+        // ---- 1. extremes and finite count
+        if (extremes(kmax, nfin) != ST_OK) return ST_NUMERIC;
         lmax = (double)Tr::value_f(kmax);
+        row_kmax = kmax;
 
         p.T = Tr::KEY_NINF; p.need = 0; p.eq_mode = 0;     // every finite logit
         n_kept = nfin;
@@ -722,6 +1307,14 @@ struct GenericLane {
             p.eq_mode = (p.need < eq) ? 2 : 1;
             n_kept = top_k;
             if (p.eq_mode == 2) tie_prepass(p.T);
+        }
+
+        // ---- nucleus without a top-k: the value bins settle most rows in two passes
+        if (bins && !have_kmax && !(top_k > 0 && top_k < nfin) && top_p > 0.0 && top_p < 1.0 && !(typical_p > 0.0 && typical_p < 1.0)) {
+            if (nucleus_by_bins(top_p, nfin, p, n_kept)) return ST_OK;
+            Sync::sync();
+            p.T = Tr::KEY_NINF; p.need = 0; p.eq_mode = 0;
+            n_kept = nfin;
         }
 
         // ---- 3. masses of the kept set

@@ -110,6 +110,7 @@ struct StepArgs {
     int tok_stride;
     int eos;
     int rows;
+    int radix_nucleus;        // 1: the general routine finds every nucleus by its radix select
     // extended-precision decode (builds with XP): the lanes' decoder states [lanes, 4], read and
     // written in place, and the lattice size that drives their digit source
     unsigned long long* xp_state;
@@ -448,6 +449,7 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
         if (!staged_ok(ln)) {       // unaligned row: the general routine reads it from global memory
             if (is_leader) {
                 GenericLane<DT, NT> g(sm.u.gen, row_of(ln), V, false);
+                g.bins = !a.radix_nucleus;
                 const LaneResult r = g.run(c_in, a.inv_tau, a.top_k, a.top_p);
                 if (tid == 0) write_result(a, ln, r, PATH_GENERAL);
             }
@@ -525,12 +527,14 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
             // no cut: every token is kept; the general routine scans the whole row
             if (CS == 1) {
                 GenericLane<DT, NT> g(sm.u.gen, rowbuf, V, true);
+                g.bins = !a.radix_nucleus;
                 const LaneResult r = g.run(c_in, a.inv_tau, a.top_k, a.top_p);
                 if (tid == 0) write_result(a, ln, r, PATH_GENERAL);
             } else {
                 cluster.sync();
                 if (is_leader) {
                     GenericLane<DT, NT> g(sm.u.gen, row_of(ln), V, true);
+                    g.bins = !a.radix_nucleus;
                     const LaneResult r = g.run(c_in, a.inv_tau, a.top_k, a.top_p);
                     if (tid == 0) write_result(a, ln, r, PATH_GENERAL);
                 }
@@ -612,6 +616,7 @@ __global__ void __launch_bounds__(ST_NT, 1) step_staged_kernel(const StepArgs a)
             if (!done) {
                 __syncthreads();
                 GenericLane<DT, NT> g(sm.u.gen, row_of(ln), V, true);
+                g.bins = !a.radix_nucleus;
                 r = g.run(c_in, a.inv_tau, a.top_k, a.top_p);
             }
             if (tid == 0) write_result(a, ln, r, done ? PATH_COMPACT : PATH_GENERAL);

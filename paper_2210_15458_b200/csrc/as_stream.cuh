@@ -64,7 +64,6 @@ struct StreamSmemT {
             int cidx[CAPV];                             // vector index of each hit vector
             unsigned long long cand[SK_CAP + 4];           // (key << 32) | ~index, any order
         } ep;
-        GenericSmem<SK_NT> gen;
     } u;
     double exp_tbl[64];
     double red_d[SK_NW];
@@ -353,13 +352,15 @@ __device__ __forceinline__ void reread_row(uint4* staging, const char* row, int 
 
 // Nucleus-only lane whose nucleus reaches below the exact depth of the list (key >= t0key).
 // The row is read again from global memory (it was just streamed, so mostly from L2):
-//   1. masses and counts of the elements below the old threshold go into a histogram over
-//      y = (x - max) * scale2, 128 bins per unit of log2 mass, 8 units deep (a list of a few
-//      hundred candidates never reaches further down, and the fewer elements fall into the
-//      window, the fewer shared-memory atomics the pass costs);
-//   2. the bins are taken from the top until their mass covers what the nucleus still lacks
-//      (with a margin for the fp32 sums): that gives a lower threshold t1 below which no
-//      nucleus token can lie, if the candidates still fit the list;
+//   1. the elements below the old threshold are counted into bins over y = (x - max) * scale2,
+//      128 bins per unit of log2 mass, 8 units deep (a list of a few hundred candidates never
+//      reaches further down, and the fewer elements fall into the window, the fewer shared-memory
+//      atomics the pass costs; counts only: integer additions to shared memory are native, fp32
+//      ones are compare-and-swap loops);
+//   2. the bins are taken from the top until the mass they hold at the least (count times the
+//      mass at the bin's lower edge) covers what the nucleus still lacks, with a margin: that
+//      gives a lower threshold t1 below which no nucleus token can lie, if the candidates still
+//      fit the list;
 //   3. everything >= t1 is collected afresh, the rest summed in fp32, and the exact epilogue
 //      runs again.  Returns false if the window or the list capacity does not suffice.
 constexpr int DP_NB = 1024;
@@ -376,11 +377,17 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2,
     const int nvec_full = (V * Tr::BYTES) >> 4;           // whole 16-byte vectors
     const float lmaxf = Tr::value_f(gmax);
     const float y0 = (t0f - lmaxf) * scale2;
-    float* hmass = reinterpret_cast<float*>(sm.u.ep.v.cvec);
-    int* hcnt = reinterpret_cast<int*>(hmass + DP_NB);
+    int* hcnt = reinterpret_cast<int*>(sm.u.ep.v.cvec) + DP_NB;        // (the staging area starts past 2 * DP_NB words)
     const double list_mass = sm.list_mass;
+    {
+        // every token that could still join weighs less than the old threshold does: if even that many
+        // of them as the list has room for cannot cover what the nucleus lacks, the pass is pointless
+        const double lacking = top_p * (list_mass + tailsum) - list_mass;
+        const double room = (double)(SK_CAP - 8 - sm.cand_count);
+        if (lacking > room * (double)ex2_approx(y0) * 1.001) { ASX_COUNT(2); return false; }
+    }
     SyncC::sync();                                         // the epilogue's arrays are dead
-    for (int i = tid; i < DP_NB; i += NT) { hmass[i] = 0.f; hcnt[i] = 0; }
+    for (int i = tid; i < DP_NB; i += NT) hcnt[i] = 0;
     if (tid == 0) sm.cand_count = 0;
     for (int i = tid; i < SK_CAP + 4; i += NT) sm.u.ep.cand[i] = 0ull;
     SyncC::sync();
@@ -403,8 +410,7 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2,
             const float d = (y0 - y) * DP_BINS_PER_UNIT;
             if (d < (float)DP_NB) {
                 const int bin = (int)d;
-                atomicAdd(&hcnt[ASX_AT(bin, DP_NB, 20)], 1);
-                atomicAdd(&hmass[ASX_AT(bin, DP_NB, 21)], ex2_approx(y));
+                red_shared_add(&hcnt[ASX_AT(bin, DP_NB, 20)], 1);
             }
         }
     });
@@ -414,16 +420,18 @@ __device__ __noinline__ bool deepen_nucleus(StreamSmem& sm, int V, float scale2,
         const double target = top_p * (list_mass + tailsum);
         const double need = (target - list_mass) * 1.002 + 1e-7 * target;
         constexpr int PER = DP_NB / 32;
+        // least mass of an element of bin i: at the bin's lower edge, y0 - (i + 1) / 128
+        auto least = [&](int i) -> double { return (double)hcnt[i] * (double)ex2_approx(y0 - (float)(i + 1) / DP_BINS_PER_UNIT); };
         double m = 0.0;
         int n = 0;
-        for (int i = 0; i < PER; ++i) { m += (double)hmass[lane * PER + i]; n += hcnt[lane * PER + i]; }
+        for (int i = 0; i < PER; ++i) { m += least(lane * PER + i); n += hcnt[lane * PER + i]; }
         const double mi = warp_incl_scan_d(m, lane);
         const int ni = warp_incl_scan_i(n, lane);
         double run = mi - m;
         int cnt = ni - n;
         int found = -1, found_cnt = 0;
         for (int i = 0; i < PER; ++i) {
-            run += (double)hmass[lane * PER + i];
+            run += least(lane * PER + i);
             cnt += hcnt[lane * PER + i];
             if (found < 0 && run >= need) { found = lane * PER + i; found_cnt = cnt; }
         }
@@ -529,6 +537,66 @@ __device__ __forceinline__ void mask_lead(uint4& q, int lead) {
         }
     }
     q = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Token of a lane that the streaming kernel leaves to deferred_lanes_kernel (never seen by a caller).
+constexpr int LANE_DEFERRED = -2;
+
+// One lane's outputs (thread 0 of the CTA that decided it).  XP: the decoder state is narrowed to the
+// token's cells [xp_lo, xp_hi) and refilled with digits of the code.
+template <bool GATHER, bool XP>
+__device__ __forceinline__ void finish_lane(const StepArgs& a, int ln, const LaneResult& r, int path,
+                                            unsigned long long xp_lo, unsigned long long xp_hi) {
+    if (XP) {
+        a.tokens[(size_t)ln * a.tok_stride] = r.token;
+        if (r.status == ST_OK) {         // narrow the interval to the token's cells, shift digits in
+            XpState xs;
+            xs.range = a.xp_state[(size_t)ln * 4]; xs.code = a.xp_state[(size_t)ln * 4 + 1];
+            xs.q = a.xp_state[(size_t)ln * 4 + 2]; xs.packed = a.xp_state[(size_t)ln * 4 + 3];
+            xp_advance(xs, xp_lo, xp_hi, (unsigned)a.xp_N);
+            a.xp_state[(size_t)ln * 4] = xs.range; a.xp_state[(size_t)ln * 4 + 1] = xs.code;
+            a.xp_state[(size_t)ln * 4 + 2] = xs.q; a.xp_state[(size_t)ln * 4 + 3] = xs.packed;
+        } else if (a.diag.lane_status) {
+            a.diag.lane_status[ln] = r.status;
+        }
+    } else if (GATHER) {
+        a.tokens[(size_t)ln * a.tok_stride] = r.token;
+        a.codes_out[ln] = r.code_out;
+        if (a.diag.lane_status && r.status != ST_OK) a.diag.lane_status[ln] = r.status;
+    } else {
+        write_result(a, ln, r, path);
+    }
+}
+
+// The lanes the streaming kernel left undecided (token == LANE_DEFERRED), through the general
+// routine on their rows in global memory (just streamed: mostly in L2).  Launched after every
+// launch of the streaming kernel, with the same arguments; CTA b looks at lanes b, b + grid, ...
+// and leaves at once where none is marked.
+constexpr int DL_NT = 256;
+template <int DT, bool GATHER, bool XP>
+__global__ void __launch_bounds__(DL_NT, 4) deferred_lanes_kernel(const StepArgs a) {
+    using Tr = Traits<DT>;
+    __shared__ GenericSmem<DL_NT> sm;
+    pdl_allow_next();
+    pdl_wait_prev();
+    for (int ln = blockIdx.x; ln < a.lanes; ln += gridDim.x) {
+        if (a.tokens[(size_t)ln * (GATHER ? a.tok_stride : 1)] != LANE_DEFERRED) continue;    // (uniform over the CTA)
+        const int ri = GATHER ? a.row_idx[(size_t)ln * a.idx_stride] : ln;
+        const char* row = reinterpret_cast<const char*>(a.logits) + (size_t)ri * (size_t)a.ld * Tr::BYTES;
+        const bool vec_ok = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
+        GenericLane<DT, DL_NT> g(sm, row, a.V, vec_ok);
+        g.bins = !a.radix_nucleus;
+        LaneResult r;
+        if (XP) {
+            XpState xs = {XP_RANGE_TOP, 0ull, 0ull, 0ull};
+            xs.range = a.xp_state[(size_t)ln * 4]; xs.code = a.xp_state[(size_t)ln * 4 + 1];
+            r = g.run_xp(xp_target(xs), a.inv_tau, a.top_k, a.top_p);      // (the state was checked by the streaming kernel)
+        } else {
+            r = g.run(lane_code(a, ln), a.inv_tau, a.top_k, a.top_p);
+        }
+        if (threadIdx.x == 0) finish_lane<GATHER, XP>(a, ln, r, PATH_GENERAL, sm.xp_lo, sm.xp_hi);
+        __syncthreads();
+    }
 }
 
 template <int DT, int CAPV, int MINB, bool UA = false, bool GATHER = false, bool XP = false>
@@ -795,20 +863,16 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         if (UA) geom(lead, bulk_bytes_l, bulk_vec_l, tail_elems_l, nsl_l);
         const char* vrow = row - lead * Tr::BYTES;     // where the copies start
 
-        // Lanes the candidate list cannot decide end in ONE call of the general routine (kept out
-        // of line so that the hot path stays small).
-        const void* general_row = nullptr;      // set = run the general routine on this row
-        bool general_vec_ok = true;
-        bool general_release = false;           // resident row in the ring: release its stages after
+        // Lanes the candidate list cannot decide are left to the kernel that follows this one on the
+        // stream (deferred_lanes_kernel: the general routine): their token is set to LANE_DEFERRED and
+        // nothing else of theirs is written.  The general routine is not part of this kernel: even out
+        // of line its register needs weighed on the allocation of the streaming passes (2-10 % of
+        // their time), and the lanes that need it are spread over the whole machine that way.
         LaneResult r;
         int path = PATH_COMPACT;
         bool decided = false;
+        bool whole_row = false;                 // a row that would have to be kept whole (no usable cut)
 
-        if (!staged_ok(ln)) {        // unaligned row: general routine from global memory
-            general_row = row;
-            general_vec_ok = false;
-        }
-        if (UA && lead) general_vec_ok = false;       // should the general routine be needed after all
         if (tid == 0) { sm.vec_count = 0; sm.cand_count = 0; }
         // the candidate array starts zeroed: entries past the count rank below every candidate,
         // which the epilogue's 4-wide rank loop relies on
@@ -816,7 +880,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
 
         // ragged end of the row (< 16 bytes): one padded vector read straight from global memory
         uint4 qt = make_uint4(ninf_word, ninf_word, ninf_word, ninf_word);
-        if (tail_elems_l > 0 && tid == 0 && !general_row) {
+        if (tail_elems_l > 0 && tid == 0) {
             uint32_t w[4];
             // (a row shorter than a granule has its lead in this vector: those elements stay masked)
             const int skip = (UA && bulk_vec_l == 0) ? lead : 0;
@@ -866,9 +930,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
 
         ASX_MARK(0);
         ASX_CTA(1);
-        if (general_row) {
-            // nothing was staged for this lane
-        } else if (resident) {
+        if (resident) {
             // ---- all stages land; max pass from shared memory.  Each vector's own maximum stays
             //      in a register, so the hit test after the threshold needs no second pass.
             float pm[SK_RES_STAGES * SK_VPT];
@@ -914,19 +976,9 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
                 decided = true;
                 for (int s = 0; s < nsl_l; ++s) release(s);
             } else if (!cut) {
-                // no cut: every token is kept; the general routine scans the row in shared memory
-                if (UA && lead) {
-                    general_row = row;                 // (a row with a lead: from global memory)
-                } else if (tail_elems_l > 0 && tid < tail_elems_l) {
-                    if (DT == DT_BF16)
-                        reinterpret_cast<unsigned short*>(ring + bulk_bytes_l)[tid] =
-                            reinterpret_cast<const unsigned short*>(vrow + bulk_bytes_l)[tid];
-                    else
-                        reinterpret_cast<uint32_t*>(ring + bulk_bytes_l)[tid] =
-                            reinterpret_cast<const uint32_t*>(vrow + bulk_bytes_l)[tid];
-                }
-                if (!(UA && lead)) general_row = ring;
-                general_release = true;
+                // (launches of this kernel always carry a cut it can serve; a row without one is deferred)
+                whole_row = true;
+                for (int s = 0; s < nsl_l; ++s) release(s);
             } else {
                 ref = Tr::value_f(gmax);
                 t0f = Tr::value_f(t0key);
@@ -1020,7 +1072,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
         const bool listed = !(resident && cut && !want_tail);
         if (listed) SyncC::sync();
         const int nvh = listed ? sm.vec_count : 0;
-        bool list_ok = !decided && !general_row && nvh <= SK_CAPV;
+        bool list_ok = !decided && !whole_row && nvh <= SK_CAPV;
         if (list_ok) {
             for (int i = tid; i < nvh; i += NT) {
                 const uint4 q = sm.u.ep.v.cvec[ASX_AT(i, SK_CAPV, 42)];
@@ -1031,7 +1083,7 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             // the ragged last vector lives in thread 0's registers
             if (tail_elems_l > 0 && tid == 0) push_vec(qt, bulk_vec_l * E - lead, t0f, t0key, want_tail, ref, tail);
         }
-        if (!list_ok && !decided && !general_row && nvh > SK_CAPV && !(UA && lead) && !*(volatile int*)&sm.poisoned) {
+        if (!list_ok && !decided && !whole_row && nvh > SK_CAPV && !(UA && lead) && !*(volatile int*)&sm.poisoned) {
             // more hit vectors than the list holds: take the candidates in one more pass, against
             // the threshold that the whole row's subset maxima give now
             ASX_COUNT(8);
@@ -1090,36 +1142,11 @@ __global__ void __launch_bounds__(SK_THREADS, MINB) step_stream_kernel(const Ste
             ASX_COUNT(5);
             if (nvh > SK_CAPV) ASX_COUNT(6);
             if (sm.cand_count > SK_CAP) ASX_COUNT(7);
-            if (!general_row) general_row = row;          // the row again, from global memory (L2)
-            SyncC::sync();
-            GenericLane<DT, NT, SyncC> gl(sm.u.gen, general_row, V, general_vec_ok);
-            bool from_gen = false;
-            if (XP) { r = gl.run_xp(tcell, a.inv_tau, a.top_k, a.top_p); from_gen = true; }
-            else r = gl.run(c_in, a.inv_tau, a.top_k, a.top_p);
-            if (XP && tid == 0 && from_gen) { sm.xp_lo = sm.u.gen.xp_lo; sm.xp_hi = sm.u.gen.xp_hi; }
-            path = PATH_GENERAL;
-            if (general_release)
-                for (int s = 0; s < nsl_l; ++s) release(s);
         }
-        if (resident && staged_ok(ln)) advance(nsl_l);
+        if (resident) advance(nsl_l);
         if (tid == 0) {
-            if (XP) {
-                a.tokens[(size_t)ln * a.tok_stride] = r.token;
-                if (r.status == ST_OK) {         // narrow the interval to the token's cells, shift digits in
-                    xs.q = a.xp_state[(size_t)ln * 4 + 2]; xs.packed = a.xp_state[(size_t)ln * 4 + 3];
-                    xp_advance(xs, sm.xp_lo, sm.xp_hi, (unsigned)a.xp_N);
-                    a.xp_state[(size_t)ln * 4] = xs.range; a.xp_state[(size_t)ln * 4 + 1] = xs.code;
-                    a.xp_state[(size_t)ln * 4 + 2] = xs.q; a.xp_state[(size_t)ln * 4 + 3] = xs.packed;
-                } else if (a.diag.lane_status) {
-                    a.diag.lane_status[ln] = r.status;
-                }
-            } else if (GATHER) {
-                a.tokens[(size_t)ln * a.tok_stride] = r.token;
-                a.codes_out[ln] = r.code_out;
-                if (a.diag.lane_status && r.status != ST_OK) a.diag.lane_status[ln] = r.status;
-            } else {
-                write_result(a, ln, r, path);
-            }
+            if (!decided) a.tokens[(size_t)ln * (GATHER ? a.tok_stride : 1)] = LANE_DEFERRED;
+            else finish_lane<GATHER, XP>(a, ln, r, path, sm.xp_lo, sm.xp_hi);
         }
         SyncC::sync();
         ASX_MARK(12);

@@ -468,6 +468,60 @@ def test_step_flat_and_adversarial_rows_fall_back(B, orc):
 
 
 @pytest.mark.parametrize("dtype", [F32, BF16])
+def test_step_wide_nucleus_through_value_bins(B, orc, dtype):
+    # nuclei of hundreds to tens of thousands of tokens (flat rows), with ties at the threshold,
+    # masked tokens and unaligned rows: the general routine settles them through bins of the logit
+    # value; the same lanes through its radix select must give the very same tokens and kept counts
+    rng = np.random.default_rng(4242)
+    cases = [(128256, 3.0, 0.8, 0.9), (50001, 1.0, 1.0, 0.5), (50001, 0.05, 1.0, 0.97),
+             (32000, 3.0, 2.0, 0.99), (9001, 2.0, 1.0, 0.3), (4099, 1.5, 1.0, 0.8)]
+    for V, sigma, temp, p in cases:
+        lanes = 10
+        x = rng.normal(0, sigma, (lanes, V)).astype(np.float32)
+        x[1, ::3] = -np.inf                                       # masked tokens
+        x[2] = np.round(x[2] * 2) / 2                             # few distinct values: ties everywhere
+        arr = _store(x, dtype)
+        codes = rng.random(lanes)
+        codes[3] = 0.0
+        codes[4] = 1.0 - 2.0 ** -53
+        ref = orc.step(arr, dtype, codes, temp, 0, p, threads=8)
+        assert V < 32000 or np.median(ref.n_kept) > 300
+        got = {}
+        for name, key, val in [("default", None, 0), ("general", B.TUNE_STEP_PATH, 1)]:
+            for radix in (0, 1):
+                try:
+                    if key is not None:
+                        B.as_tune(key, val)
+                    B.as_tune(B.TUNE_RADIX_NUCLEUS, radix)
+                    tok, c2, pt, nk, st = gpu_step(B, arr, dtype, codes, temp, 0, p)
+                finally:
+                    B.as_tune(B.TUNE_RADIX_NUCLEUS, 0)
+                    if key is not None:
+                        B.as_tune(key, 0)
+                what = "wide nucleus V=%d %s radix=%d" % (V, name, radix)
+                compare_step(ref, tok, c2, pt, nk, st, what=what)
+                # with tens of thousands of kept tokens every code lies within the usual band of a CDF
+                # boundary; both sides compute in fp64, so a band of 1e-9 still leaves rounding room
+                near = (ref.d_tok > 1e-9) & (ref.d_topp > 1e-9) & (ref.status == 0)
+                assert near.sum() >= lanes - 2, what
+                assert (tok[near] == ref.tokens[near]).all(), what
+                assert (nk[near] == ref.n_kept[near]).all(), what
+                np.testing.assert_allclose(pt[near], ref.p_tok[near], rtol=1e-9, err_msg=what)
+                np.testing.assert_allclose(c2[near], ref.codes[near], rtol=0, atol=1e-5, err_msg=what)
+                got[(name, radix)] = (tok, nk, c2)
+        for name in ("default", "general"):
+            assert (got[(name, 0)][0] == got[(name, 1)][0]).all() and (got[(name, 0)][1] == got[(name, 1)][1]).all()
+            np.testing.assert_allclose(got[(name, 0)][2], got[(name, 1)][2], rtol=0, atol=1e-6)
+    # rows off the 16-byte grid (element-wise loads in the general routine)
+    full = _store(rng.normal(0, 1.0, (9, 6007)), dtype)
+    try:
+        B.as_tune(B.TUNE_STEP_PATH, 1)
+        check(B, orc, full, dtype, rng.random(9), 1.0, 0, 0.9, V=6001, what="wide nucleus, odd pitch")
+    finally:
+        B.as_tune(B.TUNE_STEP_PATH, 0)
+
+
+@pytest.mark.parametrize("dtype", [F32, BF16])
 def test_step_nucleus_deeper_than_the_list(B, orc, dtype):
     # nucleus-only lanes whose nucleus holds a few hundred tokens: more than the exact depth of the
     # candidate list, so the threshold has to be lowered once from the mass histogram; plus lanes
