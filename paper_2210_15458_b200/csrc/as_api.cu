@@ -177,7 +177,18 @@ static int launch_stream_ua(const StepArgs& a, int stages, int sms, int want_per
     cfd.stream = st;
     cfd.attrs = attr;
     cfd.numAttrs = g_tune_serial ? 0 : 1;
-    e = cudaLaunchKernelEx(&cfd, deferred_lanes_kernel<DT, GATHER, XP>, a);
+    // rows of up to 96 KB are staged in shared memory (two CTAs per SM then)
+    static bool dl_attr_set[64] = {false};
+    auto dkern = deferred_lanes_kernel<DT, GATHER, XP>;
+    if (!dl_attr_set[dev]) {
+        e = cudaFuncSetAttribute(dkern, cudaFuncAttributeMaxDynamicSharedMemorySize, DL_STAGE_MAX);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(deferred lanes kernel)");
+        dl_attr_set[dev] = true;
+    }
+    const long long row_span = (long long)a.V * (DT == DT_BF16 ? 2 : 4) + 15 + 16;
+    const int stage_bytes = row_span <= DL_STAGE_MAX ? (int)(row_span & ~15LL) : 0;
+    cfd.dynamicSmemBytes = (size_t)stage_bytes;
+    e = cudaLaunchKernelEx(&cfd, dkern, a, stage_bytes);
     if (e != cudaSuccess) return cuda_fail(e, "deferred lanes kernel launch");
     return AS_OK;
 }

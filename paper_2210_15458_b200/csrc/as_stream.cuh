@@ -25,8 +25,9 @@
 // order, CDF prefix, crossing, rescale (Algorithm 1: w_i, (m, M),
 // c <- (c - m)/(M - m)).  For nucleus-only lanes the masses of everything else
 // are summed in fp32 (they only enter the nucleus target top_p * Z1).  Lanes the
-// list cannot decide (too many hits, nucleus deeper than the exact depth,
-// unaligned rows) go to GenericLane, which reads the row from global memory (L2).
+// list cannot decide (a nucleus deeper than the list can be made, too many ties)
+// are marked and served by deferred_lanes_kernel, launched right after this kernel:
+// GenericLane on the row in global memory (L2), four CTAs per SM.
 #pragma once
 #include "as_staged.cuh"
 
@@ -571,18 +572,33 @@ __device__ __forceinline__ void finish_lane(const StepArgs& a, int ln, const Lan
 // The lanes the streaming kernel left undecided (token == LANE_DEFERRED), through the general
 // routine on their rows in global memory (just streamed: mostly in L2).  Launched after every
 // launch of the streaming kernel, with the same arguments; CTA b looks at lanes b, b + grid, ...
-// and leaves at once where none is marked.
+// and leaves at once where none is marked.  `stage_bytes` > 0: the row fits that much dynamic shared
+// memory and is copied there first (from the 16-byte boundary below its start), so that the routine's
+// passes run from shared memory.
 constexpr int DL_NT = 256;
+constexpr int DL_STAGE_MAX = 96 * 1024 + 32;     // rows up to 96 KB are staged
 template <int DT, bool GATHER, bool XP>
-__global__ void __launch_bounds__(DL_NT, 4) deferred_lanes_kernel(const StepArgs a) {
+__global__ void __launch_bounds__(DL_NT, 4) deferred_lanes_kernel(const StepArgs a, const int stage_bytes) {
     using Tr = Traits<DT>;
     __shared__ GenericSmem<DL_NT> sm;
+    extern __shared__ uint4 dl_stage[];
     pdl_allow_next();
     pdl_wait_prev();
     for (int ln = blockIdx.x; ln < a.lanes; ln += gridDim.x) {
         if (a.tokens[(size_t)ln * (GATHER ? a.tok_stride : 1)] != LANE_DEFERRED) continue;    // (uniform over the CTA)
         const int ri = GATHER ? a.row_idx[(size_t)ln * a.idx_stride] : ln;
         const char* row = reinterpret_cast<const char*>(a.logits) + (size_t)ri * (size_t)a.ld * Tr::BYTES;
+        if (stage_bytes > 0) {
+            const int lead = (int)(reinterpret_cast<uintptr_t>(row) & 15);
+            const uint4* src = reinterpret_cast<const uint4*>(row - lead);
+            const int nfull = (lead + a.V * Tr::BYTES) >> 4;                 // whole 16-byte vectors
+            for (int i = threadIdx.x; i < nfull; i += DL_NT) dl_stage[i] = src[i];
+            // (the ragged end byte by byte: reading its whole vector could cross the end of the allocation)
+            char* dst = reinterpret_cast<char*>(dl_stage);
+            for (int i = (nfull << 4) + threadIdx.x; i < lead + a.V * Tr::BYTES; i += DL_NT) dst[i] = (row - lead)[i];
+            __syncthreads();
+            row = dst + lead;
+        }
         const bool vec_ok = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
         GenericLane<DT, DL_NT> g(sm, row, a.V, vec_ok);
         g.bins = !a.radix_nucleus;
