@@ -93,6 +93,17 @@ def test_invalid_arguments_are_rejected_on_the_host(L):
     assert L.as_step_host_work_bytes(0, 4, 10) >= 4 * 10 * 4 + 4 * 24
 
 
+def test_tuning_keys_of_the_binding_match_the_header(L):
+    import re
+    from paper_2210_15458_b200 import binding as B
+    header = open(os.path.join(ROOT, "include", "arith_sampling.h")).read()
+    keys = dict(re.findall(r"#define AS_TUNE_(\w+) (\d+)", header))
+    assert len(keys) >= 9 and len(set(keys.values())) == len(keys)
+    for name, value in keys.items():
+        assert getattr(B, "TUNE_" + name) == int(value), name
+    assert L.as_tune(B.TUNE_RADIX_NUCLEUS, 2) == B.ERR_INVALID_ARG and L.as_tune(B.TUNE_RADIX_NUCLEUS, 0) == B.OK
+
+
 def test_no_device_means_an_error_not_a_fallback(L):
     import torch
     if torch.cuda.is_available():
