@@ -584,6 +584,14 @@ __global__ void __launch_bounds__(DL_NT, 4) deferred_lanes_kernel(const StepArgs
     extern __shared__ uint4 dl_stage[];
     pdl_allow_next();
     pdl_wait_prev();
+    {
+        // this CTA's lanes looked at side by side, one per thread: usually none is marked, and a walk
+        // through them one dependent load after the other would be the whole cost of this kernel
+        int any = 0;
+        for (long long ln = blockIdx.x + (long long)threadIdx.x * gridDim.x; ln < a.lanes; ln += (long long)DL_NT * gridDim.x)
+            any |= a.tokens[(size_t)ln * (GATHER ? a.tok_stride : 1)] == LANE_DEFERRED;
+        if (!__syncthreads_or(any)) return;
+    }
     for (int ln = blockIdx.x; ln < a.lanes; ln += gridDim.x) {
         if (a.tokens[(size_t)ln * (GATHER ? a.tok_stride : 1)] != LANE_DEFERRED) continue;    // (uniform over the CTA)
         const int ri = GATHER ? a.row_idx[(size_t)ln * a.idx_stride] : ln;
